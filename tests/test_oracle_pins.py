@@ -1,0 +1,328 @@
+"""Pins for the float64 CPU oracle (no GPU needed).
+
+The paper prints no numbers for the plasticity path, so the oracle is pinned to
+what the mathematics fixes: hand-derived closed forms (tests/golden), exact
+rational arithmetic, a BLAS route, invariants, a negative control, closed-form
+and pair-wise brute-force slopes, and hand-replayed Algorithm 1 traces.
+"""
+from fractions import Fraction
+from pathlib import Path
+
+import math
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2201_06227_b200 import workloads as wl
+
+GOLDEN = Path(__file__).parent / "golden"
+
+
+def bits_of(rows):
+    """Exact bf16 bits of a small float matrix (every value must be bf16-exact)."""
+    t = torch.tensor(rows, dtype=torch.float32)
+    tb = t.to(torch.bfloat16)
+    assert torch.equal(tb.to(torch.float32), t), "fixture value is not exact in bfloat16"
+    return wl.bf16_bits(tb)
+
+
+def rand_bits(b, d, seed, relu=False, scale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    x = torch.randn((b, d), generator=g) * scale
+    if relu:
+        x = torch.relu(x)
+    return wl.bf16_bits(x.to(torch.bfloat16))
+
+
+def as_f64(bits):
+    return wl.from_bits(bits).to(torch.float64).numpy()
+
+
+# ----------------------------------------------------------------------------- closed forms
+
+def _parse_matrix(s):
+    return [[float(Fraction(v)) for v in row.split()] for row in s.split(";")]
+
+
+def _closed_form_cases():
+    for line in (GOLDEN / "sp_loss_closed_forms.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        name, b, d, at, ar, exp = [f.strip() for f in line.split("|")]
+        yield pytest.param(int(b), int(d), _parse_matrix(at), _parse_matrix(ar), float(exp), id=name)
+
+
+@pytest.mark.parametrize("b,d,at,ar,expected", list(_closed_form_cases()))
+def test_closed_form_fixture(b, d, at, ar, expected):
+    A, R = bits_of(at), bits_of(ar)
+    assert A.shape == (b, d)
+    assert oracle.sp_loss(A, R) == pytest.approx(expected, abs=1e-15)
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_b2_angle_formula(seed):
+    """b = 2: rows of the normalised Gram are unit vectors in the plane, so the loss is
+    (1/2)(2 - cos(thetaT - thetaR) - cos(phiT - phiR)) with theta, phi the row angles."""
+    A, R = rand_bits(2, 16, seed), rand_bits(2, 16, 100 + seed)
+
+    def angles(bits):
+        X = as_f64(bits)
+        a, c, e = X[0] @ X[0], X[0] @ X[1], X[1] @ X[1]
+        return math.atan2(c, a), math.atan2(e, c)
+
+    tT, pT = angles(A)
+    tR, pR = angles(R)
+    expected = 0.5 * (2.0 - math.cos(tT - tR) - math.cos(pT - pR))
+    assert oracle.sp_loss(A, R) == pytest.approx(expected, rel=1e-12, abs=1e-15)
+
+
+@pytest.mark.parametrize("b", [2, 3, 4, 9, 16])
+def test_onehot_vs_identical_rows(b):
+    """Orthogonal rows give G~_T = I, identical rows give G~_R = 1/sqrt(b) everywhere:
+    P = (1/b)[(1 - 1/sqrt b)^2 + (b-1)/b]."""
+    at = np.eye(b).tolist()
+    ar = [[1.0, 2.0, 0.5] + [0.0] * (b - 3 if b > 3 else 0)] * b
+    ar = [r[:b] if b >= 3 else r[:b] for r in ar]
+    A, R = bits_of(at), bits_of(ar)
+    expected = ((1 - 1 / math.sqrt(b)) ** 2 + (b - 1) / b) / b
+    assert oracle.sp_loss(A, R) == pytest.approx(expected, rel=1e-13)
+
+
+# ----------------------------------------------------------------------------- exact arithmetic
+
+@pytest.mark.parametrize("b,d,seed", [(2, 5, 0), (3, 7, 1), (5, 13, 2)])
+def test_gram_exact_rationals(b, d, seed):
+    """bf16 values are dyadic rationals: the Gram matrix is exact in Fractions."""
+    bits = rand_bits(b, d, seed)
+    X = as_f64(bits)
+    F = [[Fraction(float(v)) for v in row] for row in X]
+    G = oracle.gram(bits)
+    for i in range(b):
+        for j in range(b):
+            exact = sum(F[i][k] * F[j][k] for k in range(d))
+            assert G[i, j] == pytest.approx(float(exact), rel=1e-14, abs=1e-300)
+    # asymmetric index use (a transposed or dropped operand) shows here:
+    assert G[0, 1] == pytest.approx(float(sum(F[0][k] * F[1][k] for k in range(d))), rel=1e-14)
+
+
+def test_gram_not_transposed():
+    """A is b x d (samples x features): A A^T is b x b, not d x d."""
+    bits = bits_of([[1, 2, 3], [4, 5, 6]])
+    G = oracle.gram(bits)
+    assert G.shape == (2, 2)
+    assert G.tolist() == [[14.0, 32.0], [32.0, 77.0]]
+
+
+# ----------------------------------------------------------------------------- library route
+
+@pytest.mark.parametrize("b,d,relu", [(8, 4096, True), (17, 72, False), (64, 1000, True), (100, 333, False)])
+def test_blas_route(b, d, relu):
+    """G is a textbook SYRK; the same steps through numpy's float64 matmul agree."""
+    A, R = rand_bits(b, d, 7, relu), rand_bits(b, d, 8, relu)
+    loss, gt, gr = oracle.sp_loss(A, R, return_grams=True)
+
+    def route(bits):
+        X = as_f64(bits)
+        G = X @ X.T
+        return G / np.maximum(np.linalg.norm(G, axis=1, keepdims=True), oracle.EPS)
+
+    nt, nr = route(A), route(R)
+    np.testing.assert_allclose(gt, nt, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(gr, nr, rtol=0, atol=1e-13)
+    assert loss == pytest.approx(((nt - nr) ** 2).sum() / b ** 2, rel=1e-10, abs=1e-18)
+    # algebraically different route: P = (2/b)(1 - mean_i cos(angle between rows i))
+    cosines = (nt * nr).sum(axis=1)
+    assert loss == pytest.approx(2.0 / b * (1.0 - cosines.mean()), rel=1e-8, abs=1e-15)
+
+
+def test_gram_row_matches_gram():
+    bits = rand_bits(9, 257, 3)
+    G = oracle.gram(bits)
+    for i in (0, 4, 8):
+        np.testing.assert_allclose(oracle.gram_row(bits, i), G[i], rtol=1e-14)
+
+
+# ----------------------------------------------------------------------------- invariants
+
+@pytest.mark.parametrize("seed", range(3))
+def test_invariants(seed):
+    b, d = 12, 96
+    A, R = rand_bits(b, d, seed, relu=True), rand_bits(b, d, 50 + seed, relu=True)
+    base, gt, gr = oracle.sp_loss(A, R, return_grams=True)
+    # identical inputs: exactly zero
+    assert oracle.sp_loss(A, A) == 0.0
+    # bounds: entries in [-1, 1], unit rows, positive diagonal, 0 <= P <= 2/b for ReLU inputs
+    for g in (gt, gr):
+        assert np.all(np.abs(g) <= 1 + 1e-15)
+        np.testing.assert_allclose(np.linalg.norm(g, axis=1), 1.0, rtol=1e-13)
+        assert np.all(np.diag(g) > 0)
+    assert 0.0 <= base <= 2.0 / b
+    # global scalar on either side (power of two is exact in bf16): unchanged
+    A4 = wl.bf16_bits(wl.from_bits(A) * 4.0)
+    R8 = wl.bf16_bits(wl.from_bits(R) * 0.125)
+    assert oracle.sp_loss(A4, R) == pytest.approx(base, rel=1e-12)
+    assert oracle.sp_loss(A, R8) == pytest.approx(base, rel=1e-12)
+    # feature permutation (flatten order is immaterial), even a different one per side
+    p1 = np.random.default_rng(seed).permutation(d)
+    p2 = np.random.default_rng(seed + 9).permutation(d)
+    assert oracle.sp_loss(A[:, p1], R[:, p2]) == pytest.approx(base, rel=1e-11)
+    # the same sample permutation on both sides
+    ps = np.random.default_rng(seed + 5).permutation(b)
+    assert oracle.sp_loss(A[ps], R[ps]) == pytest.approx(base, rel=1e-11)
+    # symmetric in its two arguments
+    assert oracle.sp_loss(R, A) == pytest.approx(base, rel=1e-14)
+
+
+def test_general_bound_signed_inputs():
+    b = 10
+    A, R = rand_bits(b, 40, 1), rand_bits(b, 40, 2)
+    assert 0.0 <= oracle.sp_loss(A, R) <= 4.0 / b
+
+
+def test_rotation_invariance():
+    """An orthogonal map of the feature axis leaves G, hence P, unchanged.  A signed
+    permutation with a Hadamard block keeps every value exact in bf16."""
+    b, d = 6, 8
+    g = torch.Generator().manual_seed(11)
+    X = torch.randint(-4, 5, (b, d), generator=g).to(torch.float32)
+    Y = torch.randint(-4, 5, (b, d), generator=g).to(torch.float32)
+    H2 = torch.tensor([[1.0, 1.0], [1.0, -1.0]])
+    H8 = torch.kron(torch.kron(H2, H2), H2)            # H8 H8^T = 8 I : orthogonal up to a scalar
+    base = oracle.sp_loss(bits_of(X.tolist()), bits_of(Y.tolist()))
+    rot = oracle.sp_loss(bits_of((X @ H8).tolist()), bits_of((Y @ H8).tolist()))
+    assert base > 0
+    assert rot == pytest.approx(base, rel=1e-12)
+
+
+def test_negative_control_row_scaling_changes_loss():
+    """Rows of G are normalised, not rows of A: scaling one sample DOES change P.
+    (Cosine similarity of the activations would be blind to it.)"""
+    A, R = rand_bits(6, 64, 21, relu=True), rand_bits(6, 64, 22, relu=True)
+    base = oracle.sp_loss(A, R)
+    A2 = A.copy()
+    A2[2] = wl.bf16_bits(wl.from_bits(A[2:3]) * 8.0)[0]
+    assert abs(oracle.sp_loss(A2, R) - base) > 1e-3 * base
+
+
+def test_division_is_by_b_squared():
+    """P scales as 1/b^2 times the Frobenius sum: duplicating the batch (b -> 2b)
+    doubles every squared row norm of G ... checked directly against the sum."""
+    A, R = rand_bits(5, 33, 4), rand_bits(5, 33, 5)
+    loss, gt, gr = oracle.sp_loss(A, R, return_grams=True)
+    assert loss * 25 == pytest.approx(float(((gt - gr) ** 2).sum()), rel=1e-13)
+
+
+def test_zero_row_clamp():
+    A = bits_of([[0, 0, 0], [1, 2, 3]])
+    _, gt, _ = oracle.sp_loss(A, A, return_grams=True)
+    assert np.all(gt[0] == 0.0)
+    assert np.isfinite(gt).all()
+
+
+# ----------------------------------------------------------------------------- smoothing / slope
+
+def test_smooth_is_mean_of_last_min_window():
+    p = np.array([4.0, 2.0, 9.0, 1.0, 5.0, 7.0])
+    W = 3
+    expect = [4.0, 3.0, 5.0, 4.0, 5.0, 13.0 / 3.0]
+    for i, e in enumerate(expect):
+        assert oracle.smooth(p, i, W) == pytest.approx(e, rel=1e-15)
+
+
+@pytest.mark.parametrize("n", [2, 3, 5, 10, 50])
+def test_slope_closed_forms(n):
+    x = np.arange(n, dtype=np.float64)
+    assert oracle.ols_slope(3.0 - 0.25 * x) == pytest.approx(-0.25, rel=1e-13)
+    assert oracle.ols_slope(np.full(n, 7.5)) == 0.0
+    assert oracle.ols_slope(x * x) == pytest.approx(n - 1, rel=1e-12)   # y = x^2 on 0..n-1
+
+
+def test_slope_needs_two_points():
+    assert oracle.ols_slope(np.array([1.0])) == math.inf
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_slope_pairwise_brute_force(seed):
+    """s = sum_{i<j}(x_j-x_i)(y_j-y_i) / sum_{i<j}(x_j-x_i)^2 (an identity of OLS)."""
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(2, 9))
+    y = rng.normal(size=n)
+    num = sum((j - i) * (y[j] - y[i]) for i in range(n) for j in range(i + 1, n))
+    den = sum((j - i) ** 2 for i in range(n) for j in range(i + 1, n))
+    assert oracle.ols_slope(y) == pytest.approx(num / den, rel=1e-12, abs=1e-15)
+    assert oracle.ols_slope(y) == pytest.approx(np.polyfit(np.arange(n), y, 1)[0], rel=1e-10, abs=1e-13)
+
+
+def _tok(v):
+    if v == "x":
+        return None
+    if v in ("inf", "-inf"):
+        return float(v)
+    return float(Fraction(v))
+
+
+def _trace_cases():
+    for line in (GOLDEN / "alg1_traces.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        f = [s.strip() for s in line.split("|")]
+        yield pytest.param(int(f[1]), float(f[2]), bool(int(f[3])),
+                           [float(v) for v in f[4].split()],
+                           [_tok(v) for v in f[5].split()], [_tok(v) for v in f[6].split()],
+                           [_tok(v) for v in f[7].split()], int(f[8]), id=f[0])
+
+
+@pytest.mark.parametrize("W,T,signed,hist,smoothed,slopes,counters,freeze_eval", list(_trace_cases()))
+def test_algorithm1_hand_traces(W, T, signed, hist, smoothed, slopes, counters, freeze_eval):
+    out = oracle.plasticity_replay(hist, W, T, signed_test=signed)
+    assert out["freeze_eval"] == freeze_eval
+    assert out["converged"] == (freeze_eval >= 0)
+    for i, (sm, sl) in enumerate(zip(smoothed, slopes)):
+        if sm is None:
+            assert math.isnan(out["smoothed"][i]) and math.isnan(out["slopes"][i])
+        else:
+            assert out["smoothed"][i] == pytest.approx(sm, rel=1e-6)      # float32 readings
+            assert out["slopes"][i] == pytest.approx(sl, rel=1e-6, abs=1e-7)
+    # counters: replay prefixes and read the final counter of each
+    for i, c in enumerate(counters):
+        if c is None:
+            continue
+        assert oracle.plasticity_replay(hist[: i + 1], W, T, signed_test=signed)["counter"] == c
+
+
+def test_earliest_convergence_is_W():
+    for W in (2, 5, 9):
+        out = oracle.plasticity_replay(np.zeros(30, dtype=np.float32), W, 1e-9)
+        assert out["freeze_eval"] == W
+    # a window of one point has no line to fit: W = 1 never converges
+    assert not oracle.plasticity_replay(np.zeros(30, dtype=np.float32), 1, 1.0)["converged"]
+    # fewer than W+1 readings can never converge
+    assert not oracle.plasticity_replay(np.zeros(5, dtype=np.float32), 5, 1.0)["converged"]
+
+
+def test_linear_history_slope_after_window_fills():
+    """Once the window is full, smoothing a straight line keeps its slope."""
+    W, beta = 6, -0.03125
+    hist = (2.0 + beta * np.arange(40)).astype(np.float32)
+    out = oracle.plasticity_replay(hist, W, 1e-3)
+    np.testing.assert_allclose(out["slopes"][2 * W:], beta, rtol=1e-6)
+    assert not out["converged"]
+
+
+def test_nan_is_never_stale():
+    hist = np.array([1, 1, np.nan, 1, 1, 1, 1, 1, 1, 1, 1, 1], dtype=np.float32)
+    out = oracle.plasticity_replay(hist, 2, 0.5)
+    # NaN poisons the smoothed values for W readings and the fit for W more
+    assert out["freeze_eval"] > 2 + 2
+
+
+def test_larger_T_or_smaller_W_freezes_earlier():
+    """Sensitivity direction stated in Sec. 6.4: smaller W / larger T freeze earlier."""
+    w = wl.WORKLOADS["resnet56"]
+    hist = wl.make_history(w, [1e-2] * 4, H=60)[0]
+    f = lambda W, T: oracle.plasticity_replay(hist, W, T)["freeze_eval"]
+    a, b_, c = f(10, 1e-4), f(10, 1e-3), f(5, 1e-4)
+    assert a != -1 and b_ != -1 and b_ < a
+    assert c != -1 and c < a
+    assert f(10, 1e-12) == -1
