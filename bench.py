@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Benchmark of the plasticity-evaluation path (SP loss of all modules + freezing rule).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one pass of the whole path over one synthetic mini-batch: egeria_sp_loss_batch
+(Gram + finalisation kernels) followed by egeria_plasticity_step.  Prints ONE JSON line.
+With N > 1 (torchrun) every rank evaluates its own replica of the workload on its own
+GPU; there is no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import numpy as np
+import torch
+
+from paper_2201_06227_b200 import workloads as wl
+
+METRIC = "module-evals/s (SP loss, all modules)"
+UNIT = "module-evals/s"
+PEAKS_FILE = ROOT / "MEASURED_PEAKS.json"
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def hbm_peak():
+    try:
+        return float(json.loads(PEAKS_FILE.read_text())["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for (_, l) in self.lines]
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(smax)) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w: wl.Workload, budget_s: float = 12.0, max_modules: int = 4):
+    """Time the CPU oracle, as it stands, on the first modules of the workload."""
+    import oracle
+    oracle.build()
+    done, spent = 0, 0.0
+    for l in range(min(w.M, max_modules)):
+        at, ar = wl.make_module(w, l, "cpu")
+        ta, tr = wl.bf16_bits(at), wl.bf16_bits(ar)
+        t0 = time.perf_counter()
+        oracle.sp_loss(ta, tr)
+        spent += time.perf_counter() - t0
+        done += 1
+        if spent >= budget_s:
+            break
+    # the freezing rule on one reading per module is negligible beside the loss
+    return {"value": done / spent, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"modules 0..{done - 1} of {w.M} ({w.name}), float64 SP loss, {spent:.1f} s"}, spent, done
+
+
+# ----------------------------------------------------------------------------- reference arm (the oracle)
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.WORKLOADS[args.workload]
+    per_step_budget = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(w, budget_s=per_step_budget, max_modules=1)
+    spent_total, done_total, cores, sample = 0.0, 0, 1, ""
+    for _ in range(args.steps):
+        cb, spent, done = oracle_sample(w, budget_s=per_step_budget, max_modules=2)
+        spent_total += spent
+        done_total += done
+        cores, sample = cb["cores"], cb["sample"]
+    value = done_total / spent_total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * spent_total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "b": w.b, "modules": w.M,
+                                        "note": "each step is a bounded sample (first modules) of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def time_workload(eg, w, device, steps, warmup, n_sets, stream, time_gram=True):
+    """Device-timed steps of one workload.  Returns (seconds, gram_ms_per_call, launches_per_step, ctx, data)."""
+    sets = []
+    for s in range(n_sets):
+        at, ar = [], []
+        for l in range(w.M):
+            t, r = wl.make_pair(w.b, w.d[l], w.kind, w.sigma_of(l), w.seed_of(l) + 7919 * s, device)
+            at.append(t)
+            ar.append(r)
+        sets.append((at, ar))
+    flags = eg.FLAG_TIME_GRAM if time_gram else 0
+    ctx = eg.Context(list(w.d), w.b, w.W, float(np.float32(w.T)), flags, device=device)
+    losses = torch.empty(w.M, dtype=torch.float32, device=device)
+    slopes = torch.empty(w.M, dtype=torch.float64, device=device)
+    mask = torch.empty(w.M, dtype=torch.uint8, device=device)
+    ptrs = [(ctx._ptr_array(at, w.b, True), ctx._ptr_array(ar, w.b, True)) for at, ar in sets]
+    sp = int(stream.cuda_stream)
+
+    def step(i):
+        pa, pr = ptrs[i % n_sets]
+        ctx.sp_loss_batch_raw(pa, pr, w.b, losses.data_ptr(), sp)
+        ctx.egeria_plasticity_step(losses, slopes, mask, stream)
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize(device)
+    if time_gram:
+        ctx.egeria_gram_kernel_time()
+    l0 = ctx.egeria_launch_count()
+    return ctx, step, (losses, slopes, mask), sets, l0
+
+
+def run_ours(args):
+    from paper_2201_06227_b200 import binding as eg
+    eg.lib()  # fail loudly if the CUDA library is missing
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the path has no CPU implementation")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", rank=rank, world_size=world,
+                                device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream(device)
+    w = wl.WORKLOADS[args.workload]
+    n_sets = 1 if w.input_bytes > 4 * 126e6 else max(2, int(np.ceil(8 * 126e6 / w.input_bytes)))
+    n_sets = min(n_sets, 16)
+
+    ctx, step, outs, sets, l0 = time_workload(eg, w, device, args.steps, args.warmup, n_sets, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    barrier()
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i)
+    ev1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    elapsed_ms = ev0.elapsed_time(ev1)
+    gram_ms, gram_calls = ctx.egeria_gram_kernel_time()
+    launches = ctx.egeria_launch_count() - l0
+    ctx.check_device_status()
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    elapsed_ms = float(t.item())
+    value = world * w.M * args.steps / (elapsed_ms * 1e-3)
+
+    # ---- end to end through the host entry point (pinned host buffers, copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        at, ar = sets[0]
+        host_t = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in at]
+        host_r = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in ar]
+        ctx_h = eg.Context(list(w.d), w.b, w.W, float(np.float32(w.T)), eg.FLAG_HOST_STAGING, device=device)
+        host_losses = torch.empty(w.M, dtype=torch.float32, pin_memory=True)
+        host_mask = torch.empty(w.M, dtype=torch.uint8, pin_memory=True)
+        dev_losses = torch.empty(w.M, dtype=torch.float32, device=device)
+        dev_mask = torch.empty(w.M, dtype=torch.uint8, device=device)
+
+        def e2e_step():
+            ctx_h.egeria_sp_loss_batch_host(host_t, host_r, host_losses, stream)
+            dev_losses.copy_(host_losses, non_blocking=True)
+            ctx_h.egeria_plasticity_step(dev_losses, None, dev_mask, stream)
+            host_mask.copy_(dev_mask, non_blocking=True)
+            torch.cuda.synchronize(device)
+
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        for _ in range(min(args.warmup, 2)):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        barrier()
+        dt = time.perf_counter() - t0
+        tt = torch.tensor([dt], dtype=torch.float64, device=device)
+        if dist is not None:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * w.M * e2e_steps / float(tt.item()), "unit": UNIT,
+               "h2d_bytes_per_step": w.input_bytes + 4 * w.M, "d2h_bytes_per_step": 4 * w.M + w.M,
+               "steps": e2e_steps}
+        ctx_h.close()
+        del host_t, host_r
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = hbm_peak()
+    gram_s = (gram_ms / max(1, gram_calls)) * 1e-3
+    achieved = w.input_bytes / gram_s / 1e9 if gram_s > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "gram_tc_kernel", "achieved": achieved, "peak": peak,
+                "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "algorithmic_bytes_per_launch": w.input_bytes,
+                "avg_launch_ms": gram_s * 1e3, "launches_timed": gram_calls}
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu_baseline, _, _ = oracle_sample(w)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 inputs, f32 accumulate, f64 reductions",
+        "data": "synthetic",
+        "config": {"workload": w.name, "b": w.b, "modules": w.M, "sum_d": w.sum_d,
+                   "input_bytes_per_step": w.input_bytes, "parallelism": f"replicas x{world}",
+                   "cache": ("inputs larger than L2" if n_sets == 1 else
+                             f"rotating {n_sets} input sets ({n_sets * w.input_bytes / 1e6:.0f} MB) larger than L2")},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+        "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="gpt2_medium", choices=wl.ORDER)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,183 @@
+/*
+ * egeria.h -- C ABI of the B200 (sm_100a) plasticity-evaluation library.
+ *
+ * The library evaluates the "training plasticity" of every monitored layer
+ * module of a network (Egeria, Sec. 4.2.1, Eq. 1) and turns each module's
+ * plasticity history into the freezing decision of Sec. 4.2.2 / Algorithm 1.
+ *
+ * Notation (the paper's): b = mini-batch size; module l has training and
+ * reference activations A_T^(l), A_R^(l), flattened per sample to b x d_l;
+ * P_i^(l) = plasticity at evaluation i; W = window (moving-average span, fit
+ * window and number of consecutive low-slope evaluations); T = slope tolerance.
+ *
+ * Conventions for every call
+ *   - "device" pointers are CUDA device memory owned by the caller; "host"
+ *     pointers are ordinary host memory.  The library allocates no device
+ *     memory: all scratch lives in the caller's workspace (see
+ *     egeria_workspace_bytes).
+ *   - cuda_stream is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls enqueue work on it and return without synchronising, unless the
+ *     call's comment says otherwise.
+ *   - Activations are bfloat16, row-major [b, d_l] (sample-major), contiguous.
+ *   - Errors are returned as egeria_status; nothing throws or aborts.  There is
+ *     no CPU fallback: without an sm_100 device the compute calls fail with
+ *     EGERIA_ERR_UNSUPPORTED_DEVICE or EGERIA_ERR_CUDA.
+ *   - One context per stream; a context is not thread-safe.
+ */
+#ifndef EGERIA_H_
+#define EGERIA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct egeria_ctx egeria_ctx; /* opaque, library-owned host object */
+
+typedef enum {
+    EGERIA_OK = 0,
+    EGERIA_ERR_INVALID_ARG = 1,        /* NULL pointer, M < 1, b out of range, W < 1, ... */
+    EGERIA_ERR_UNSUPPORTED_SHAPE = 2,  /* d_l < 1, b > 256, ... */
+    EGERIA_ERR_UNSUPPORTED_DEVICE = 3, /* current device is not compute capability 10.x */
+    EGERIA_ERR_WORKSPACE = 4,          /* workspace NULL, misaligned or too small */
+    EGERIA_ERR_CUDA = 5,               /* a CUDA runtime/driver call failed */
+    EGERIA_ERR_TIMEOUT = 6             /* a bounded device-side wait ran out (see egeria_device_status) */
+} egeria_status;
+
+enum {
+    /* Use the literal test of Algorithm 1, slope < T, instead of |slope| < T. */
+    EGERIA_FLAG_SIGNED_SLOPE = 1u,
+    /* Compute every Gram matrix with the CUDA-core kernel (plain loads, FMA)
+     * instead of the TMA + tcgen05 kernel.  Same results up to summation order. */
+    EGERIA_FLAG_FORCE_SIMT = 2u,
+    /* Keep the two row-normalised similarity matrices of every module in the
+     * workspace so that egeria_debug_dump_gram can return them. */
+    EGERIA_FLAG_KEEP_GRAMS = 4u,
+    /* Reserve device staging for egeria_sp_loss_batch_host in the workspace. */
+    EGERIA_FLAG_HOST_STAGING = 8u,
+    /* Record a CUDA event before and after the Gram kernel(s) of every
+     * egeria_sp_loss_batch call, for egeria_gram_kernel_time. */
+    EGERIA_FLAG_TIME_GRAM = 16u
+};
+
+#define EGERIA_MAX_B 256          /* largest supported mini-batch size */
+#define EGERIA_WORKSPACE_ALIGN 1024
+
+/* Bytes of device workspace a context with these parameters needs.  Pure host
+ * arithmetic (no CUDA call).  Returns 0 for invalid arguments.
+ *   M      number of monitored modules (>= 1)
+ *   d      host array [M], flattened per-sample size of each module (>= 1)
+ *   b_max  largest b any call will pass (2..EGERIA_MAX_B)
+ *   W      window (>= 1)
+ *   flags  EGERIA_FLAG_* (KEEP_GRAMS and HOST_STAGING enlarge the workspace) */
+size_t egeria_workspace_bytes(int M, const int64_t *d, int b_max, int W, uint32_t flags);
+
+/* Create a context for M modules [inputs of Algorithm 1: W, T; module shapes].
+ *   out        receives the context
+ *   T          host array [M] of per-module tolerances, or NULL to use T_all
+ *   workspace  device memory, EGERIA_WORKSPACE_ALIGN-aligned, caller-owned, at
+ *              least egeria_workspace_bytes(...) long; must outlive the context
+ * Clears the plasticity state (as egeria_plasticity_reset) synchronously on the
+ * current device.  W = 1 is accepted but can never converge (no line through
+ * one point). */
+egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d, int b_max,
+                                       int W, const float *T, float T_all, void *workspace,
+                                       size_t workspace_bytes, uint32_t flags);
+
+/* Free the host object.  The workspace stays the caller's. */
+egeria_status egeria_plasticity_destroy(egeria_ctx *ctx);
+
+/* Plasticity of every module for one mini-batch [Sec. 4.2.1, Eq. 1]:
+ *   G = A A^T (b x b, fp32 accumulation of bf16 products) for A_T and A_R,
+ *   every row of G scaled to unit L2 norm (norms below 1e-12 are clamped, so an
+ *   all-zero sample gives a zero row), P = ||G~_T - G~_R||_F^2 / b^2.
+ *   At, Ar      host arrays [M] of device pointers, bf16 [b, d_l] each
+ *   b           2..b_max
+ *   d           host array [M]; must equal the d given at creation
+ *   out_losses  device float [M]
+ * Modules whose d_l is a multiple of 8 and whose pointers are 16-byte aligned
+ * take the TMA + tcgen05 kernel; others take the CUDA-core kernel.
+ * NaN/Inf in the inputs propagate to the loss. */
+egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const void *const *At,
+                                   const void *const *Ar, int b, const int64_t *d,
+                                   float *out_losses);
+
+/* Same evaluation from HOST activations: copies every A_T, A_R to the staging
+ * area of the workspace (needs EGERIA_FLAG_HOST_STAGING), evaluates, copies the
+ * M losses back to out_losses_host and synchronises the stream before returning.
+ *   At_host, Ar_host  host arrays [M] of host pointers (pinned memory copies
+ *                     fastest), bf16 [b, d_l]
+ *   out_losses_host   host float [M] */
+egeria_status egeria_sp_loss_batch_host(egeria_ctx *ctx, void *cuda_stream,
+                                        const void *const *At_host, const void *const *Ar_host,
+                                        int b, const int64_t *d, float *out_losses_host);
+
+/* One evaluation of the freezing rule for every module [Sec. 4.2.2, Eq. 2,
+ * Algorithm 1]: append the new reading, smooth (mean of the last min(i+1, W)
+ * readings), append to the module's list, fit a least-squares line to the last
+ * min(len, W) smoothed values against 0,1,2,..., compare the slope with T
+ * (|s| < T, strict; fewer than two points or NaN is "not stale"), update the
+ * consecutive-stale counter; a module is converged once its counter reaches W
+ * and its state then stops advancing.  All arithmetic is float64.
+ *   losses      device float [M], e.g. the out_losses of egeria_sp_loss_batch
+ *   out_slopes  device double [M] (slope of this evaluation; the last one for a
+ *               module that had already converged), may be NULL
+ *   out_mask    device uint8 [M], 1 = converged (freeze), may be NULL */
+egeria_status egeria_plasticity_step(egeria_ctx *ctx, void *cuda_stream, const float *losses,
+                                     double *out_slopes, uint8_t *out_mask);
+
+/* The same rule over whole histories, from a cleared state that is private to
+ * the call (the context's step state is not touched).
+ *   hist             device float [M, H] row-major raw readings
+ *   out_slopes       device double [M, H]; NaN after a module converged; may be NULL
+ *   out_mask         device uint8 [M]
+ *   out_freeze_eval  device int32 [M]: evaluation index at which the counter
+ *                    reached W, -1 if never; may be NULL */
+egeria_status egeria_plasticity_replay(egeria_ctx *ctx, void *cuda_stream, const float *hist,
+                                       int H, double *out_slopes, uint8_t *out_mask,
+                                       int32_t *out_freeze_eval);
+
+/* Clear the step state (histories, counters, masks), e.g. when the caller
+ * unfreezes after a learning-rate drop [Sec. 4.2.2 "Unfreezing"].  If halve_W
+ * is non-zero the window is halved first (never below 2), as the paper does
+ * for refreezing. */
+egeria_status egeria_plasticity_reset(egeria_ctx *ctx, void *cuda_stream, int halve_W);
+
+/* Current window of the context (changes only through egeria_plasticity_reset). */
+int egeria_plasticity_window(const egeria_ctx *ctx);
+
+/* Test hook: copy the row-normalised similarity matrices of one module, as
+ * left by the last egeria_sp_loss_batch, to device float [b, b] buffers.
+ * Needs EGERIA_FLAG_KEEP_GRAMS. */
+egeria_status egeria_debug_dump_gram(egeria_ctx *ctx, void *cuda_stream, int module,
+                                     float *Gt_norm, float *Gr_norm);
+
+/* Test hook: the static work split of one evaluation, pure host arithmetic.
+ * Writes up to max_units rows {module, side (0 = T, 1 = R, 2 = both), first
+ * 64-element block, number of blocks, CTA} to out_units and the unit count to
+ * n_units.  n_ctas is the number of persistent CTAs to split over. */
+egeria_status egeria_debug_plan(int M, const int64_t *d, int b, int n_ctas, int32_t *out_units,
+                                int max_units, int *n_units);
+
+/* Synchronise the stream of the last call and report the device status word:
+ * EGERIA_OK, or EGERIA_ERR_TIMEOUT if a bounded wait inside a kernel ran out
+ * (the kernel then skipped its remaining work; results are invalid). */
+egeria_status egeria_device_status(egeria_ctx *ctx);
+
+/* Measurement hook (needs EGERIA_FLAG_TIME_GRAM): device time, in milliseconds,
+ * spent in the Gram kernels of the egeria_sp_loss_batch calls made since the
+ * last query (the finalisation kernel is not included), and the number of those
+ * calls.  Waits for the last recorded event.  Resets the tally. */
+egeria_status egeria_gram_kernel_time(egeria_ctx *ctx, double *total_ms, int64_t *n_calls);
+
+/* Number of kernels the library has launched through this context so far. */
+int64_t egeria_launch_count(const egeria_ctx *ctx);
+
+const char *egeria_status_string(egeria_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EGERIA_H_ */

@@ -1,0 +1,250 @@
+"""ctypes binding of ``libegeria.so`` -- argument marshalling only.
+
+Every function here has the name of the C entry point it calls (``include/egeria.h``).
+PyTorch appears only as the owner of device memory and streams; every step of the
+plasticity evaluation runs inside the library's CUDA kernels.  There is no fallback:
+if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libegeria.so"
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+FLAG_SIGNED_SLOPE, FLAG_FORCE_SIMT, FLAG_KEEP_GRAMS, FLAG_HOST_STAGING, FLAG_TIME_GRAM = 1, 2, 4, 8, 16
+MAX_B = 256
+WORKSPACE_ALIGN = 1024
+
+EXPORTS = [
+    "egeria_workspace_bytes", "egeria_plasticity_create", "egeria_plasticity_destroy",
+    "egeria_sp_loss_batch", "egeria_sp_loss_batch_host", "egeria_plasticity_step",
+    "egeria_plasticity_replay", "egeria_plasticity_reset", "egeria_plasticity_window",
+    "egeria_debug_dump_gram", "egeria_debug_plan", "egeria_device_status", "egeria_launch_count",
+    "egeria_gram_kernel_time",
+    "egeria_status_string",
+]
+
+
+class EgeriaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {status_string(status)} (status {int(status)})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library.  Raises if it has not been built -- there is no other path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2201_06227_b200.build`")
+    L = ctypes.CDLL(str(_LIB_PATH))
+    vp, i64p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64)
+    L.egeria_workspace_bytes.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int, ctypes.c_uint32]
+    L.egeria_workspace_bytes.restype = ctypes.c_size_t
+    L.egeria_plasticity_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int,
+                                           ctypes.POINTER(ctypes.c_float), ctypes.c_float, vp, ctypes.c_size_t,
+                                           ctypes.c_uint32]
+    L.egeria_plasticity_destroy.argtypes = [vp]
+    L.egeria_sp_loss_batch.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, i64p, vp]
+    L.egeria_sp_loss_batch_host.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, i64p, vp]
+    L.egeria_plasticity_step.argtypes = [vp, vp, vp, vp, vp]
+    L.egeria_plasticity_replay.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp]
+    L.egeria_plasticity_reset.argtypes = [vp, vp, ctypes.c_int]
+    L.egeria_plasticity_window.argtypes = [vp]
+    L.egeria_debug_dump_gram.argtypes = [vp, vp, ctypes.c_int, vp, vp]
+    L.egeria_debug_plan.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int,
+                                    ctypes.POINTER(ctypes.c_int32), ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+    L.egeria_device_status.argtypes = [vp]
+    L.egeria_gram_kernel_time.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
+    L.egeria_launch_count.argtypes = [vp]
+    L.egeria_launch_count.restype = ctypes.c_int64
+    L.egeria_status_string.argtypes = [ctypes.c_int]
+    L.egeria_status_string.restype = ctypes.c_char_p
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().egeria_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise EgeriaError(status, where)
+
+
+def _i64(seq: Sequence[int]):
+    arr = (ctypes.c_int64 * len(seq))(*[int(v) for v in seq])
+    return arr
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def egeria_workspace_bytes(M: int, d: Sequence[int], b_max: int, W: int, flags: int = 0) -> int:
+    return int(lib().egeria_workspace_bytes(int(M), _i64(d), int(b_max), int(W), int(flags)))
+
+
+def egeria_debug_plan(d: Sequence[int], b: int, n_ctas: int) -> np.ndarray:
+    """Rows {module, side, first block, blocks, cta} of the static work split."""
+    M = len(d)
+    cap = 2 * M + n_ctas + 8
+    out = np.zeros((cap, 5), dtype=np.int32)
+    n = ctypes.c_int(0)
+    st = lib().egeria_debug_plan(M, _i64(d), int(b), int(n_ctas),
+                                 out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), cap, ctypes.byref(n))
+    _check(st, "egeria_debug_plan")
+    return out[: n.value].copy()
+
+
+class Context:
+    """Owner of one ``egeria_ctx`` and of its workspace tensor."""
+
+    def __init__(self, d: Sequence[int], b_max: int, W: int, T, flags: int = 0, device="cuda"):
+        self.d = [int(v) for v in d]
+        self.M = len(self.d)
+        self.b_max = int(b_max)
+        self.flags = int(flags)
+        self.device = torch.device(device)
+        self._d_arr = _i64(self.d)
+        nbytes = egeria_workspace_bytes(self.M, self.d, b_max, W, flags)
+        if nbytes == 0:
+            raise EgeriaError(ERR_INVALID_ARG, "egeria_workspace_bytes")
+        self.workspace_bytes = nbytes
+        raw = torch.empty(nbytes + WORKSPACE_ALIGN, dtype=torch.uint8, device=self.device)
+        off = (-raw.data_ptr()) % WORKSPACE_ALIGN
+        self._raw = raw
+        self._ws_ptr = raw.data_ptr() + off
+        if np.isscalar(T):
+            t_arr, t_all = None, float(T)
+        else:
+            t_np = np.ascontiguousarray(T, dtype=np.float32)
+            assert t_np.shape == (self.M,)
+            t_arr, t_all = t_np.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), 0.0
+        handle = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            st = lib().egeria_plasticity_create(ctypes.byref(handle), self.M, self._d_arr, self.b_max, int(W),
+                                                t_arr, ctypes.c_float(t_all), ctypes.c_void_p(self._ws_ptr),
+                                                nbytes, self.flags)
+        _check(st, "egeria_plasticity_create")
+        self._h = handle
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            lib().egeria_plasticity_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ calls
+    def _ptr_array(self, tensors: Sequence[torch.Tensor], b: int, on_device: bool):
+        if len(tensors) != self.M:
+            raise ValueError("one activation per module is required")
+        ptrs = (ctypes.c_void_p * self.M)()
+        for m, t in enumerate(tensors):
+            if t.dtype != torch.bfloat16 or t.shape != (b, self.d[m]) or not t.is_contiguous():
+                raise ValueError(f"module {m}: expected contiguous bfloat16 [{b}, {self.d[m]}]")
+            if t.is_cuda != on_device:
+                raise ValueError(f"module {m}: tensor is on the wrong side of the bus")
+            ptrs[m] = t.data_ptr()
+        return ptrs
+
+    def egeria_sp_loss_batch(self, At: Sequence[torch.Tensor], Ar: Sequence[torch.Tensor],
+                             out_losses: Optional[torch.Tensor] = None,
+                             stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        b = int(At[0].shape[0])
+        if out_losses is None:
+            out_losses = torch.empty(self.M, dtype=torch.float32, device=self.device)
+        pa, pr = self._ptr_array(At, b, True), self._ptr_array(Ar, b, True)
+        st = lib().egeria_sp_loss_batch(self._h, _stream_ptr(stream), pa, pr, b, self._d_arr,
+                                        out_losses.data_ptr())
+        _check(st, "egeria_sp_loss_batch")
+        return out_losses
+
+    def sp_loss_batch_raw(self, pa, pr, b: int, out_ptr: int, stream_ptr: int) -> None:
+        """Same call with ready-made pointer arrays (benchmark loops)."""
+        _check(lib().egeria_sp_loss_batch(self._h, stream_ptr, pa, pr, b, self._d_arr, out_ptr),
+               "egeria_sp_loss_batch")
+
+    def egeria_sp_loss_batch_host(self, At: Sequence[torch.Tensor], Ar: Sequence[torch.Tensor],
+                                  out_losses: Optional[torch.Tensor] = None,
+                                  stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        b = int(At[0].shape[0])
+        if out_losses is None:
+            out_losses = torch.empty(self.M, dtype=torch.float32)
+        pa, pr = self._ptr_array(At, b, False), self._ptr_array(Ar, b, False)
+        st = lib().egeria_sp_loss_batch_host(self._h, _stream_ptr(stream), pa, pr, b, self._d_arr,
+                                             out_losses.data_ptr())
+        _check(st, "egeria_sp_loss_batch_host")
+        return out_losses
+
+    def egeria_plasticity_step(self, losses: torch.Tensor, out_slopes: Optional[torch.Tensor] = None,
+                               out_mask: Optional[torch.Tensor] = None,
+                               stream: Optional[torch.cuda.Stream] = None):
+        assert losses.is_cuda and losses.dtype == torch.float32 and losses.numel() == self.M
+        if out_slopes is None:
+            out_slopes = torch.empty(self.M, dtype=torch.float64, device=self.device)
+        if out_mask is None:
+            out_mask = torch.empty(self.M, dtype=torch.uint8, device=self.device)
+        st = lib().egeria_plasticity_step(self._h, _stream_ptr(stream), losses.data_ptr(),
+                                          out_slopes.data_ptr(), out_mask.data_ptr())
+        _check(st, "egeria_plasticity_step")
+        return out_slopes, out_mask
+
+    def egeria_plasticity_replay(self, hist: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+        assert hist.is_cuda and hist.dtype == torch.float32 and hist.dim() == 2 and hist.shape[0] == self.M
+        hist = hist.contiguous()
+        H = int(hist.shape[1])
+        slopes = torch.empty((self.M, H), dtype=torch.float64, device=self.device)
+        mask = torch.empty(self.M, dtype=torch.uint8, device=self.device)
+        freeze_eval = torch.empty(self.M, dtype=torch.int32, device=self.device)
+        st = lib().egeria_plasticity_replay(self._h, _stream_ptr(stream), hist.data_ptr(), H, slopes.data_ptr(),
+                                            mask.data_ptr(), freeze_eval.data_ptr())
+        _check(st, "egeria_plasticity_replay")
+        return slopes, mask, freeze_eval
+
+    def egeria_plasticity_reset(self, halve_W: bool = False, stream: Optional[torch.cuda.Stream] = None) -> None:
+        _check(lib().egeria_plasticity_reset(self._h, _stream_ptr(stream), int(bool(halve_W))),
+               "egeria_plasticity_reset")
+
+    def egeria_plasticity_window(self) -> int:
+        return int(lib().egeria_plasticity_window(self._h))
+
+    def egeria_debug_dump_gram(self, module: int, b: int, stream: Optional[torch.cuda.Stream] = None):
+        gt = torch.empty((b, b), dtype=torch.float32, device=self.device)
+        gr = torch.empty((b, b), dtype=torch.float32, device=self.device)
+        st = lib().egeria_debug_dump_gram(self._h, _stream_ptr(stream), int(module), gt.data_ptr(), gr.data_ptr())
+        _check(st, "egeria_debug_dump_gram")
+        return gt, gr
+
+    def egeria_device_status(self) -> int:
+        return int(lib().egeria_device_status(self._h))
+
+    def check_device_status(self) -> None:
+        _check(self.egeria_device_status(), "egeria_device_status")
+
+    def egeria_gram_kernel_time(self):
+        """(total milliseconds, calls) of the Gram kernels since the last query."""
+        ms, n = ctypes.c_double(), ctypes.c_int64()
+        _check(lib().egeria_gram_kernel_time(self._h, ctypes.byref(ms), ctypes.byref(n)), "egeria_gram_kernel_time")
+        return ms.value, n.value
+
+    def egeria_launch_count(self) -> int:
+        return int(lib().egeria_launch_count(self._h))

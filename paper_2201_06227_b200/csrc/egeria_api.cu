@@ -1,0 +1,540 @@
+// C ABI of the plasticity-evaluation library: argument checks, workspace layout, the
+// static work split, tensor-map encoding and kernel launches.  See include/egeria.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/egeria.h"
+#include "finalize.cuh"
+#include "gram_simt.cuh"
+#include "gram_tc.cuh"
+#include "plan.h"
+#include "slope.cuh"
+
+namespace egeria {
+
+constexpr int kMaxCtas = 160;  // sizing bound for the work split (a B200 has 148 SMs)
+constexpr int kMaxW = 2048;    // replay keeps 2 * W doubles in shared memory
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Offsets of everything the library keeps in the caller's workspace.
+struct Layout {
+    size_t status, tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides, rowloss, tickets, T,
+        raw, plist, n_evals, counter, freeze_eval, last_slope, losses, keep, slots, staging, total;
+    size_t slot_bytes_cap;  // bytes reserved for partial slots
+};
+
+static int64_t units_cap(int M, int b_max) {
+    int64_t cap = 0;
+    for (int mode = 0; mode <= mode_of_b(b_max); ++mode) {
+        const int64_t u = max_units(M, mode, kMaxCtas);
+        if (u > cap) cap = u;
+    }
+    return cap;
+}
+
+static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flags, Layout &L) {
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t o = off;
+        off = align_up(off + bytes, 256);
+        return o;
+    };
+    L.status = take(256);
+    L.tmaps = take((size_t)2 * M * sizeof(CUtensorMap));
+    L.modules = take((size_t)M * sizeof(ModulePtrs));
+    L.units = take((size_t)units_cap(M, b_max) * sizeof(Unit));
+    L.cta_begin_tc = take((kMaxCtas + 1) * sizeof(int32_t));
+    L.cta_begin_simt = take((kMaxCtas + 1) * sizeof(int32_t));
+    L.sides = take((size_t)2 * M * sizeof(SideInfo));
+    L.rowloss = take((size_t)M * kMaxB * sizeof(double));
+    L.tickets = take((size_t)M * sizeof(int32_t));
+    L.T = take((size_t)M * sizeof(float));
+    L.raw = take((size_t)M * W * sizeof(double));
+    L.plist = take((size_t)M * W * sizeof(double));
+    L.n_evals = take((size_t)M * sizeof(int32_t));
+    L.counter = take((size_t)M * sizeof(int32_t));
+    L.freeze_eval = take((size_t)M * sizeof(int32_t));
+    L.last_slope = take((size_t)M * sizeof(double));
+    L.losses = take((size_t)M * sizeof(float));
+    L.keep = off;
+    if (flags & EGERIA_FLAG_KEEP_GRAMS) take((size_t)M * 2 * b_max * b_max * sizeof(float));
+    size_t slot_bytes = 0;
+    for (int mode = 0; mode <= mode_of_b(b_max); ++mode) {
+        const size_t s = (size_t)max_units(M, mode, kMaxCtas) * slot_floats_of_mode(mode) * sizeof(float);
+        if (s > slot_bytes) slot_bytes = s;
+    }
+    L.slot_bytes_cap = slot_bytes;
+    L.slots = take(slot_bytes);
+    L.staging = off;
+    if (flags & EGERIA_FLAG_HOST_STAGING) {
+        for (int m = 0; m < M; ++m) {
+            take((size_t)b_max * d[m] * 2);
+            take((size_t)b_max * d[m] * 2);
+        }
+    }
+    L.total = align_up(off, EGERIA_WORKSPACE_ALIGN);
+    return true;
+}
+
+static egeria_status check_shapes(int M, const int64_t *d, int b_max, int W) {
+    if (M < 1 || !d || W < 1 || W > kMaxW) return EGERIA_ERR_INVALID_ARG;
+    if (b_max < 2) return EGERIA_ERR_INVALID_ARG;
+    if (b_max > EGERIA_MAX_B) return EGERIA_ERR_UNSUPPORTED_SHAPE;
+    for (int m = 0; m < M; ++m) {
+        if (d[m] < 1) return EGERIA_ERR_UNSUPPORTED_SHAPE;
+        // TMA coordinates are 32-bit element indices
+        if (d[m] > (int64_t)0x7fffffff - 2 * kKBlock) return EGERIA_ERR_UNSUPPORTED_SHAPE;
+    }
+    return EGERIA_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+}  // namespace egeria
+
+using namespace egeria;
+
+struct egeria_ctx {
+    int M = 0, b_max = 0, W = 0, W_cap = 0;
+    uint32_t flags = 0;
+    std::vector<int64_t> d;
+    uint8_t *ws = nullptr;
+    size_t ws_bytes = 0;
+    Layout L{};
+    int n_ctas = 0;
+    EncodeTiledFn encode = nullptr;
+    bool attrs_set = false;
+    // what the device-side plan currently describes
+    int plan_b = -1;
+    std::vector<const void *> plan_At, plan_Ar;
+    Plan plan;
+    cudaStream_t last_stream = nullptr;
+    int64_t launches = 0;
+    std::vector<void *> staging_t, staging_r;
+    // EGERIA_FLAG_TIME_GRAM: event pairs around the Gram kernel launches since the last query
+    std::vector<cudaEvent_t> ev_pool;
+    size_t ev_used = 0;
+
+    template <class T>
+    T *at(size_t off) const {
+        return reinterpret_cast<T *>(ws + off);
+    }
+    SlopeState slope_state() const {
+        SlopeState st;
+        st.raw = at<double>(L.raw);
+        st.plist = at<double>(L.plist);
+        st.n_evals = at<int32_t>(L.n_evals);
+        st.counter = at<int32_t>(L.counter);
+        st.freeze_eval = at<int32_t>(L.freeze_eval);
+        st.last_slope = at<double>(L.last_slope);
+        st.T = at<float>(L.T);
+        st.W_cap = W_cap;
+        return st;
+    }
+};
+
+#define EG_CUDA(call)                                   \
+    do {                                                \
+        cudaError_t e_ = (call);                        \
+        if (e_ != cudaSuccess) return EGERIA_ERR_CUDA;  \
+    } while (0)
+
+extern "C" {
+
+const char *egeria_status_string(egeria_status s) {
+    switch (s) {
+        case EGERIA_OK: return "ok";
+        case EGERIA_ERR_INVALID_ARG: return "invalid argument";
+        case EGERIA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case EGERIA_ERR_UNSUPPORTED_DEVICE: return "unsupported device (needs compute capability 10.x)";
+        case EGERIA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case EGERIA_ERR_CUDA: return "CUDA call failed";
+        case EGERIA_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+size_t egeria_workspace_bytes(int M, const int64_t *d, int b_max, int W, uint32_t flags) {
+    if (check_shapes(M, d, b_max, W) != EGERIA_OK) return 0;
+    Layout L;
+    make_layout(M, d, b_max, W, flags, L);
+    return L.total;
+}
+
+egeria_status egeria_debug_plan(int M, const int64_t *d, int b, int n_ctas, int32_t *out_units, int max_units_out,
+                                int *n_units) {
+    if (!out_units || !n_units || n_ctas < 1 || max_units_out < 0) return EGERIA_ERR_INVALID_ARG;
+    egeria_status s = check_shapes(M, d, b, 1);
+    if (s != EGERIA_OK) return s;
+    std::vector<uint8_t> tc_ok(M);
+    for (int m = 0; m < M; ++m) tc_ok[m] = (d[m] % 8 == 0);
+    Plan plan;
+    build_plan(M, d, b, n_ctas, tc_ok.data(), plan);
+    *n_units = (int)plan.units.size();
+    for (int i = 0; i < (int)plan.units.size() && i < max_units_out; ++i) {
+        const Unit &u = plan.units[i];
+        int32_t *row = out_units + 5 * i;
+        row[0] = u.module;
+        row[1] = u.side;
+        row[2] = u.kb0;
+        row[3] = u.nkb;
+        row[4] = u.cta;
+    }
+    return EGERIA_OK;
+}
+
+egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d, int b_max, int W, const float *T,
+                                       float T_all, void *workspace, size_t workspace_bytes, uint32_t flags) {
+    if (!out) return EGERIA_ERR_INVALID_ARG;
+    *out = nullptr;
+    egeria_status s = check_shapes(M, d, b_max, W);
+    if (s != EGERIA_OK) return s;
+    Layout L;
+    make_layout(M, d, b_max, W, flags, L);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % EGERIA_WORKSPACE_ALIGN) != 0 ||
+        workspace_bytes < L.total)
+        return EGERIA_ERR_WORKSPACE;
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    EG_CUDA(cudaGetDevice(&dev));
+    EG_CUDA(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return EGERIA_ERR_UNSUPPORTED_DEVICE;
+
+    egeria_ctx *ctx = new (std::nothrow) egeria_ctx();
+    if (!ctx) return EGERIA_ERR_INVALID_ARG;
+    ctx->M = M;
+    ctx->b_max = b_max;
+    ctx->W = W;
+    ctx->W_cap = W;
+    ctx->flags = flags;
+    ctx->d.assign(d, d + M);
+    ctx->ws = static_cast<uint8_t *>(workspace);
+    ctx->ws_bytes = workspace_bytes;
+    ctx->L = L;
+    ctx->n_ctas = prop.multiProcessorCount < kMaxCtas ? prop.multiProcessorCount : kMaxCtas;
+
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn) {
+        delete ctx;
+        return EGERIA_ERR_CUDA;
+    }
+    ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+
+    if (flags & EGERIA_FLAG_HOST_STAGING) {
+        size_t off = L.staging;  // same walk as make_layout
+        for (int m = 0; m < M; ++m) {
+            ctx->staging_t.push_back(ctx->ws + off);
+            off = align_up(off + (size_t)b_max * d[m] * 2, 256);
+            ctx->staging_r.push_back(ctx->ws + off);
+            off = align_up(off + (size_t)b_max * d[m] * 2, 256);
+        }
+    }
+
+    std::vector<float> Th(M);
+    for (int m = 0; m < M; ++m) Th[m] = T ? T[m] : T_all;
+    cudaError_t e = cudaMemset(ctx->ws + L.status, 0, 256);
+    if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.tickets, 0, (size_t)M * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->ws + L.T, Th.data(), (size_t)M * sizeof(float), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) {
+        plasticity_clear_kernel<<<(M + 127) / 128, 128>>>(ctx->slope_state(), M);
+        ctx->launches++;
+        e = cudaDeviceSynchronize();
+    }
+    if (e != cudaSuccess) {
+        delete ctx;
+        return EGERIA_ERR_CUDA;
+    }
+    *out = ctx;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_plasticity_destroy(egeria_ctx *ctx) {
+    if (!ctx) return EGERIA_ERR_INVALID_ARG;
+    for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+    delete ctx;
+    return EGERIA_OK;
+}
+
+int egeria_plasticity_window(const egeria_ctx *ctx) { return ctx ? ctx->W : 0; }
+int64_t egeria_launch_count(const egeria_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"
+
+namespace egeria {
+
+static egeria_status encode_map(egeria_ctx *ctx, CUtensorMap *tm, const void *base, int b, int64_t d, int box_rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)b};
+    cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kKBlock, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box,
+                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? EGERIA_OK : EGERIA_ERR_CUDA;
+}
+
+// Bring the device-side plan (units, tensor maps, pointers) up to date with this call.
+static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const void *const *At, const void *const *Ar,
+                                  int b) {
+    const int M = ctx->M;
+    bool same = (ctx->plan_b == b) && (int)ctx->plan_At.size() == M;
+    for (int m = 0; m < M && same; ++m) same = (ctx->plan_At[m] == At[m]) && (ctx->plan_Ar[m] == Ar[m]);
+    if (same) return EGERIA_OK;
+
+    std::vector<uint8_t> tc_ok(M);
+    for (int m = 0; m < M; ++m) {
+        const bool aligned = (reinterpret_cast<uintptr_t>(At[m]) % 16 == 0) &&
+                             (reinterpret_cast<uintptr_t>(Ar[m]) % 16 == 0) && (ctx->d[m] % 8 == 0);
+        tc_ok[m] = aligned && !(ctx->flags & EGERIA_FLAG_FORCE_SIMT);
+    }
+    build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), ctx->plan);
+    const Plan &P = ctx->plan;
+    if ((size_t)P.units.size() * slot_floats_of_mode(P.mode) * sizeof(float) > ctx->L.slot_bytes_cap)
+        return EGERIA_ERR_WORKSPACE;
+
+    const int box_rows = (P.mode == kStacked) ? 64 : (P.mode == kSingle1 ? 128 : 256);
+    std::vector<CUtensorMap> maps(2 * (size_t)M);
+    std::vector<ModulePtrs> mods(M);
+    memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
+    for (int m = 0; m < M; ++m) {
+        mods[m] = ModulePtrs{At[m], Ar[m], ctx->d[m]};
+        if (!tc_ok[m]) continue;
+        egeria_status s = encode_map(ctx, &maps[2 * m], At[m], b, ctx->d[m], box_rows);
+        if (s == EGERIA_OK) s = encode_map(ctx, &maps[2 * m + 1], Ar[m], b, ctx->d[m], box_rows);
+        if (s != EGERIA_OK) return s;
+    }
+    const Layout &L = ctx->L;
+    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.tmaps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice,
+                            stream));
+    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.modules, mods.data(), mods.size() * sizeof(ModulePtrs),
+                            cudaMemcpyHostToDevice, stream));
+    if (!P.units.empty())
+        EG_CUDA(cudaMemcpyAsync(ctx->ws + L.units, P.units.data(), P.units.size() * sizeof(Unit),
+                                cudaMemcpyHostToDevice, stream));
+    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, stream));
+    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.cta_begin_simt, P.cta_begin_simt.data(),
+                            P.cta_begin_simt.size() * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo),
+                            cudaMemcpyHostToDevice, stream));
+    ctx->plan_b = b;
+    ctx->plan_At.assign(At, At + M);
+    ctx->plan_Ar.assign(Ar, Ar + M);
+    return EGERIA_OK;
+}
+
+template <int MODE>
+static cudaError_t launch_tc(egeria_ctx *ctx, cudaStream_t stream, const TcParams &tp) {
+    gram_tc_kernel<MODE><<<ctx->n_ctas, kTcThreads, TcCfg<MODE>::kSmemBytes, stream>>>(tp);
+    return cudaGetLastError();
+}
+
+static egeria_status set_attrs(egeria_ctx *ctx) {
+    if (ctx->attrs_set) return EGERIA_OK;
+    EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kStacked>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcCfg<kStacked>::kSmemBytes));
+    EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kSingle1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcCfg<kSingle1>::kSmemBytes));
+    EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kSingle2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcCfg<kSingle2>::kSmemBytes));
+    ctx->attrs_set = true;
+    return EGERIA_OK;
+}
+
+}  // namespace egeria
+
+extern "C" {
+
+egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const void *const *At, const void *const *Ar,
+                                   int b, const int64_t *d, float *out_losses) {
+    if (!ctx || !At || !Ar || !d || !out_losses) return EGERIA_ERR_INVALID_ARG;
+    if (b < 2 || b > ctx->b_max) return EGERIA_ERR_INVALID_ARG;
+    for (int m = 0; m < ctx->M; ++m) {
+        if (d[m] != ctx->d[m]) return EGERIA_ERR_INVALID_ARG;
+        if (!At[m] || !Ar[m]) return EGERIA_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(At[m]) | reinterpret_cast<uintptr_t>(Ar[m])) & 1) return EGERIA_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    egeria_status s = set_attrs(ctx);
+    if (s != EGERIA_OK) return s;
+    s = refresh_plan(ctx, stream, At, Ar, b);
+    if (s != EGERIA_OK) return s;
+
+    const Layout &L = ctx->L;
+    const Plan &P = ctx->plan;
+    const int64_t slot_floats = slot_floats_of_mode(P.mode);
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (ctx->flags & EGERIA_FLAG_TIME_GRAM) {
+        if (ctx->ev_used + 2 > ctx->ev_pool.size()) {
+            cudaEvent_t a, c;
+            EG_CUDA(cudaEventCreate(&a));
+            EG_CUDA(cudaEventCreate(&c));
+            ctx->ev_pool.push_back(a);
+            ctx->ev_pool.push_back(c);
+        }
+        ev0 = ctx->ev_pool[ctx->ev_used];
+        ev1 = ctx->ev_pool[ctx->ev_used + 1];
+        ctx->ev_used += 2;
+        EG_CUDA(cudaEventRecord(ev0, stream));
+    }
+    if (P.n_units_tc > 0) {
+        TcParams tp;
+        tp.tmaps = ctx->at<CUtensorMap>(L.tmaps);
+        tp.units = ctx->at<Unit>(L.units);
+        tp.cta_begin = ctx->at<int32_t>(L.cta_begin_tc);
+        tp.slots = ctx->at<float>(L.slots);
+        tp.slot_floats = slot_floats;
+        tp.b = b;
+        tp.status = ctx->at<int32_t>(L.status);
+        cudaError_t e = (P.mode == kStacked)   ? launch_tc<kStacked>(ctx, stream, tp)
+                        : (P.mode == kSingle1) ? launch_tc<kSingle1>(ctx, stream, tp)
+                                               : launch_tc<kSingle2>(ctx, stream, tp);
+        if (e != cudaSuccess) return EGERIA_ERR_CUDA;
+        ctx->launches++;
+    }
+    if ((int)P.units.size() > P.n_units_tc) {
+        SimtParams sp;
+        sp.modules = ctx->at<ModulePtrs>(L.modules);
+        sp.units = ctx->at<Unit>(L.units) + P.n_units_tc;
+        sp.cta_begin = ctx->at<int32_t>(L.cta_begin_simt);
+        sp.slots = ctx->at<float>(L.slots);
+        sp.slot_floats = slot_floats;
+        sp.b = b;
+        sp.mode = P.mode;
+        gram_simt_kernel<<<ctx->n_ctas, kSimtThreads, 0, stream>>>(sp);
+        if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+        ctx->launches++;
+    }
+    if (ev1) EG_CUDA(cudaEventRecord(ev1, stream));
+    FinParams fp;
+    fp.slots = ctx->at<float>(L.slots);
+    fp.slot_floats = slot_floats;
+    fp.sides = ctx->at<SideInfo>(L.sides);
+    fp.b = b;
+    fp.out_losses = out_losses;
+    fp.rowloss = ctx->at<double>(L.rowloss);
+    fp.tickets = ctx->at<int32_t>(L.tickets);
+    fp.keep = (ctx->flags & EGERIA_FLAG_KEEP_GRAMS) ? ctx->at<float>(L.keep) : nullptr;
+    dim3 grid(ctx->M, (b + kFinRowsPerCta - 1) / kFinRowsPerCta);
+    finalize_kernel<<<grid, kFinThreads, 0, stream>>>(fp);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_sp_loss_batch_host(egeria_ctx *ctx, void *cuda_stream, const void *const *At_host,
+                                        const void *const *Ar_host, int b, const int64_t *d, float *out_losses_host) {
+    if (!ctx || !At_host || !Ar_host || !d || !out_losses_host) return EGERIA_ERR_INVALID_ARG;
+    if (!(ctx->flags & EGERIA_FLAG_HOST_STAGING)) return EGERIA_ERR_WORKSPACE;
+    if (b < 2 || b > ctx->b_max) return EGERIA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (int m = 0; m < ctx->M; ++m) {
+        if (d[m] != ctx->d[m] || !At_host[m] || !Ar_host[m]) return EGERIA_ERR_INVALID_ARG;
+        const size_t bytes = (size_t)b * d[m] * 2;
+        EG_CUDA(cudaMemcpyAsync(ctx->staging_t[m], At_host[m], bytes, cudaMemcpyHostToDevice, stream));
+        EG_CUDA(cudaMemcpyAsync(ctx->staging_r[m], Ar_host[m], bytes, cudaMemcpyHostToDevice, stream));
+    }
+    float *dev_losses = ctx->at<float>(ctx->L.losses);
+    egeria_status s = egeria_sp_loss_batch(ctx, cuda_stream, ctx->staging_t.data(), ctx->staging_r.data(), b, d,
+                                           dev_losses);
+    if (s != EGERIA_OK) return s;
+    EG_CUDA(cudaMemcpyAsync(out_losses_host, dev_losses, (size_t)ctx->M * sizeof(float), cudaMemcpyDeviceToHost,
+                            stream));
+    EG_CUDA(cudaStreamSynchronize(stream));
+    return EGERIA_OK;
+}
+
+egeria_status egeria_plasticity_step(egeria_ctx *ctx, void *cuda_stream, const float *losses, double *out_slopes,
+                                     uint8_t *out_mask) {
+    if (!ctx || !losses) return EGERIA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    plasticity_step_kernel<<<ctx->M, 32, 0, stream>>>(ctx->slope_state(), ctx->M, ctx->W,
+                                                      (ctx->flags & EGERIA_FLAG_SIGNED_SLOPE) ? 1 : 0, losses,
+                                                      out_slopes, out_mask);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_plasticity_replay(egeria_ctx *ctx, void *cuda_stream, const float *hist, int H,
+                                       double *out_slopes, uint8_t *out_mask, int32_t *out_freeze_eval) {
+    if (!ctx || !hist || H < 0 || !out_mask) return EGERIA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    plasticity_replay_kernel<<<ctx->M, 32, 2 * (size_t)ctx->W * sizeof(double), stream>>>(
+        ctx->at<float>(ctx->L.T), ctx->M, ctx->W, (ctx->flags & EGERIA_FLAG_SIGNED_SLOPE) ? 1 : 0, hist, H,
+        out_slopes, out_mask, out_freeze_eval);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_plasticity_reset(egeria_ctx *ctx, void *cuda_stream, int halve_W) {
+    if (!ctx) return EGERIA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    if (halve_W) {
+        int w = ctx->W / 2;
+        ctx->W = w < 2 ? (ctx->W < 2 ? ctx->W : 2) : w;
+    }
+    plasticity_clear_kernel<<<(ctx->M + 127) / 128, 128, 0, stream>>>(ctx->slope_state(), ctx->M);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_debug_dump_gram(egeria_ctx *ctx, void *cuda_stream, int module, float *Gt_norm,
+                                     float *Gr_norm) {
+    if (!ctx || !Gt_norm || !Gr_norm || module < 0 || module >= ctx->M) return EGERIA_ERR_INVALID_ARG;
+    if (!(ctx->flags & EGERIA_FLAG_KEEP_GRAMS)) return EGERIA_ERR_WORKSPACE;
+    if (ctx->plan_b < 2) return EGERIA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t bb = (size_t)ctx->plan_b * ctx->plan_b;
+    const float *keep = ctx->at<float>(ctx->L.keep);
+    EG_CUDA(cudaMemcpyAsync(Gt_norm, keep + (size_t)(2 * module) * bb, bb * sizeof(float), cudaMemcpyDeviceToDevice,
+                            stream));
+    EG_CUDA(cudaMemcpyAsync(Gr_norm, keep + (size_t)(2 * module + 1) * bb, bb * sizeof(float),
+                            cudaMemcpyDeviceToDevice, stream));
+    return EGERIA_OK;
+}
+
+egeria_status egeria_gram_kernel_time(egeria_ctx *ctx, double *total_ms, int64_t *n_calls) {
+    if (!ctx || !total_ms || !n_calls) return EGERIA_ERR_INVALID_ARG;
+    if (!(ctx->flags & EGERIA_FLAG_TIME_GRAM)) return EGERIA_ERR_INVALID_ARG;
+    double sum = 0.0;
+    for (size_t i = 0; i + 1 < ctx->ev_used; i += 2) {
+        EG_CUDA(cudaEventSynchronize(ctx->ev_pool[i + 1]));
+        float ms = 0.f;
+        EG_CUDA(cudaEventElapsedTime(&ms, ctx->ev_pool[i], ctx->ev_pool[i + 1]));
+        sum += ms;
+    }
+    *total_ms = sum;
+    *n_calls = (int64_t)(ctx->ev_used / 2);
+    ctx->ev_used = 0;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_device_status(egeria_ctx *ctx) {
+    if (!ctx) return EGERIA_ERR_INVALID_ARG;
+    EG_CUDA(cudaStreamSynchronize(ctx->last_stream));
+    int32_t word = 0;
+    EG_CUDA(cudaMemcpy(&word, ctx->ws + ctx->L.status, sizeof(word), cudaMemcpyDeviceToHost));
+    if (word == kStatusTimeout) return EGERIA_ERR_TIMEOUT;
+    return word == 0 ? EGERIA_OK : EGERIA_ERR_CUDA;
+}
+
+}  // extern "C"

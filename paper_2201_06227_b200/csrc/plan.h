@@ -1,0 +1,151 @@
+// Work split of one plasticity evaluation: plain host/device structs and the
+// pure host routine that builds them.  No CUDA calls in here.
+#pragma once
+#include <stdint.h>
+
+#include <vector>
+
+#ifndef __CUDACC__
+#define __host__
+#define __device__
+#endif
+
+namespace egeria {
+
+// The feature axis is cut into blocks of 64 bf16 values (128 bytes: one swizzle row).
+constexpr int kKBlock = 64;
+
+// How the b rows of A_T / A_R are laid into MMA tiles.
+//   kStacked : b <= 64.  One tile per module: A_T in rows 0..63 and A_R in rows 64..127 of a
+//              128-row slab, one 128x128 MMA; the two diagonal 64x64 blocks are G_T and G_R.
+//   kSingle1 : b <= 128. One tile per (module, side): 128-row slab, one 128x128 MMA.
+//   kSingle2 : b <= 256. One tile per (module, side): 256-row slab, the upper triangle of
+//              2x2 blocks of 128 (G00|G01 as one 128x256 MMA, G11 as one 128x128 MMA).
+enum Mode : int { kStacked = 0, kSingle1 = 1, kSingle2 = 2 };
+
+__host__ __device__ inline int mode_of_b(int b) { return b <= 64 ? kStacked : (b <= 128 ? kSingle1 : kSingle2); }
+__host__ __device__ inline int pitch_of_mode(int mode) { return mode == kStacked ? 64 : (mode == kSingle1 ? 128 : 256); }
+// fp32 values of one partial-Gram slot.
+__host__ __device__ inline int64_t slot_floats_of_mode(int mode) {
+    return mode == kStacked ? 2 * 64 * 64 : (mode == kSingle1 ? 128 * 128 : 256 * 256);
+}
+
+// One work unit: a K-range of one tile, done by one CTA, leaving one partial Gram in `slot`.
+struct Unit {
+    int32_t module;
+    int32_t side;  // 0 = A_T, 1 = A_R, 2 = both (kStacked)
+    int32_t kb0;   // first 64-element block
+    int32_t nkb;   // number of blocks
+    int32_t slot;  // partial slot index
+    int32_t cta;   // owning CTA
+};
+
+// Where the partial Grams of one (module, side) are.
+struct SideInfo {
+    int32_t first_slot;
+    int32_t n_slots;
+    int32_t side_off;  // float offset of this side inside a slot (kStacked: side * 64 * 64)
+    int32_t pitch;     // row pitch of the partial, in floats
+};
+
+// Per-module pointers for the CUDA-core kernel.
+struct ModulePtrs {
+    const void *At;
+    const void *Ar;
+    int64_t d;
+};
+
+struct Plan {
+    int mode = 0;
+    int n_ctas = 0;
+    std::vector<Unit> units;        // tensor-core units first, then CUDA-core units
+    int n_units_tc = 0;
+    std::vector<int32_t> cta_begin_tc;    // [n_ctas + 1] into units[0 .. n_units_tc)
+    std::vector<int32_t> cta_begin_simt;  // [n_ctas + 1] into units[n_units_tc ..), relative to 0
+    std::vector<SideInfo> sides;    // [2 * M]
+};
+
+inline int64_t kblocks_of(int64_t d) { return (d + kKBlock - 1) / kKBlock; }
+
+// Upper bound on the number of units (hence slots) for any b of one mode.
+inline int64_t max_units(int M, int mode, int n_ctas) {
+    int64_t tiles = (mode == kStacked) ? M : 2 * (int64_t)M;
+    return tiles + n_ctas;
+}
+
+namespace detail {
+struct Tile {
+    int32_t module;
+    int32_t side;
+    int64_t nkb;
+};
+
+// Cut the concatenated block sequence of `tiles` into n_ctas near-equal contiguous ranges;
+// every (tile, range) intersection becomes a unit.
+inline void split_tiles(const std::vector<Tile> &tiles, int n_ctas, int slot0, std::vector<Unit> &units,
+                        std::vector<int32_t> &cta_begin) {
+    int64_t total = 0;
+    for (const Tile &t : tiles) total += t.nkb;
+    cta_begin.assign(n_ctas + 1, 0);
+    const int base = (int)units.size();
+    size_t ti = 0;
+    int64_t tile_start = 0;  // global block index of tiles[ti]'s first block
+    for (int c = 0; c < n_ctas; ++c) {
+        cta_begin[c] = (int)units.size() - base;
+        const int64_t lo = total * c / n_ctas, hi = total * (c + 1) / n_ctas;
+        int64_t pos = lo;
+        while (pos < hi) {
+            while (ti < tiles.size() && tile_start + tiles[ti].nkb <= pos) {
+                tile_start += tiles[ti].nkb;
+                ++ti;
+            }
+            const Tile &t = tiles[ti];
+            const int64_t end = (tile_start + t.nkb < hi) ? tile_start + t.nkb : hi;
+            Unit u;
+            u.module = t.module;
+            u.side = t.side;
+            u.kb0 = (int32_t)(pos - tile_start);
+            u.nkb = (int32_t)(end - pos);
+            u.slot = slot0 + (int)units.size() - base;
+            u.cta = c;
+            units.push_back(u);
+            pos = end;
+        }
+    }
+    cta_begin[n_ctas] = (int)units.size() - base;
+}
+}  // namespace detail
+
+// tc_ok[m] != 0: module m may use the TMA + tcgen05 kernel.
+inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t *tc_ok, Plan &plan) {
+    plan.mode = mode_of_b(b);
+    plan.n_ctas = n_ctas;
+    plan.units.clear();
+    plan.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0});
+    std::vector<detail::Tile> tc, simt;
+    for (int m = 0; m < M; ++m) {
+        std::vector<detail::Tile> &dst = tc_ok[m] ? tc : simt;
+        if (plan.mode == kStacked) {
+            dst.push_back({m, 2, kblocks_of(d[m])});
+        } else {
+            dst.push_back({m, 0, kblocks_of(d[m])});
+            dst.push_back({m, 1, kblocks_of(d[m])});
+        }
+    }
+    detail::split_tiles(tc, n_ctas, 0, plan.units, plan.cta_begin_tc);
+    plan.n_units_tc = (int)plan.units.size();
+    detail::split_tiles(simt, n_ctas, plan.n_units_tc, plan.units, plan.cta_begin_simt);
+    const int pitch = pitch_of_mode(plan.mode);
+    for (const Unit &u : plan.units) {
+        for (int s = 0; s < 2; ++s) {
+            if (u.side != 2 && u.side != s) continue;
+            SideInfo &si = plan.sides[2 * (size_t)u.module + s];
+            if (si.n_slots == 0) si.first_slot = u.slot;
+            si.n_slots += 1;
+            si.side_off = (plan.mode == kStacked) ? s * 64 * 64 : 0;
+            si.pitch = pitch;
+        }
+    }
+}
+
+}  // namespace egeria

@@ -25,3 +25,10 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """The CUDA library is built in-tree (nvcc cross-compiles without a GPU)."""
+    from paper_2201_06227_b200 import build
+    build.build()

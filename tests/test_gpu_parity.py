@@ -1,0 +1,373 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 CPU oracle,
+element by element on the same seeded bf16 inputs.
+
+Tolerances (stated for the plasticity path): row-normalised Gram entries within 1e-4
+absolute; loss within 1e-3 relative or 1e-7 absolute; freeze masks identical except
+where the oracle's |slope| is within 1e-6 of T.
+"""
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2201_06227_b200 import binding as eg
+from paper_2201_06227_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = Path(__file__).parent / "golden"
+ENTRY_ATOL = 1e-4
+LOSS_RTOL, LOSS_ATOL = 1e-3, 1e-7
+DEV = "cuda"
+
+
+def assert_loss_close(gpu, ref, what=""):
+    gpu, ref = np.asarray(gpu, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    tol = np.maximum(LOSS_RTOL * np.abs(ref), LOSS_ATOL)
+    bad = ~(np.abs(gpu - ref) <= tol)
+    assert not bad.any(), f"{what} loss mismatch at {np.nonzero(bad)[0]}: gpu={gpu[bad]} oracle={ref[bad]}"
+
+
+def run_gpu(at, ar, flags=0, keep=False, W=5, T=1e-3):
+    """One evaluation through the C ABI.  at/ar: lists of CUDA bf16 [b, d_m] tensors."""
+    b = at[0].shape[0]
+    d = [t.shape[1] for t in at]
+    ctx = eg.Context(d, b, W, T, flags | (eg.FLAG_KEEP_GRAMS if keep else 0), device=DEV)
+    losses = ctx.egeria_sp_loss_batch(at, ar)
+    grams = [ctx.egeria_debug_dump_gram(m, b) for m in range(len(d))] if keep else None
+    ctx.check_device_status()
+    out = losses.cpu().numpy()
+    if keep:
+        grams = [(g[0].cpu().numpy(), g[1].cpu().numpy()) for g in grams]
+    ctx.close()
+    return out, grams
+
+
+def compare_with_oracle(at, ar, flags=0, what=""):
+    losses, grams = run_gpu(at, ar, flags, keep=True)
+    for m, (t, r) in enumerate(zip(at, ar)):
+        ref, gt, gr = oracle.sp_loss(wl.bf16_bits(t), wl.bf16_bits(r), return_grams=True)
+        np.testing.assert_allclose(grams[m][0], gt, rtol=0, atol=ENTRY_ATOL, err_msg=f"{what} G~_T module {m}")
+        np.testing.assert_allclose(grams[m][1], gr, rtol=0, atol=ENTRY_ATOL, err_msg=f"{what} G~_R module {m}")
+        assert_loss_close(losses[m:m + 1], [ref], f"{what} module {m}")
+    return losses
+
+
+# ----------------------------------------------------------------------------- small shapes
+
+SMALL_B = [2, 3, 8, 17, 32, 64, 65, 100, 128, 129, 200, 256]
+SMALL_D = [8, 64, 72, 4096, 4104]
+
+
+@pytest.mark.parametrize("b", SMALL_B)
+@pytest.mark.parametrize("d", SMALL_D)
+def test_single_module_tensor_core_path(b, d):
+    kind = "relu" if (b + d) % 2 == 0 else "normal"
+    at, ar = wl.make_pair(b, d, kind, 0.3, seed=1000 * b + d, device=DEV)
+    compare_with_oracle([at], [ar], what=f"b={b} d={d}")
+
+
+@pytest.mark.parametrize("b,d", [(2, 1), (5, 7), (8, 100), (64, 1001), (100, 333), (130, 250), (256, 65)])
+def test_single_module_cuda_core_path_for_unaligned_d(b, d):
+    at, ar = wl.make_pair(b, d, "normal", 0.3, seed=77 + b + d, device=DEV)
+    compare_with_oracle([at], [ar], what=f"b={b} d={d}")
+
+
+@pytest.mark.parametrize("b", [8, 64, 128, 256])
+def test_forced_cuda_core_path_matches_oracle(b):
+    at, ar = wl.make_pair(b, 2048, "relu", 0.2, seed=5 + b, device=DEV)
+    compare_with_oracle([at], [ar], flags=eg.FLAG_FORCE_SIMT, what=f"simt b={b}")
+
+
+def test_misaligned_pointer_takes_cuda_core_path():
+    b, d = 16, 264
+    base_t = torch.zeros(b * d + 8, dtype=torch.bfloat16, device=DEV)
+    base_r = torch.zeros(b * d + 8, dtype=torch.bfloat16, device=DEV)
+    t, r = wl.make_pair(b, d, "normal", 0.3, seed=9, device=DEV)
+    at = base_t[1:1 + b * d].view(b, d)   # 2-byte offset: not 16-byte aligned
+    ar = base_r[1:1 + b * d].view(b, d)
+    at.copy_(t)
+    ar.copy_(r)
+    assert at.data_ptr() % 16 != 0
+    compare_with_oracle([at], [ar], what="misaligned")
+
+
+@pytest.mark.parametrize("b", [24, 96, 160])
+def test_many_modules_mixed_sizes(b):
+    """Several tiles per CTA, K-ranges cut inside modules, ragged tails, one unaligned module."""
+    ds = [64, 8, 4104, 12345 * 8, 520, 1001, 30000, 72, 96 * 64]
+    at, ar = [], []
+    for m, d in enumerate(ds):
+        t, r = wl.make_pair(b, d, "relu" if m % 2 else "normal", 0.05 + 0.05 * m, seed=300 + m, device=DEV)
+        at.append(t)
+        ar.append(r)
+    compare_with_oracle(at, ar, what=f"mixed b={b}")
+
+
+# ----------------------------------------------------------------------------- closed forms / invariants on the GPU
+
+def _fixture_cases():
+    for line in (GOLDEN / "sp_loss_closed_forms.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        name, b, d, at, ar, exp = [f.strip() for f in line.split("|")]
+        parse = lambda s: [[float(v) for v in row.split()] for row in s.split(";")]
+        yield pytest.param(parse(at), parse(ar), float(exp), id=name)
+
+
+@pytest.mark.parametrize("at,ar,expected", list(_fixture_cases()))
+def test_closed_form_fixture_on_gpu(at, ar, expected):
+    t = torch.tensor(at, dtype=torch.bfloat16, device=DEV)
+    r = torch.tensor(ar, dtype=torch.bfloat16, device=DEV)
+    losses, _ = run_gpu([t], [r])
+    assert_loss_close(losses, [expected])
+
+
+@pytest.mark.parametrize("b,d", [(8, 4096), (64, 8192), (128, 4096), (256, 2048)])
+def test_invariants_on_gpu(b, d):
+    at, ar = wl.make_pair(b, d, "relu", 0.2, seed=b + d, device=DEV)
+    base, _ = run_gpu([at], [ar])
+    same, _ = run_gpu([at], [at.clone()])
+    assert abs(same[0]) <= 1e-7
+    again, _ = run_gpu([at], [ar])
+    assert again[0].tobytes() == base[0].tobytes()              # deterministic
+    scaled, _ = run_gpu([at * 4.0], [ar * 0.125])               # exact in bf16, exact in fp32
+    assert scaled[0].tobytes() == base[0].tobytes()
+    perm = torch.randperm(b, generator=torch.Generator().manual_seed(1)).to(DEV)
+    permuted, _ = run_gpu([at[perm].contiguous()], [ar[perm].contiguous()])
+    assert_loss_close(permuted, base.astype(np.float64))
+
+
+def test_nan_propagates_and_zero_rows_are_clamped():
+    at, ar = wl.make_pair(16, 256, "normal", 0.2, seed=3, device=DEV)
+    z = at.clone()
+    z[5] = 0
+    losses, grams = run_gpu([z], [ar], keep=True)
+    assert np.all(grams[0][0][5] == 0.0) and np.isfinite(losses).all()
+    ref = oracle.sp_loss(wl.bf16_bits(z), wl.bf16_bits(ar))
+    assert_loss_close(losses, [ref])
+    n = at.clone()
+    n[2, 7] = float("nan")
+    losses, _ = run_gpu([n], [ar])
+    assert np.isnan(losses[0])
+
+
+# ----------------------------------------------------------------------------- named workloads
+
+def test_tiny_workload_full():
+    w = wl.WORKLOADS["tiny"]
+    at, ar = wl.make_activations(w, DEV)
+    compare_with_oracle(at, ar, what="tiny")
+
+
+def test_resnet56_workload_full():
+    w = wl.WORKLOADS["resnet56"]
+    at, ar = wl.make_activations(w, DEV)
+    compare_with_oracle(at, ar, what="resnet56")
+
+
+def test_bert_base_workload_full():
+    w = wl.WORKLOADS["bert_base"]
+    at, ar = wl.make_activations(w, DEV)
+    compare_with_oracle(at, ar, what="bert_base")
+
+
+def _sampled_check(name, full_modules, row_modules, rows):
+    """Full-size workload in the benchmark's launch configuration; the oracle checks the
+    whole loss of a few modules and sampled rows of the normalised Grams of others."""
+    w = wl.WORKLOADS[name]
+    at, ar = wl.make_activations(w, DEV)
+    losses, grams = run_gpu(at, ar, keep=True, W=w.W, T=w.T)
+    assert np.isfinite(losses).all() and np.all(losses >= 0) and np.all(losses <= 4.0 / w.b)
+    for m in full_modules:
+        ref, gt, gr = oracle.sp_loss(wl.bf16_bits(at[m]), wl.bf16_bits(ar[m]), return_grams=True)
+        np.testing.assert_allclose(grams[m][0], gt, rtol=0, atol=ENTRY_ATOL)
+        np.testing.assert_allclose(grams[m][1], gr, rtol=0, atol=ENTRY_ATOL)
+        assert_loss_close(losses[m:m + 1], [ref], f"{name} module {m}")
+    for m in row_modules:
+        for side, acts in enumerate((at, ar)):
+            bits = wl.bf16_bits(acts[m])
+            for i in rows:
+                g = oracle.gram_row(bits, i)
+                gn = g / max(np.linalg.norm(g), oracle.EPS)
+                np.testing.assert_allclose(grams[m][side][i], gn, rtol=0, atol=ENTRY_ATOL)
+    # properties that hold at any size: unit rows, symmetric-positive diagonal
+    for m in range(w.M):
+        for side in (0, 1):
+            np.testing.assert_allclose(np.linalg.norm(grams[m][side].astype(np.float64), axis=1), 1.0, atol=1e-5)
+            assert np.all(np.diag(grams[m][side]) > 0)
+
+
+def test_resnet50_workload_sampled():
+    _sampled_check("resnet50", full_modules=[0, 5, 15], row_modules=[3, 9, 12], rows=[0, 31, 63])
+
+
+def test_gpt2_medium_workload_sampled():
+    _sampled_check("gpt2_medium", full_modules=[0, 23], row_modules=[7, 11, 16], rows=[0, 127, 128, 255])
+
+
+# ----------------------------------------------------------------------------- host entry point
+
+def test_host_entry_matches_device_entry():
+    ds, b = [4096, 520, 1001], 48
+    at, ar = [], []
+    for m, d in enumerate(ds):
+        t, r = wl.make_pair(b, d, "relu", 0.2, seed=40 + m, device="cpu")
+        at.append(t.pin_memory())
+        ar.append(r.pin_memory())
+    ctx = eg.Context(ds, b, 5, 1e-3, eg.FLAG_HOST_STAGING, device=DEV)
+    host = ctx.egeria_sp_loss_batch_host(at, ar).numpy().copy()
+    dev = ctx.egeria_sp_loss_batch([t.to(DEV) for t in at], [r.to(DEV) for r in ar]).cpu().numpy()
+    assert host.tobytes() == dev.tobytes()
+    ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+    assert_loss_close(host, ref)
+    ctx.close()
+
+
+def test_call_error_paths():
+    at, ar = wl.make_pair(8, 64, "normal", 0.1, seed=1, device=DEV)
+    ctx = eg.Context([64], 8, 5, 1e-3, device=DEV)
+    big_t, big_r = wl.make_pair(16, 64, "normal", 0.1, seed=1, device=DEV)
+    with pytest.raises(eg.EgeriaError) as e:
+        ctx.egeria_sp_loss_batch([big_t], [big_r])       # b > b_max
+    assert e.value.status == eg.ERR_INVALID_ARG
+    with pytest.raises(eg.EgeriaError) as e:
+        ctx.egeria_sp_loss_batch_host([at.cpu()], [ar.cpu()])   # no staging reserved
+    assert e.value.status == eg.ERR_WORKSPACE
+    with pytest.raises(eg.EgeriaError) as e:
+        ctx.egeria_debug_dump_gram(0, 8)                 # grams not kept
+    assert e.value.status == eg.ERR_WORKSPACE
+    out = ctx.egeria_sp_loss_batch([at], [ar])           # still usable afterwards
+    assert np.isfinite(out.cpu().numpy()).all()
+    ctx.close()
+
+
+def test_changing_b_and_pointers_between_calls():
+    ctx = eg.Context([4096, 264], 128, 5, 1e-3, device=DEV)
+    for b in (128, 8, 70, 8):
+        at, ar = [], []
+        for m, d in enumerate((4096, 264)):
+            t, r = wl.make_pair(b, d, "relu", 0.2, seed=b + m, device=DEV)
+            at.append(t)
+            ar.append(r)
+        got = ctx.egeria_sp_loss_batch(at, ar).cpu().numpy()
+        ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+        assert_loss_close(got, ref, f"b={b}")
+    ctx.check_device_status()
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- freezing rule
+
+def masks_agree(gpu_mask, gpu_fe, hist, W, T, signed=False):
+    for m in range(hist.shape[0]):
+        ref = oracle.plasticity_replay(hist[m], W, T, signed_test=signed)
+        s = ref["slopes"][np.isfinite(ref["slopes"])]
+        near = np.any(np.abs((s if signed else np.abs(s)) - T) <= 1e-6) if len(s) else False
+        if near:
+            continue
+        assert bool(gpu_mask[m]) == ref["converged"], f"module {m}"
+        assert int(gpu_fe[m]) == ref["freeze_eval"], f"module {m}"
+
+
+@pytest.mark.parametrize("name,level", [("resnet56", None), ("resnet56", 1e-2), ("resnet50", 2e-2),
+                                        ("bert_base", 5e-3), ("gpt2_medium", 3e-2)])
+def test_replay_matches_oracle(name, level):
+    w = wl.WORKLOADS[name]
+    levels = [1e-6 * (1 + l) for l in range(w.M)] if level is None else [level * (1 + 0.1 * l) for l in range(w.M)]
+    hist = wl.make_history(w, levels)
+    T32 = np.float32(w.T)
+    ctx = eg.Context([64] * w.M, 8, w.W, float(T32), device=DEV)
+    slopes, mask, fe = ctx.egeria_plasticity_replay(torch.from_numpy(hist).to(DEV))
+    slopes, mask, fe = slopes.cpu().numpy(), mask.cpu().numpy(), fe.cpu().numpy()
+    n_conv = 0
+    for m in range(w.M):
+        ref = oracle.plasticity_replay(hist[m], w.W, float(T32))
+        live = ~np.isnan(ref["slopes"])
+        assert np.array_equal(np.isnan(slopes[m]), ~live) or not ref["converged"]
+        np.testing.assert_allclose(slopes[m][live], ref["slopes"][live], rtol=1e-9, atol=1e-15)
+        n_conv += ref["converged"]
+    masks_agree(mask, fe, hist, w.W, float(T32))
+    if level is not None and name != "bert_base":
+        assert 0 < n_conv < w.M, "the synthetic history should give a non-trivial mask"
+    ctx.close()
+
+
+@pytest.mark.parametrize("signed", [False, True])
+def test_step_matches_replay_and_oracle(signed):
+    M, W, T, H = 6, 4, np.float32(2e-3), 40
+    rng = np.random.default_rng(5)
+    k = np.arange(H)
+    hist = np.stack([0.05 * np.exp(-k / (2.0 + 3 * m)) * (1 + 0.5 * (m % 2) * np.sin(k)) + 0.01
+                     + 1e-4 * rng.normal(size=H) for m in range(M)]).astype(np.float32)
+    flags = eg.FLAG_SIGNED_SLOPE if signed else 0
+    ctx = eg.Context([64] * M, 8, W, float(T), flags, device=DEV)
+    hist_dev = torch.from_numpy(hist).to(DEV)
+    step_slopes = np.empty((M, H))
+    step_mask = np.empty((M, H), dtype=np.uint8)
+    for i in range(H):
+        s, mk = ctx.egeria_plasticity_step(hist_dev[:, i].contiguous())
+        step_slopes[:, i], step_mask[:, i] = s.cpu().numpy(), mk.cpu().numpy()
+    for m in range(M):
+        for i in (3, 10, H - 1):
+            ref = oracle.plasticity_replay(hist[m, : i + 1], W, float(T), signed_test=signed)
+            sl = ref["slopes"][np.isfinite(ref["slopes"]) | np.isinf(ref["slopes"])]
+            near = np.any(np.abs(np.abs(sl[np.isfinite(sl)]) - T) <= 1e-6)
+            if not near:
+                assert bool(step_mask[m, i]) == ref["converged"]
+            if not ref["converged"]:
+                assert step_slopes[m, i] == pytest.approx(ref["slopes"][i], rel=1e-9, abs=1e-15)
+    # reset clears the state; halving the window follows the unfreezing rule
+    ctx.egeria_plasticity_reset(halve_W=True)
+    assert ctx.egeria_plasticity_window() == 2
+    s, mk = ctx.egeria_plasticity_step(hist_dev[:, 0].contiguous())
+    assert np.all(np.isinf(s.cpu().numpy())) and not mk.cpu().numpy().any()
+    ctx.close()
+
+
+def test_alg1_hand_traces_on_gpu():
+    from fractions import Fraction
+    for line in (GOLDEN / "alg1_traces.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        f = [s.strip() for s in line.split("|")]
+        W, T, signed = int(f[1]), float(f[2]), bool(int(f[3]))
+        hist = np.array([[float(v) for v in f[4].split()]], dtype=np.float32)
+        ctx = eg.Context([64], 8, W, T, eg.FLAG_SIGNED_SLOPE if signed else 0, device=DEV)
+        slopes, mask, fe = ctx.egeria_plasticity_replay(torch.from_numpy(hist).to(DEV))
+        assert int(fe[0]) == int(f[8]), f[0]
+        assert bool(mask[0]) == (int(f[8]) >= 0)
+        for i, tok in enumerate(f[6].split()):
+            got = float(slopes[0, i])
+            if tok == "x":
+                assert np.isnan(got)
+            elif tok == "inf":
+                assert np.isinf(got)
+            else:
+                assert got == pytest.approx(float(Fraction(tok)), rel=1e-6, abs=1e-7)
+        ctx.close()
+
+
+def test_tiny_end_to_end_chain():
+    """20 real evaluations of the tiny workload: GPU losses -> GPU slopes/mask against
+    oracle losses -> oracle slopes/mask."""
+    w = wl.WORKLOADS["tiny"]
+    T32 = float(np.float32(w.T))
+    ctx = eg.Context(list(w.d), w.b, w.W, T32, device=DEV)
+    gpu_losses, ref_losses, masks = [], [], []
+    for k, sigma in enumerate(wl.tiny_history_sigmas(w)):
+        at, ar = wl.make_module(w, 0, DEV, sigma=sigma, seed_offset=k)
+        out = ctx.egeria_sp_loss_batch([at], [ar])
+        s, mk = ctx.egeria_plasticity_step(out)
+        gpu_losses.append(float(out.cpu()[0]))
+        masks.append(int(mk.cpu()[0]))
+        ref_losses.append(oracle.sp_loss(wl.bf16_bits(at), wl.bf16_bits(ar)))
+    assert_loss_close(gpu_losses, ref_losses, "tiny history")
+    ref = oracle.plasticity_replay(np.array(ref_losses, dtype=np.float32), w.W, T32)
+    sl = ref["slopes"][np.isfinite(ref["slopes"])]
+    if not np.any(np.abs(np.abs(sl) - T32) <= 1e-6):
+        assert bool(masks[-1]) == ref["converged"]
+    ctx.check_device_status()
+    ctx.close()

@@ -1,0 +1,140 @@
+"""CPU-only checks of the C-ABI library: it loads, exports what the header declares,
+and its host-side logic (argument checks, workspace sizing, work split) is right.
+No compute call is made here."""
+import ctypes
+import re
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+from paper_2201_06227_b200 import binding as eg
+from paper_2201_06227_b200 import workloads as wl
+
+HEADER = Path(__file__).resolve().parent.parent / "include" / "egeria.h"
+
+
+def declared_symbols():
+    text = re.sub(r"/\*.*?\*/", "", HEADER.read_text(), flags=re.S)
+    return sorted(set(re.findall(r"\b(egeria_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    L = eg.lib()
+    names = declared_symbols()
+    assert len(names) >= 12
+    for name in names:
+        assert hasattr(L, name), f"{name} is declared in egeria.h but not exported"
+    assert sorted(eg.EXPORTS) == names
+
+
+def test_status_strings():
+    for s in range(7):
+        assert eg.status_string(s) not in ("", "unknown status")
+    assert eg.status_string(99) == "unknown status"
+
+
+def test_workspace_bytes_is_pure_and_monotone():
+    d = [4096, 8192]
+    base = eg.egeria_workspace_bytes(2, d, 64, 10)
+    assert base > 0 and base % eg.WORKSPACE_ALIGN == 0
+    assert eg.egeria_workspace_bytes(2, d, 64, 10) == base
+    assert eg.egeria_workspace_bytes(2, d, 128, 10) > base
+    assert eg.egeria_workspace_bytes(2, d, 256, 10) > eg.egeria_workspace_bytes(2, d, 128, 10)
+    keep = eg.egeria_workspace_bytes(2, d, 64, 10, eg.FLAG_KEEP_GRAMS)
+    assert keep >= base + 2 * 2 * 64 * 64 * 4
+    stage = eg.egeria_workspace_bytes(2, d, 64, 10, eg.FLAG_HOST_STAGING)
+    assert stage >= base + 2 * 64 * sum(d) * 2
+
+
+@pytest.mark.parametrize("M,d,b,W", [(0, [8], 8, 5), (1, [0], 8, 5), (1, [8], 1, 5), (1, [8], 257, 5),
+                                     (1, [8], 8, 0), (1, [8], 8, 100000), (1, [2 ** 31], 8, 5)])
+def test_workspace_bytes_rejects_bad_arguments(M, d, b, W):
+    assert eg.egeria_workspace_bytes(M, d, b, W) == 0
+
+
+def _create(M, d, b_max, W, ws_ptr, ws_bytes, flags=0):
+    h = ctypes.c_void_p()
+    st = eg.lib().egeria_plasticity_create(ctypes.byref(h), M, eg._i64(d), b_max, W, None,
+                                           ctypes.c_float(1e-3), ctypes.c_void_p(ws_ptr), ws_bytes, flags)
+    return st, h
+
+
+def test_create_error_paths_need_no_gpu():
+    assert _create(0, [8], 8, 5, 0, 0)[0] == eg.ERR_INVALID_ARG
+    assert _create(1, [8], 1, 5, 0, 0)[0] == eg.ERR_INVALID_ARG
+    assert _create(1, [8], 300, 5, 0, 0)[0] == eg.ERR_UNSUPPORTED_SHAPE
+    assert _create(1, [-4], 8, 5, 0, 0)[0] == eg.ERR_UNSUPPORTED_SHAPE
+    assert _create(1, [8], 8, 5, 0, 0)[0] == eg.ERR_WORKSPACE             # NULL workspace
+    assert _create(1, [8], 8, 5, 1024 + 8, 1 << 30)[0] == eg.ERR_WORKSPACE  # misaligned
+    assert _create(1, [8], 8, 5, 4096, 16)[0] == eg.ERR_WORKSPACE          # too small
+    L = eg.lib()
+    assert L.egeria_plasticity_create(None, 1, eg._i64([8]), 8, 5, None, ctypes.c_float(0), None, 0, 0) \
+        == eg.ERR_INVALID_ARG
+    assert L.egeria_plasticity_destroy(None) == eg.ERR_INVALID_ARG
+    assert L.egeria_device_status(None) == eg.ERR_INVALID_ARG
+    assert L.egeria_plasticity_step(None, None, None, None, None) == eg.ERR_INVALID_ARG
+    assert L.egeria_plasticity_window(None) == 0
+
+
+def test_create_without_a_device_fails_loudly():
+    """With a valid workspace pointer but no sm_100 device the call must fail, never fall back."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    n = eg.egeria_workspace_bytes(1, [64], 8, 5)
+    st, h = _create(1, [64], 8, 5, 1 << 20, n)
+    assert st in (eg.ERR_CUDA, eg.ERR_UNSUPPORTED_DEVICE)
+    assert not h.value
+
+
+# ----------------------------------------------------------------------------- the work split
+
+def _check_plan(d, b, n_ctas):
+    units = eg.egeria_debug_plan(d, b, n_ctas)
+    M = len(d)
+    sides = [2] if b <= 64 else [0, 1]
+    nkb = [(x + 63) // 64 for x in d]
+    # every (module, side) is covered exactly once, by contiguous ascending ranges
+    for m in range(M):
+        for s in sides:
+            rows = units[(units[:, 0] == m) & (units[:, 1] == s)]
+            assert len(rows) >= 1
+            pos = 0
+            for r in rows:
+                assert r[2] == pos and r[3] >= 1
+                pos += r[3]
+            assert pos == nkb[m]
+    assert len(units) == sum(len(units[(units[:, 0] == m)]) for m in range(M))
+    # unit count bound used for workspace sizing
+    assert len(units) <= len(sides) * M + 2 * n_ctas
+    # balance among tensor-core-eligible work: per-CTA block counts differ by at most 1
+    tc = units[np.isin(units[:, 0], [m for m in range(M) if d[m] % 8 == 0])]
+    if len(tc):
+        per = np.bincount(tc[:, 4], weights=tc[:, 3], minlength=n_ctas)
+        assert per.max() - per.min() <= 1
+    # CTAs are visited in order
+    assert np.all(np.diff(tc[:, 4]) >= 0)
+    return units
+
+
+@pytest.mark.parametrize("name", wl.ORDER)
+def test_plan_covers_named_workloads(name):
+    w = wl.WORKLOADS[name]
+    _check_plan(list(w.d), w.b, 148)
+
+
+@pytest.mark.parametrize("d,b,n", [([8], 2, 148), ([64, 72, 4104], 17, 148), ([4096] * 5, 100, 7),
+                                   ([1000, 24, 8], 256, 3), ([63, 65, 130], 129, 148), ([4096], 8, 1)])
+def test_plan_odd_shapes(d, b, n):
+    _check_plan(d, b, n)
+
+
+def test_plan_rejects_bad_arguments():
+    out = np.zeros((4, 5), dtype=np.int32)
+    n = ctypes.c_int()
+    L = eg.lib()
+    p = out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+    assert L.egeria_debug_plan(1, eg._i64([8]), 8, 0, p, 4, ctypes.byref(n)) == eg.ERR_INVALID_ARG
+    assert L.egeria_debug_plan(1, eg._i64([8]), 400, 4, p, 4, ctypes.byref(n)) == eg.ERR_UNSUPPORTED_SHAPE
+    assert L.egeria_debug_plan(1, eg._i64([8]), 8, 4, None, 4, ctypes.byref(n)) == eg.ERR_INVALID_ARG
