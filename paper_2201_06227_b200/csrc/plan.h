@@ -67,10 +67,11 @@ struct Plan {
 
 inline int64_t kblocks_of(int64_t d) { return (d + kKBlock - 1) / kKBlock; }
 
-// Upper bound on the number of units (hence slots) for any b of one mode.
+// Upper bound on the number of units (hence slots) for any b of one mode: every tile, plus
+// one extra unit per CTA boundary in each of the two splits (tensor-core and CUDA-core).
 inline int64_t max_units(int M, int mode, int n_ctas) {
     int64_t tiles = (mode == kStacked) ? M : 2 * (int64_t)M;
-    return tiles + n_ctas;
+    return tiles + 2 * (int64_t)n_ctas;
 }
 
 namespace detail {
