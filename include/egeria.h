@@ -166,6 +166,31 @@ egeria_status egeria_debug_plan(int M, const int64_t *d, int b, int n_ctas, int3
  * (the kernel then skipped its remaining work; results are invalid). */
 egeria_status egeria_device_status(egeria_ctx *ctx);
 
+/* Plasticity of ONE module with no workspace and no allocation of any kind.
+ * The paper has no counterpart to this call; it exists for callers that cannot
+ * obtain device memory at the moment they need an evaluation: code that runs
+ * where cudaMalloc is forbidden or would stall (a framework whose caching
+ * allocator owns all of HBM so that a raw allocation fails, a latency-critical
+ * loop that must avoid the device-wide synchronisation an allocation or free
+ * implies, a plugin that is handed a stream but no allocator).  Such callers
+ * cannot size and allocate the workspace a context needs either.
+ *
+ * The scratch of this call (partial Gram matrices, work split, tensor maps) is
+ * a fixed 6 MiB array inside the library image; every GPU that loads the
+ * library holds it until the process exits.  The price is a size limit:
+ *   b  2..128 (larger b returns EGERIA_ERR_UNSUPPORTED_SHAPE), any d >= 1,
+ * and the feature axis is split over 32 CTAs only, so it is slower than a
+ * context on large d.  Same arithmetic as egeria_sp_loss_batch.
+ *   At, Ar    device bf16 [b, d] (caller-owned)     out_loss  device float [1]
+ * The first call on each device looks up the array's device address and sets
+ * kernel attributes (with that device current); make that first call outside
+ * any stream capture.  All calls share the one array, which keeps the previous
+ * call's contents (the call clears the words that must start at zero): two
+ * calls that overlap on the GPU, from different streams or threads, race.
+ * Calls on one stream are safe back to back.  Not thread-safe. */
+egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At, const void *Ar, int b,
+                                    int64_t d, float *out_loss);
+
 /* Measurement hook (needs EGERIA_FLAG_TIME_GRAM): device time, in milliseconds,
  * spent in the Gram kernels of the egeria_sp_loss_batch calls made since the
  * last query (the finalisation kernel is not included), and the number of those

@@ -26,7 +26,7 @@ EXPORTS = [
     "egeria_sp_loss_batch", "egeria_sp_loss_batch_host", "egeria_plasticity_step",
     "egeria_plasticity_replay", "egeria_plasticity_reset", "egeria_plasticity_window",
     "egeria_debug_dump_gram", "egeria_debug_plan", "egeria_device_status", "egeria_launch_count",
-    "egeria_gram_kernel_time",
+    "egeria_gram_kernel_time", "egeria_sp_loss_static",
     "egeria_status_string",
 ]
 
@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
                                     ctypes.POINTER(ctypes.c_int32), ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
     L.egeria_device_status.argtypes = [vp]
     L.egeria_gram_kernel_time.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
+    L.egeria_sp_loss_static.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_int64, vp]
     L.egeria_launch_count.argtypes = [vp]
     L.egeria_launch_count.restype = ctypes.c_int64
     L.egeria_status_string.argtypes = [ctypes.c_int]
@@ -108,6 +109,25 @@ def egeria_debug_plan(d: Sequence[int], b: int, n_ctas: int) -> np.ndarray:
                                  out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), cap, ctypes.byref(n))
     _check(st, "egeria_debug_plan")
     return out[: n.value].copy()
+
+
+def egeria_sp_loss_static(At: torch.Tensor, Ar: torch.Tensor, out_loss: Optional[torch.Tensor] = None,
+                          stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Plasticity of one module through the entry point that allocates nothing.
+
+    The library uses only its built-in scratch array; `out_loss` (device float[1]) is the
+    caller's.  Pass it in to keep this wrapper allocation-free as well."""
+    if At.dtype != torch.bfloat16 or At.shape != Ar.shape or At.dim() != 2 or not (At.is_cuda and Ar.is_cuda):
+        raise ValueError("expected two CUDA bfloat16 [b, d] tensors of the same shape")
+    if not (At.is_contiguous() and Ar.is_contiguous()):
+        raise ValueError("activations must be contiguous")
+    if out_loss is None:
+        out_loss = torch.empty(1, dtype=torch.float32, device=At.device)
+    with torch.cuda.device(At.device):
+        st = lib().egeria_sp_loss_static(_stream_ptr(stream), At.data_ptr(), Ar.data_ptr(), int(At.shape[0]),
+                                         int(At.shape[1]), out_loss.data_ptr())
+    _check(st, "egeria_sp_loss_static")
+    return out_loss
 
 
 class Context:

@@ -538,3 +538,176 @@ egeria_status egeria_device_status(egeria_ctx *ctx) {
 }
 
 }  // extern "C"
+
+// =====================================================================================
+// Allocation-free single-module evaluation (egeria_sp_loss_static).
+//
+// All scratch of this entry point is the fixed array below, which is part of the library
+// image: every GPU that loads the library carries these 6 MiB until the process exits.
+// Nothing here calls cudaMalloc, cudaFree or any routine that allocates device memory.
+// =====================================================================================
+namespace egeria {
+
+constexpr int kStaticMaxB = 128;                   // largest b of the allocation-free entry point
+constexpr int kStaticCtas = 32;                    // CTAs the feature axis is split over
+constexpr size_t kStaticScratchBytes = 6u << 20;   // 6 MiB
+constexpr int kStaticMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticLayout {
+    size_t tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides, rowloss, ticket, slots, total;
+};
+
+static StaticLayout static_layout() {
+    StaticLayout L;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t o = off;
+        off = align_up(off + bytes, 256);
+        return o;
+    };
+    L.tmaps = take(2 * sizeof(CUtensorMap));
+    L.modules = take(sizeof(ModulePtrs));
+    L.units = take((size_t)max_units(1, kSingle1, kStaticCtas) * sizeof(Unit));
+    L.cta_begin_tc = take((kStaticCtas + 1) * sizeof(int32_t));
+    L.cta_begin_simt = take((kStaticCtas + 1) * sizeof(int32_t));
+    L.sides = take(2 * sizeof(SideInfo));
+    L.rowloss = take(kMaxB * sizeof(double));
+    L.ticket = take(2 * sizeof(int32_t));  // [0] finalisation ticket, [1] status word
+    L.slots = take((size_t)max_units(1, kSingle1, kStaticCtas) * slot_floats_of_mode(kSingle1) * sizeof(float));
+    L.total = off;
+    return L;
+}
+
+// Per-device set-up state.  g_static_scratch is a host-side stand-in for the symbol, not a
+// device address: the address a kernel may use comes from cudaGetSymbolAddress, asked once
+// per device with that device current.
+struct StaticDevice {
+    unsigned char *scratch = nullptr;
+    EncodeTiledFn encode = nullptr;
+};
+static StaticDevice g_static_dev[kStaticMaxDevices];
+
+static egeria_status static_setup(int dev, StaticDevice **out) {
+    if (dev < 0 || dev >= kStaticMaxDevices) return EGERIA_ERR_UNSUPPORTED_DEVICE;
+    StaticDevice &sd = g_static_dev[dev];
+    if (!sd.scratch) {
+        cudaDeviceProp prop;
+        EG_CUDA(cudaGetDeviceProperties(&prop, dev));
+        if (prop.major != 10) return EGERIA_ERR_UNSUPPORTED_DEVICE;
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return EGERIA_ERR_CUDA;
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || !fn)
+            return EGERIA_ERR_CUDA;
+        EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kStacked>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     TcCfg<kStacked>::kSmemBytes));
+        EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kSingle1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     TcCfg<kSingle1>::kSmemBytes));
+        sd.encode = reinterpret_cast<EncodeTiledFn>(fn);
+        sd.scratch = static_cast<unsigned char *>(ptr);
+    }
+    *out = &sd;
+    return EGERIA_OK;
+}
+
+}  // namespace egeria
+
+extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At, const void *Ar, int b, int64_t d,
+                                               float *out_loss) {
+    if (!At || !Ar || !out_loss || b < 2) return EGERIA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(At) | reinterpret_cast<uintptr_t>(Ar)) & 1) return EGERIA_ERR_INVALID_ARG;
+    if (b > kStaticMaxB) return EGERIA_ERR_UNSUPPORTED_SHAPE;  // beyond the fixed scratch
+    if (d < 1 || d > (int64_t)0x7fffffff - 2 * kKBlock) return EGERIA_ERR_UNSUPPORTED_SHAPE;
+    const StaticLayout L = static_layout();
+    static_assert(kStaticScratchBytes >= (5u << 20), "scratch array too small for its layout");
+    if (L.total > kStaticScratchBytes) return EGERIA_ERR_WORKSPACE;
+
+    int dev = 0;
+    EG_CUDA(cudaGetDevice(&dev));
+    StaticDevice *sd = nullptr;
+    egeria_status s = static_setup(dev, &sd);
+    if (s != EGERIA_OK) return s;
+    unsigned char *ws = sd->scratch;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    const uint8_t tc_ok = (reinterpret_cast<uintptr_t>(At) % 16 == 0) && (reinterpret_cast<uintptr_t>(Ar) % 16 == 0) &&
+                          (d % 8 == 0);
+    Plan P;
+    build_plan(1, &d, b, kStaticCtas, &tc_ok, P);
+    if ((int64_t)P.units.size() > max_units(1, kSingle1, kStaticCtas)) return EGERIA_ERR_WORKSPACE;
+
+    CUtensorMap maps[2];
+    memset(maps, 0, sizeof(maps));
+    if (tc_ok) {
+        const int box_rows = (P.mode == kStacked) ? 64 : 128;
+        const void *bases[2] = {At, Ar};
+        for (int side = 0; side < 2; ++side) {
+            cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)b};
+            cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+            cuuint32_t box[2] = {(cuuint32_t)kKBlock, (cuuint32_t)box_rows};
+            cuuint32_t estr[2] = {1, 1};
+            if (sd->encode(&maps[side], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(bases[side]), dims,
+                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return EGERIA_ERR_CUDA;
+        }
+    }
+    const ModulePtrs mod{At, Ar, d};
+    // The array keeps whatever the previous call left: the ticket and the status word must
+    // start at zero; everything else is overwritten before it is read.
+    EG_CUDA(cudaMemsetAsync(ws + L.ticket, 0, 2 * sizeof(int32_t), stream));
+    EG_CUDA(cudaMemcpyAsync(ws + L.tmaps, maps, sizeof(maps), cudaMemcpyHostToDevice, stream));
+    EG_CUDA(cudaMemcpyAsync(ws + L.modules, &mod, sizeof(mod), cudaMemcpyHostToDevice, stream));
+    EG_CUDA(cudaMemcpyAsync(ws + L.units, P.units.data(), P.units.size() * sizeof(Unit), cudaMemcpyHostToDevice,
+                            stream));
+    EG_CUDA(cudaMemcpyAsync(ws + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, stream));
+    EG_CUDA(cudaMemcpyAsync(ws + L.cta_begin_simt, P.cta_begin_simt.data(), P.cta_begin_simt.size() * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, stream));
+    EG_CUDA(cudaMemcpyAsync(ws + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo), cudaMemcpyHostToDevice,
+                            stream));
+
+    const int64_t slot_floats = slot_floats_of_mode(P.mode);
+    int32_t *ticket = reinterpret_cast<int32_t *>(ws + L.ticket);
+    if (P.n_units_tc > 0) {
+        TcParams tp;
+        tp.tmaps = reinterpret_cast<const CUtensorMap *>(ws + L.tmaps);
+        tp.units = reinterpret_cast<const Unit *>(ws + L.units);
+        tp.cta_begin = reinterpret_cast<const int32_t *>(ws + L.cta_begin_tc);
+        tp.slots = reinterpret_cast<float *>(ws + L.slots);
+        tp.slot_floats = slot_floats;
+        tp.b = b;
+        tp.status = ticket + 1;
+        if (P.mode == kStacked)
+            gram_tc_kernel<kStacked><<<kStaticCtas, kTcThreads, TcCfg<kStacked>::kSmemBytes, stream>>>(tp);
+        else
+            gram_tc_kernel<kSingle1><<<kStaticCtas, kTcThreads, TcCfg<kSingle1>::kSmemBytes, stream>>>(tp);
+    } else {
+        SimtParams sp;
+        sp.modules = reinterpret_cast<const ModulePtrs *>(ws + L.modules);
+        sp.units = reinterpret_cast<const Unit *>(ws + L.units);
+        sp.cta_begin = reinterpret_cast<const int32_t *>(ws + L.cta_begin_simt);
+        sp.slots = reinterpret_cast<float *>(ws + L.slots);
+        sp.slot_floats = slot_floats;
+        sp.b = b;
+        sp.mode = P.mode;
+        gram_simt_kernel<<<kStaticCtas, kSimtThreads, 0, stream>>>(sp);
+    }
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    FinParams fp;
+    fp.slots = reinterpret_cast<const float *>(ws + L.slots);
+    fp.slot_floats = slot_floats;
+    fp.sides = reinterpret_cast<const SideInfo *>(ws + L.sides);
+    fp.b = b;
+    fp.out_losses = out_loss;
+    fp.rowloss = reinterpret_cast<double *>(ws + L.rowloss);
+    fp.tickets = ticket;
+    fp.keep = nullptr;
+    finalize_kernel<<<dim3(1, (b + kFinRowsPerCta - 1) / kFinRowsPerCta), kFinThreads, 0, stream>>>(fp);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    return EGERIA_OK;
+}
