@@ -148,6 +148,44 @@ def run_reference(args):
 
 # ----------------------------------------------------------------------------- our arm
 
+def pick_workload(args) -> wl.Workload:
+    w = wl.WORKLOADS[args.workload]
+    if args.modules and args.modules < w.M:
+        import dataclasses
+        w = dataclasses.replace(w, d=w.d[: args.modules])   # first modules only (profiling captures)
+    return w
+
+
+def n_sets_for(w: wl.Workload) -> int:
+    """Input sets to rotate over so that timed reads come from HBM, not from the 126 MB L2."""
+    if w.input_bytes > 4 * 126e6:
+        return 1
+    return min(16, max(2, int(np.ceil(8 * 126e6 / w.input_bytes))))
+
+
+def measure_other(eg, name, device, stream, steps, warmup):
+    """Short device-timed run of another named workload (context for the headline line)."""
+    w = wl.WORKLOADS[name]
+    n_sets = n_sets_for(w)
+    ctx, step, outs, sets, l0 = time_workload(eg, w, device, steps, warmup, n_sets, stream)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for i in range(steps):
+        step(warmup + i)
+    ev1.record(stream)
+    torch.cuda.synchronize(device)
+    ms = ev0.elapsed_time(ev1) / steps
+    gram_ms, calls = ctx.egeria_gram_kernel_time()
+    ctx.check_device_status()
+    ctx.close()
+    peak, _ = hbm_peak()
+    gram_s = gram_ms / max(1, calls) * 1e-3
+    return {"b": w.b, "modules": w.M, "input_bytes_per_step": w.input_bytes, "ms_per_step": ms,
+            "value": w.M / (ms * 1e-3), "gram_kernel_ms": gram_s * 1e3,
+            "gram_GBps": w.input_bytes / gram_s / 1e9, "roofline_frac": w.input_bytes / gram_s / 1e9 / peak,
+            "step_frac_of_hbm_roofline": (w.input_bytes / (peak * 1e9)) / (ms * 1e-3), "input_sets": n_sets}
+
+
 def time_workload(eg, w, device, steps, warmup, n_sets, stream, time_gram=True):
     """Device-timed steps of one workload.  Returns (seconds, gram_ms_per_call, launches_per_step, ctx, data)."""
     sets = []
@@ -197,9 +235,8 @@ def run_ours(args):
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     stream = torch.cuda.current_stream(device)
-    w = wl.WORKLOADS[args.workload]
-    n_sets = 1 if w.input_bytes > 4 * 126e6 else max(2, int(np.ceil(8 * 126e6 / w.input_bytes)))
-    n_sets = min(n_sets, 16)
+    w = pick_workload(args)
+    n_sets = n_sets_for(w)
 
     ctx, step, outs, sets, l0 = time_workload(eg, w, device, args.steps, args.warmup, n_sets, stream)
 
@@ -286,6 +323,12 @@ def run_ours(args):
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
         cpu_baseline, _, _ = oracle_sample(w)
+    others = None
+    if world == 1 and not args.no_others:
+        ctx.close()
+        del sets, step
+        torch.cuda.empty_cache()
+        others = {n: measure_other(eg, n, device, stream, 20, 5) for n in wl.ORDER if n != w.name}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
@@ -296,8 +339,9 @@ def run_ours(args):
                    "cache": ("inputs larger than L2" if n_sets == 1 else
                              f"rotating {n_sets} input sets ({n_sets * w.input_bytes / 1e6:.0f} MB) larger than L2")},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-        "cpu_baseline": cpu_baseline,
+        "cpu_baseline": cpu_baseline, "other_workloads": others,
     }
+    line["roofline"]["step_frac"] = (w.input_bytes / (peak * 1e9)) / (elapsed_ms * 1e-3 / args.steps)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
@@ -314,6 +358,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the short runs of the other workloads")
+    ap.add_argument("--modules", type=int, default=0, help="use only the first N modules (profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":

@@ -19,14 +19,19 @@ namespace egeria {
 
 constexpr int kMaxCtas = 160;  // sizing bound for the work split (a B200 has 148 SMs)
 constexpr int kMaxW = 2048;    // replay keeps 2 * W doubles in shared memory
+constexpr int kPlanSlots = 16; // device-side plans kept, keyed by (b, activation pointers)
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Offsets of everything the library keeps in the caller's workspace.
 struct Layout {
-    size_t status, tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides, rowloss, tickets, T,
-        raw, plist, n_evals, counter, freeze_eval, last_slope, losses, keep, slots, staging, total;
+    size_t status, rowloss, tickets, T, raw, plist, n_evals, counter, freeze_eval, last_slope, losses, keep,
+        slots, staging, total;
     size_t slot_bytes_cap;  // bytes reserved for partial slots
+    // Device-side plans (tensor maps, pointers, unit table, per-CTA ranges, slot ranges): kPlanSlots
+    // regions of plan_stride bytes from plan0; the offsets below are relative to a region.
+    size_t plan0, plan_stride;
+    size_t tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides;
 };
 
 static int64_t units_cap(int M, int b_max) {
@@ -46,12 +51,19 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
         return o;
     };
     L.status = take(256);
-    L.tmaps = take((size_t)2 * M * sizeof(CUtensorMap));
-    L.modules = take((size_t)M * sizeof(ModulePtrs));
-    L.units = take((size_t)units_cap(M, b_max) * sizeof(Unit));
-    L.cta_begin_tc = take((kMaxCtas + 1) * sizeof(int32_t));
-    L.cta_begin_simt = take((kMaxCtas + 1) * sizeof(int32_t));
-    L.sides = take((size_t)2 * M * sizeof(SideInfo));
+    {
+        size_t saved = off;
+        off = 0;
+        L.tmaps = take((size_t)2 * M * sizeof(CUtensorMap));
+        L.modules = take((size_t)M * sizeof(ModulePtrs));
+        L.units = take((size_t)units_cap(M, b_max) * sizeof(Unit));
+        L.cta_begin_tc = take((kMaxCtas + 1) * sizeof(int32_t));
+        L.cta_begin_simt = take((kMaxCtas + 1) * sizeof(int32_t));
+        L.sides = take((size_t)2 * M * sizeof(SideInfo));
+        L.plan_stride = off;
+        off = saved;
+        L.plan0 = take(L.plan_stride * kPlanSlots);
+    }
     L.rowloss = take((size_t)M * kMaxB * sizeof(double));
     L.tickets = take((size_t)M * sizeof(int32_t));
     L.T = take((size_t)M * sizeof(float));
@@ -113,10 +125,19 @@ struct egeria_ctx {
     int n_ctas = 0;
     EncodeTiledFn encode = nullptr;
     bool attrs_set = false;
-    // what the device-side plan currently describes
-    int plan_b = -1;
-    std::vector<const void *> plan_At, plan_Ar;
-    Plan plan;
+    // device-side plans, least recently used one is replaced
+    struct PlanEntry {
+        int b = -1;
+        std::vector<const void *> At, Ar;
+        Plan plan;
+        uint64_t last_use = 0;
+    };
+    PlanEntry plans[kPlanSlots];
+    int cur = 0;           // entry the last egeria_sp_loss_batch used
+    int plan_b = -1;       // its b
+    uint64_t use_clock = 0;
+    std::vector<uint8_t> pack;  // host image of one plan region
+    uint8_t *plan_region(int i) const { return ws + L.plan0 + (size_t)i * L.plan_stride; }
     cudaStream_t last_stream = nullptr;
     int64_t launches = 0;
     std::vector<void *> staging_t, staging_r;
@@ -285,13 +306,24 @@ static egeria_status encode_map(egeria_ctx *ctx, CUtensorMap *tm, const void *ba
     return r == CUDA_SUCCESS ? EGERIA_OK : EGERIA_ERR_CUDA;
 }
 
-// Bring the device-side plan (units, tensor maps, pointers) up to date with this call.
+// Select (or build and upload) the device-side plan for this (b, pointers).
 static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const void *const *At, const void *const *Ar,
                                   int b) {
     const int M = ctx->M;
-    bool same = (ctx->plan_b == b) && (int)ctx->plan_At.size() == M;
-    for (int m = 0; m < M && same; ++m) same = (ctx->plan_At[m] == At[m]) && (ctx->plan_Ar[m] == Ar[m]);
-    if (same) return EGERIA_OK;
+    const size_t pbytes = (size_t)M * sizeof(void *);
+    int lru = 0;
+    for (int i = 0; i < kPlanSlots; ++i) {
+        egeria_ctx::PlanEntry &e = ctx->plans[i];
+        if (e.b == b && memcmp(e.At.data(), At, pbytes) == 0 && memcmp(e.Ar.data(), Ar, pbytes) == 0) {
+            e.last_use = ++ctx->use_clock;
+            ctx->cur = i;
+            ctx->plan_b = b;
+            return EGERIA_OK;
+        }
+        if (e.last_use < ctx->plans[lru].last_use) lru = i;
+    }
+    egeria_ctx::PlanEntry &e = ctx->plans[lru];
+    e.b = -1;  // invalid until the upload below has been enqueued
 
     std::vector<uint8_t> tc_ok(M);
     for (int m = 0; m < M; ++m) {
@@ -299,15 +331,18 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
                              (reinterpret_cast<uintptr_t>(Ar[m]) % 16 == 0) && (ctx->d[m] % 8 == 0);
         tc_ok[m] = aligned && !(ctx->flags & EGERIA_FLAG_FORCE_SIMT);
     }
-    build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), ctx->plan);
-    const Plan &P = ctx->plan;
-    if ((size_t)P.units.size() * slot_floats_of_mode(P.mode) * sizeof(float) > ctx->L.slot_bytes_cap)
+    build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), e.plan);
+    const Plan &P = e.plan;
+    const Layout &L = ctx->L;
+    if ((size_t)P.units.size() * slot_floats_of_mode(P.mode) * sizeof(float) > L.slot_bytes_cap ||
+        L.units + P.units.size() * sizeof(Unit) > L.cta_begin_tc)
         return EGERIA_ERR_WORKSPACE;
 
+    ctx->pack.assign(L.plan_stride, 0);
+    uint8_t *img = ctx->pack.data();
     const int box_rows = (P.mode == kStacked) ? 64 : (P.mode == kSingle1 ? 128 : 256);
-    std::vector<CUtensorMap> maps(2 * (size_t)M);
-    std::vector<ModulePtrs> mods(M);
-    memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
+    CUtensorMap *maps = reinterpret_cast<CUtensorMap *>(img + L.tmaps);
+    ModulePtrs *mods = reinterpret_cast<ModulePtrs *>(img + L.modules);
     for (int m = 0; m < M; ++m) {
         mods[m] = ModulePtrs{At[m], Ar[m], ctx->d[m]};
         if (!tc_ok[m]) continue;
@@ -315,23 +350,18 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
         if (s == EGERIA_OK) s = encode_map(ctx, &maps[2 * m + 1], Ar[m], b, ctx->d[m], box_rows);
         if (s != EGERIA_OK) return s;
     }
-    const Layout &L = ctx->L;
-    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.tmaps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice,
-                            stream));
-    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.modules, mods.data(), mods.size() * sizeof(ModulePtrs),
-                            cudaMemcpyHostToDevice, stream));
-    if (!P.units.empty())
-        EG_CUDA(cudaMemcpyAsync(ctx->ws + L.units, P.units.data(), P.units.size() * sizeof(Unit),
-                                cudaMemcpyHostToDevice, stream));
-    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t),
-                            cudaMemcpyHostToDevice, stream));
-    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.cta_begin_simt, P.cta_begin_simt.data(),
-                            P.cta_begin_simt.size() * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
-    EG_CUDA(cudaMemcpyAsync(ctx->ws + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo),
-                            cudaMemcpyHostToDevice, stream));
+    if (!P.units.empty()) memcpy(img + L.units, P.units.data(), P.units.size() * sizeof(Unit));
+    memcpy(img + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t));
+    memcpy(img + L.cta_begin_simt, P.cta_begin_simt.data(), P.cta_begin_simt.size() * sizeof(int32_t));
+    memcpy(img + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo));
+    // One copy from pageable memory: the runtime stages it before returning, so `pack` may be reused.
+    EG_CUDA(cudaMemcpyAsync(ctx->plan_region(lru), img, L.plan_stride, cudaMemcpyHostToDevice, stream));
+    e.b = b;
+    e.At.assign(At, At + M);
+    e.Ar.assign(Ar, Ar + M);
+    e.last_use = ++ctx->use_clock;
+    ctx->cur = lru;
     ctx->plan_b = b;
-    ctx->plan_At.assign(At, At + M);
-    ctx->plan_Ar.assign(Ar, Ar + M);
     return EGERIA_OK;
 }
 
@@ -374,7 +404,8 @@ egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const voi
     if (s != EGERIA_OK) return s;
 
     const Layout &L = ctx->L;
-    const Plan &P = ctx->plan;
+    const Plan &P = ctx->plans[ctx->cur].plan;
+    const uint8_t *region = ctx->plan_region(ctx->cur);
     const int64_t slot_floats = slot_floats_of_mode(P.mode);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     if (ctx->flags & EGERIA_FLAG_TIME_GRAM) {
@@ -392,9 +423,9 @@ egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const voi
     }
     if (P.n_units_tc > 0) {
         TcParams tp;
-        tp.tmaps = ctx->at<CUtensorMap>(L.tmaps);
-        tp.units = ctx->at<Unit>(L.units);
-        tp.cta_begin = ctx->at<int32_t>(L.cta_begin_tc);
+        tp.tmaps = reinterpret_cast<const CUtensorMap *>(region + L.tmaps);
+        tp.units = reinterpret_cast<const Unit *>(region + L.units);
+        tp.cta_begin = reinterpret_cast<const int32_t *>(region + L.cta_begin_tc);
         tp.slots = ctx->at<float>(L.slots);
         tp.slot_floats = slot_floats;
         tp.b = b;
@@ -407,9 +438,9 @@ egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const voi
     }
     if ((int)P.units.size() > P.n_units_tc) {
         SimtParams sp;
-        sp.modules = ctx->at<ModulePtrs>(L.modules);
-        sp.units = ctx->at<Unit>(L.units) + P.n_units_tc;
-        sp.cta_begin = ctx->at<int32_t>(L.cta_begin_simt);
+        sp.modules = reinterpret_cast<const ModulePtrs *>(region + L.modules);
+        sp.units = reinterpret_cast<const Unit *>(region + L.units) + P.n_units_tc;
+        sp.cta_begin = reinterpret_cast<const int32_t *>(region + L.cta_begin_simt);
         sp.slots = ctx->at<float>(L.slots);
         sp.slot_floats = slot_floats;
         sp.b = b;
@@ -422,7 +453,7 @@ egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const voi
     FinParams fp;
     fp.slots = ctx->at<float>(L.slots);
     fp.slot_floats = slot_floats;
-    fp.sides = ctx->at<SideInfo>(L.sides);
+    fp.sides = reinterpret_cast<const SideInfo *>(region + L.sides);
     fp.b = b;
     fp.out_losses = out_losses;
     fp.rowloss = ctx->at<double>(L.rowloss);
