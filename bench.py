@@ -146,6 +146,22 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- multi-rank helpers
+
+def max_over_ranks(x: float, dist, device) -> float:
+    """The slowest rank's figure (every multi-GPU time is the max over ranks)."""
+    if dist is None:
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, modules: int, steps: int, seconds: float) -> float:
+    """module-evals/s of the whole job: every rank evaluates its own replica of all modules."""
+    return world * modules * steps / seconds
+
+
 # ----------------------------------------------------------------------------- our arm
 
 def pick_workload(args) -> wl.Workload:
@@ -264,11 +280,8 @@ def run_ours(args):
     gram_ms, gram_calls = ctx.egeria_gram_kernel_time()
     launches = ctx.egeria_launch_count() - l0
     ctx.check_device_status()
-    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    elapsed_ms = float(t.item())
-    value = world * w.M * args.steps / (elapsed_ms * 1e-3)
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, device)
+    value = whole_job_value(world, w.M, args.steps, elapsed_ms * 1e-3)
 
     # ---- end to end through the host entry point (pinned host buffers, copies inside the timed region)
     e2e = None
@@ -298,10 +311,8 @@ def run_ours(args):
             e2e_step()
         barrier()
         dt = time.perf_counter() - t0
-        tt = torch.tensor([dt], dtype=torch.float64, device=device)
-        if dist is not None:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * w.M * e2e_steps / float(tt.item()), "unit": UNIT,
+        dt = max_over_ranks(dt, dist, device)
+        e2e = {"value": whole_job_value(world, w.M, e2e_steps, dt), "unit": UNIT,
                "h2d_bytes_per_step": w.input_bytes + 4 * w.M, "d2h_bytes_per_step": 4 * w.M + w.M,
                "steps": e2e_steps}
         ctx_h.close()
