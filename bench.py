@@ -3,8 +3,9 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-A step is one pass of the whole path over one synthetic mini-batch: egeria_sp_loss_batch
-(Gram + finalisation kernels) followed by egeria_plasticity_step.  Prints ONE JSON line.
+A step is one pass of the whole path over one synthetic mini-batch: egeria_plasticity_evaluate
+(Gram kernel, then the finalisation kernel that also advances the freezing rule).  Prints ONE
+JSON line.
 With N > 1 (torchrun) every rank evaluates its own replica of the workload on its own
 GPU; there is no data-path collective.
 """
@@ -220,10 +221,11 @@ def time_workload(eg, w, device, steps, warmup, n_sets, stream, time_gram=True):
     ptrs = [(ctx._ptr_array(at, w.b, True), ctx._ptr_array(ar, w.b, True)) for at, ar in sets]
     sp = int(stream.cuda_stream)
 
+    lp, slp, mp = losses.data_ptr(), slopes.data_ptr(), mask.data_ptr()
+
     def step(i):
         pa, pr = ptrs[i % n_sets]
-        ctx.sp_loss_batch_raw(pa, pr, w.b, losses.data_ptr(), sp)
-        ctx.egeria_plasticity_step(losses, slopes, mask, stream)
+        ctx.plasticity_evaluate_raw(pa, pr, w.b, lp, slp, mp, sp)   # SP loss of all modules + freezing rule
 
     for i in range(warmup):
         step(i)

@@ -128,6 +128,17 @@ egeria_status egeria_sp_loss_batch_host(egeria_ctx *ctx, void *cuda_stream,
 egeria_status egeria_plasticity_step(egeria_ctx *ctx, void *cuda_stream, const float *losses,
                                      double *out_slopes, uint8_t *out_mask);
 
+/* One whole evaluation in one call: egeria_sp_loss_batch followed by
+ * egeria_plasticity_step on the losses just computed [Algorithm 1,
+ * checkPlasticity: calculateSPLoss, smoothPlasticity, windowLinearFit, counter].
+ * The freezing rule of a module is advanced by the thread block that finishes
+ * the module's loss, so no extra kernel is launched.  Arguments as in the two
+ * calls; out_slopes and out_mask may be NULL.  Results are identical to the two
+ * separate calls. */
+egeria_status egeria_plasticity_evaluate(egeria_ctx *ctx, void *cuda_stream, const void *const *At,
+                                         const void *const *Ar, int b, const int64_t *d,
+                                         float *out_losses, double *out_slopes, uint8_t *out_mask);
+
 /* The same rule over whole histories, from a cleared state that is private to
  * the call (the context's step state is not touched).
  *   hist             device float [M, H] row-major raw readings

@@ -26,7 +26,7 @@ EXPORTS = [
     "egeria_sp_loss_batch", "egeria_sp_loss_batch_host", "egeria_plasticity_step",
     "egeria_plasticity_replay", "egeria_plasticity_reset", "egeria_plasticity_window",
     "egeria_debug_dump_gram", "egeria_debug_plan", "egeria_device_status", "egeria_launch_count",
-    "egeria_gram_kernel_time", "egeria_sp_loss_static",
+    "egeria_gram_kernel_time", "egeria_sp_loss_static", "egeria_plasticity_evaluate",
     "egeria_status_string",
 ]
 
@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
     L.egeria_sp_loss_batch.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, i64p, vp]
     L.egeria_sp_loss_batch_host.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, i64p, vp]
     L.egeria_plasticity_step.argtypes = [vp, vp, vp, vp, vp]
+    L.egeria_plasticity_evaluate.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, i64p,
+                                             vp, vp, vp]
     L.egeria_plasticity_replay.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp]
     L.egeria_plasticity_reset.argtypes = [vp, vp, ctypes.c_int]
     L.egeria_plasticity_window.argtypes = [vp]
@@ -197,6 +199,25 @@ class Context:
                                         out_losses.data_ptr())
         _check(st, "egeria_sp_loss_batch")
         return out_losses
+
+    def egeria_plasticity_evaluate(self, At: Sequence[torch.Tensor], Ar: Sequence[torch.Tensor],
+                                   stream: Optional[torch.cuda.Stream] = None):
+        """Losses, slopes and freeze mask of one evaluation (SP loss + freezing rule)."""
+        b = int(At[0].shape[0])
+        losses = torch.empty(self.M, dtype=torch.float32, device=self.device)
+        slopes = torch.empty(self.M, dtype=torch.float64, device=self.device)
+        mask = torch.empty(self.M, dtype=torch.uint8, device=self.device)
+        pa, pr = self._ptr_array(At, b, True), self._ptr_array(Ar, b, True)
+        st = lib().egeria_plasticity_evaluate(self._h, _stream_ptr(stream), pa, pr, b, self._d_arr,
+                                              losses.data_ptr(), slopes.data_ptr(), mask.data_ptr())
+        _check(st, "egeria_plasticity_evaluate")
+        return losses, slopes, mask
+
+    def plasticity_evaluate_raw(self, pa, pr, b: int, losses_ptr: int, slopes_ptr: int, mask_ptr: int,
+                                stream_ptr: int) -> None:
+        """Same call with ready-made pointer arrays (benchmark loops)."""
+        _check(lib().egeria_plasticity_evaluate(self._h, stream_ptr, pa, pr, b, self._d_arr, losses_ptr,
+                                                slopes_ptr, mask_ptr), "egeria_plasticity_evaluate")
 
     def sp_loss_batch_raw(self, pa, pr, b: int, out_ptr: int, stream_ptr: int) -> None:
         """Same call with ready-made pointer arrays (benchmark loops)."""

@@ -365,6 +365,17 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
     return EGERIA_OK;
 }
 
+static cudaError_t launch_finalize(const FinParams &fp, int M, int b, cudaStream_t stream) {
+    const dim3 grid(M, (b + kFinRowsPerCta - 1) / kFinRowsPerCta);
+    if (b <= 64)
+        finalize_kernel<2><<<grid, kFinThreads, 0, stream>>>(fp);
+    else if (b <= 128)
+        finalize_kernel<4><<<grid, kFinThreads, 0, stream>>>(fp);
+    else
+        finalize_kernel<8><<<grid, kFinThreads, 0, stream>>>(fp);
+    return cudaGetLastError();
+}
+
 template <int MODE>
 static cudaError_t launch_tc(egeria_ctx *ctx, cudaStream_t stream, const TcParams &tp) {
     gram_tc_kernel<MODE><<<ctx->n_ctas, kTcThreads, TcCfg<MODE>::kSmemBytes, stream>>>(tp);
@@ -385,10 +396,9 @@ static egeria_status set_attrs(egeria_ctx *ctx) {
 
 }  // namespace egeria
 
-extern "C" {
-
-egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const void *const *At, const void *const *Ar,
-                                   int b, const int64_t *d, float *out_losses) {
+static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void *const *At, const void *const *Ar,
+                                  int b, const int64_t *d, float *out_losses, bool fuse_step, double *out_slopes,
+                                  uint8_t *out_mask) {
     if (!ctx || !At || !Ar || !d || !out_losses) return EGERIA_ERR_INVALID_ARG;
     if (b < 2 || b > ctx->b_max) return EGERIA_ERR_INVALID_ARG;
     for (int m = 0; m < ctx->M; ++m) {
@@ -459,11 +469,28 @@ egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const voi
     fp.rowloss = ctx->at<double>(L.rowloss);
     fp.tickets = ctx->at<int32_t>(L.tickets);
     fp.keep = (ctx->flags & EGERIA_FLAG_KEEP_GRAMS) ? ctx->at<float>(L.keep) : nullptr;
-    dim3 grid(ctx->M, (b + kFinRowsPerCta - 1) / kFinRowsPerCta);
-    finalize_kernel<<<grid, kFinThreads, 0, stream>>>(fp);
-    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    fp.fuse_step = fuse_step ? 1 : 0;
+    fp.W = ctx->W;
+    fp.signed_test = (ctx->flags & EGERIA_FLAG_SIGNED_SLOPE) ? 1 : 0;
+    fp.st = ctx->slope_state();
+    fp.out_slopes = out_slopes;
+    fp.out_mask = out_mask;
+    if (launch_finalize(fp, ctx->M, b, stream) != cudaSuccess) return EGERIA_ERR_CUDA;
     ctx->launches++;
     return EGERIA_OK;
+}
+
+extern "C" {
+
+egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const void *const *At, const void *const *Ar,
+                                   int b, const int64_t *d, float *out_losses) {
+    return sp_loss_impl(ctx, cuda_stream, At, Ar, b, d, out_losses, false, nullptr, nullptr);
+}
+
+egeria_status egeria_plasticity_evaluate(egeria_ctx *ctx, void *cuda_stream, const void *const *At,
+                                         const void *const *Ar, int b, const int64_t *d, float *out_losses,
+                                         double *out_slopes, uint8_t *out_mask) {
+    return sp_loss_impl(ctx, cuda_stream, At, Ar, b, d, out_losses, true, out_slopes, out_mask);
 }
 
 egeria_status egeria_sp_loss_batch_host(egeria_ctx *ctx, void *cuda_stream, const void *const *At_host,
@@ -738,7 +765,12 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     fp.rowloss = reinterpret_cast<double *>(ws + L.rowloss);
     fp.tickets = ticket;
     fp.keep = nullptr;
-    finalize_kernel<<<dim3(1, (b + kFinRowsPerCta - 1) / kFinRowsPerCta), kFinThreads, 0, stream>>>(fp);
-    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    fp.fuse_step = 0;
+    fp.W = 0;
+    fp.signed_test = 0;
+    fp.st = SlopeState{};
+    fp.out_slopes = nullptr;
+    fp.out_mask = nullptr;
+    if (launch_finalize(fp, 1, b, stream) != cudaSuccess) return EGERIA_ERR_CUDA;
     return EGERIA_OK;
 }

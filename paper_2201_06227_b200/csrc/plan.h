@@ -81,8 +81,12 @@ struct Tile {
     int64_t nkb;
 };
 
-// Cut the concatenated block sequence of `tiles` into n_ctas near-equal contiguous ranges;
-// every (tile, range) intersection becomes a unit.
+// Cut the concatenated block sequence of `tiles` into near-equal contiguous ranges, one per
+// CTA; every (tile, range) intersection becomes a unit.  Small problems use fewer CTAs, so
+// that a range has at least kMinBlocksPerCta blocks: a shorter range costs the same latency
+// and only adds partial slots for the finaliser to read.
+constexpr int kMinBlocksPerCta = 8;
+
 inline void split_tiles(const std::vector<Tile> &tiles, int n_ctas, int slot0, std::vector<Unit> &units,
                         std::vector<int32_t> &cta_begin) {
     int64_t total = 0;
@@ -91,9 +95,13 @@ inline void split_tiles(const std::vector<Tile> &tiles, int n_ctas, int slot0, s
     const int base = (int)units.size();
     size_t ti = 0;
     int64_t tile_start = 0;  // global block index of tiles[ti]'s first block
+    int64_t used = (total + kMinBlocksPerCta - 1) / kMinBlocksPerCta;
+    if (used > n_ctas) used = n_ctas;
+    if (used < 1) used = 1;
     for (int c = 0; c < n_ctas; ++c) {
         cta_begin[c] = (int)units.size() - base;
-        const int64_t lo = total * c / n_ctas, hi = total * (c + 1) / n_ctas;
+        if (c >= used) continue;  // idle CTA: empty range
+        const int64_t lo = total * c / used, hi = total * (c + 1) / used;
         int64_t pos = lo;
         while (pos < hi) {
             while (ti < tiles.size() && tile_start + tiles[ti].nkb <= pos) {

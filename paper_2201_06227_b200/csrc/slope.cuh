@@ -68,18 +68,17 @@ __device__ __forceinline__ double plasticity_advance(double *raw, double *plist,
     return slope;
 }
 
-// One new reading per module.  grid = M warps (one 32-thread block each).
-__global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int M, int W, int signed_test,
-                                                             const float *losses, double *out_slopes,
-                                                             uint8_t *out_mask) {
-    const int m = blockIdx.x, lane = threadIdx.x;
-    if (m >= M) return;
+// One new reading for module m, by one warp: Algorithm 1 on the context's state.
+__device__ __forceinline__ void plasticity_step_module(const SlopeState &st, int m, int W, int signed_test,
+                                                       float reading, double *out_slopes, uint8_t *out_mask,
+                                                       int lane) {
     int n_evals = st.n_evals[m], counter = st.counter[m], freeze_eval = st.freeze_eval[m];
     double slope = st.last_slope[m];
+    __syncwarp();
     if (counter < W) {
         slope = plasticity_advance(st.raw + (int64_t)m * st.W_cap, st.plist + (int64_t)m * st.W_cap, n_evals,
-                                   counter, freeze_eval, (double)losses[m], W, (double)st.T[m],
-                                   signed_test != 0, lane);
+                                   counter, freeze_eval, (double)reading, W, (double)st.T[m], signed_test != 0,
+                                   lane);
         if (lane == 0) {
             st.n_evals[m] = n_evals;
             st.counter[m] = counter;
@@ -91,6 +90,15 @@ __global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int 
         if (out_slopes) out_slopes[m] = slope;
         if (out_mask) out_mask[m] = (counter >= W) ? 1 : 0;
     }
+}
+
+// One new reading per module.  grid = M warps (one 32-thread block each).
+__global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int M, int W, int signed_test,
+                                                             const float *losses, double *out_slopes,
+                                                             uint8_t *out_mask) {
+    const int m = blockIdx.x, lane = threadIdx.x;
+    if (m >= M) return;
+    plasticity_step_module(st, m, W, signed_test, losses[m], out_slopes, out_mask, lane);
 }
 
 // Whole histories from a cleared private state (rings in shared memory: 2 * W doubles).

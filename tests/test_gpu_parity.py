@@ -327,6 +327,30 @@ def test_step_matches_replay_and_oracle(signed):
     ctx.close()
 
 
+def test_evaluate_equals_separate_calls():
+    """egeria_plasticity_evaluate = egeria_sp_loss_batch + egeria_plasticity_step, bit for bit."""
+    ds, b, W, T = [4096, 520, 1001, 8192], 72, 3, float(np.float32(5e-4))
+    fused = eg.Context(ds, b, W, T, device=DEV)
+    split = eg.Context(ds, b, W, T, device=DEV)
+    for k in range(8):
+        at, ar = [], []
+        for m, d in enumerate(ds):
+            t, r = wl.make_pair(b, d, "relu", 0.3 / (1 + k), seed=500 + 10 * k + m, device=DEV)
+            at.append(t)
+            ar.append(r)
+        l1, s1, m1 = fused.egeria_plasticity_evaluate(at, ar)
+        l2 = split.egeria_sp_loss_batch(at, ar)
+        s2, m2 = split.egeria_plasticity_step(l2)
+        assert l1.cpu().numpy().tobytes() == l2.cpu().numpy().tobytes()
+        assert s1.cpu().numpy().tobytes() == s2.cpu().numpy().tobytes()
+        assert m1.cpu().numpy().tobytes() == m2.cpu().numpy().tobytes()
+    ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+    assert_loss_close(l1.cpu().numpy(), ref)
+    fused.check_device_status()
+    fused.close()
+    split.close()
+
+
 def test_alg1_hand_traces_on_gpu():
     from fractions import Fraction
     for line in (GOLDEN / "alg1_traces.txt").read_text().splitlines():
