@@ -25,7 +25,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Offsets of everything the library keeps in the caller's workspace.
 struct Layout {
-    size_t status, rowloss, tickets, T, raw, plist, n_evals, counter, freeze_eval, last_slope, losses, keep,
+    size_t status, rowloss, tickets, fin_ctr, T, raw, plist, n_evals, counter, freeze_eval, last_slope, losses, keep,
         slots, staging, total;
     size_t slot_bytes_cap;  // bytes reserved for partial slots
     // Device-side plans (tensor maps, pointers, unit table, per-CTA ranges, slot ranges): kPlanSlots
@@ -66,6 +66,7 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
     }
     L.rowloss = take((size_t)M * kMaxB * sizeof(double));
     L.tickets = take((size_t)M * sizeof(int32_t));
+    L.fin_ctr = take((size_t)2 * M * sizeof(FinCounters));  // two sets, used by alternate launches
     L.T = take((size_t)M * sizeof(float));
     L.raw = take((size_t)M * W * sizeof(double));
     L.plist = take((size_t)M * W * sizeof(double));
@@ -140,6 +141,7 @@ struct egeria_ctx {
     uint8_t *plan_region(int i) const { return ws + L.plan0 + (size_t)i * L.plan_stride; }
     cudaStream_t last_stream = nullptr;
     int64_t launches = 0;
+    uint32_t tc_launches = 0;  // selects the set of progress counters the next tensor-core launch uses
     std::vector<void *> staging_t, staging_r;
     // EGERIA_FLAG_TIME_GRAM: event pairs around the Gram kernel launches since the last query
     std::vector<cudaEvent_t> ev_pool;
@@ -267,6 +269,7 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     for (int m = 0; m < M; ++m) Th[m] = T ? T[m] : T_all;
     cudaError_t e = cudaMemset(ctx->ws + L.status, 0, 256);
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.tickets, 0, (size_t)M * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.fin_ctr, 0, (size_t)2 * M * sizeof(FinCounters));
     if (e == cudaSuccess) e = cudaMemcpy(ctx->ws + L.T, Th.data(), (size_t)M * sizeof(float), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) {
         plasticity_clear_kernel<<<(M + 127) / 128, 128>>>(ctx->slope_state(), M);
@@ -340,7 +343,7 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
 
     ctx->pack.assign(L.plan_stride, 0);
     uint8_t *img = ctx->pack.data();
-    const int box_rows = (P.mode == kStacked) ? 64 : (P.mode == kSingle1 ? 128 : 256);
+    const int box_rows = pitch_of_mode(P.mode);  // rows of one TMA box: all rows of one side
     CUtensorMap *maps = reinterpret_cast<CUtensorMap *>(img + L.tmaps);
     ModulePtrs *mods = reinterpret_cast<ModulePtrs *>(img + L.modules);
     for (int m = 0; m < M; ++m) {
@@ -367,29 +370,51 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
 
 static cudaError_t launch_finalize(const FinParams &fp, int M, int b, cudaStream_t stream) {
     const dim3 grid(M, (b + kFinRowsPerCta - 1) / kFinRowsPerCta);
-    if (b <= 64)
-        finalize_kernel<2><<<grid, kFinThreads, 0, stream>>>(fp);
-    else if (b <= 128)
-        finalize_kernel<4><<<grid, kFinThreads, 0, stream>>>(fp);
-    else
-        finalize_kernel<8><<<grid, kFinThreads, 0, stream>>>(fp);
+    switch (fin_nc_of_b(b)) {
+        case 1: finalize_kernel<1><<<grid, kFinThreads, 0, stream>>>(fp); break;
+        case 2: finalize_kernel<2><<<grid, kFinThreads, 0, stream>>>(fp); break;
+        case 4: finalize_kernel<4><<<grid, kFinThreads, 0, stream>>>(fp); break;
+        default: finalize_kernel<8><<<grid, kFinThreads, 0, stream>>>(fp); break;
+    }
     return cudaGetLastError();
 }
 
-template <int MODE>
-static cudaError_t launch_tc(egeria_ctx *ctx, cudaStream_t stream, const TcParams &tp) {
-    gram_tc_kernel<MODE><<<ctx->n_ctas, kTcThreads, TcCfg<MODE>::kSmemBytes, stream>>>(tp);
+static cudaError_t launch_tc_mode(int mode, int n_ctas, cudaStream_t stream, const TcParams &tp) {
+    switch (mode) {
+        case kStacked32:
+            gram_tc_kernel<kStacked32><<<n_ctas, kTcThreads, TcCfg<kStacked32>::kSmemBytes, stream>>>(tp);
+            break;
+        case kStacked64:
+            gram_tc_kernel<kStacked64><<<n_ctas, kTcThreads, TcCfg<kStacked64>::kSmemBytes, stream>>>(tp);
+            break;
+        case kSingle1:
+            gram_tc_kernel<kSingle1><<<n_ctas, kTcThreads, TcCfg<kSingle1>::kSmemBytes, stream>>>(tp);
+            break;
+        default:
+            gram_tc_kernel<kSingle2><<<n_ctas, kTcThreads, TcCfg<kSingle2>::kSmemBytes, stream>>>(tp);
+            break;
+    }
     return cudaGetLastError();
+}
+
+static cudaError_t set_tc_attrs() {
+    cudaError_t e = cudaFuncSetAttribute(gram_tc_kernel<kStacked32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         TcCfg<kStacked32>::kSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gram_tc_kernel<kStacked64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcCfg<kStacked64>::kSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gram_tc_kernel<kSingle1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcCfg<kSingle1>::kSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gram_tc_kernel<kSingle2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcCfg<kSingle2>::kSmemBytes);
+    return e;
 }
 
 static egeria_status set_attrs(egeria_ctx *ctx) {
     if (ctx->attrs_set) return EGERIA_OK;
-    EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kStacked>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TcCfg<kStacked>::kSmemBytes));
-    EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kSingle1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TcCfg<kSingle1>::kSmemBytes));
-    EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kSingle2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TcCfg<kSingle2>::kSmemBytes));
+    EG_CUDA(set_tc_attrs());
     ctx->attrs_set = true;
     return EGERIA_OK;
 }
@@ -431,22 +456,39 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         ctx->ev_used += 2;
         EG_CUDA(cudaEventRecord(ev0, stream));
     }
+    FinCommon fc;
+    fc.slots = ctx->at<float>(L.slots);
+    fc.slot_floats = slot_floats;
+    fc.sides = reinterpret_cast<const SideInfo *>(region + L.sides);
+    fc.b = b;
+    fc.out_losses = out_losses;
+    fc.rowloss = ctx->at<double>(L.rowloss);
+    fc.keep = (ctx->flags & EGERIA_FLAG_KEEP_GRAMS) ? ctx->at<float>(L.keep) : nullptr;
+    fc.fuse_step = fuse_step ? 1 : 0;
+    fc.W = ctx->W;
+    fc.signed_test = (ctx->flags & EGERIA_FLAG_SIGNED_SLOPE) ? 1 : 0;
+    fc.st = ctx->slope_state();
+    fc.out_slopes = out_slopes;
+    fc.out_mask = out_mask;
     if (P.n_units_tc > 0) {
         TcParams tp;
         tp.tmaps = reinterpret_cast<const CUtensorMap *>(region + L.tmaps);
         tp.units = reinterpret_cast<const Unit *>(region + L.units);
         tp.cta_begin = reinterpret_cast<const int32_t *>(region + L.cta_begin_tc);
         tp.slots = ctx->at<float>(L.slots);
-        tp.slot_floats = slot_floats;
-        tp.b = b;
         tp.status = ctx->at<int32_t>(L.status);
-        cudaError_t e = (P.mode == kStacked)   ? launch_tc<kStacked>(ctx, stream, tp)
-                        : (P.mode == kSingle1) ? launch_tc<kSingle1>(ctx, stream, tp)
-                                               : launch_tc<kSingle2>(ctx, stream, tp);
-        if (e != cudaSuccess) return EGERIA_ERR_CUDA;
+        FinCounters *sets = ctx->at<FinCounters>(L.fin_ctr);
+        const uint32_t set = ctx->tc_launches & 1u;
+        tp.ctr = sets + (size_t)set * ctx->M;
+        tp.ctr_next = sets + (size_t)(set ^ 1u) * ctx->M;
+        tp.M = ctx->M;
+        tp.fin = fc;
+        if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
+        ctx->tc_launches++;
         ctx->launches++;
     }
-    if ((int)P.units.size() > P.n_units_tc) {
+    const bool any_simt = (int)P.units.size() > P.n_units_tc;
+    if (any_simt) {
         SimtParams sp;
         sp.modules = reinterpret_cast<const ModulePtrs *>(region + L.modules);
         sp.units = reinterpret_cast<const Unit *>(region + L.units) + P.n_units_tc;
@@ -460,23 +502,14 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         ctx->launches++;
     }
     if (ev1) EG_CUDA(cudaEventRecord(ev1, stream));
-    FinParams fp;
-    fp.slots = ctx->at<float>(L.slots);
-    fp.slot_floats = slot_floats;
-    fp.sides = reinterpret_cast<const SideInfo *>(region + L.sides);
-    fp.b = b;
-    fp.out_losses = out_losses;
-    fp.rowloss = ctx->at<double>(L.rowloss);
-    fp.tickets = ctx->at<int32_t>(L.tickets);
-    fp.keep = (ctx->flags & EGERIA_FLAG_KEEP_GRAMS) ? ctx->at<float>(L.keep) : nullptr;
-    fp.fuse_step = fuse_step ? 1 : 0;
-    fp.W = ctx->W;
-    fp.signed_test = (ctx->flags & EGERIA_FLAG_SIGNED_SLOPE) ? 1 : 0;
-    fp.st = ctx->slope_state();
-    fp.out_slopes = out_slopes;
-    fp.out_mask = out_mask;
-    if (launch_finalize(fp, ctx->M, b, stream) != cudaSuccess) return EGERIA_ERR_CUDA;
-    ctx->launches++;
+    if (any_simt) {
+        // the CUDA-core modules are finished by a kernel of their own
+        FinParams fp;
+        fp.c = fc;
+        fp.tickets = ctx->at<int32_t>(L.tickets);
+        if (launch_finalize(fp, ctx->M, b, stream) != cudaSuccess) return EGERIA_ERR_CUDA;
+        ctx->launches++;
+    }
     return EGERIA_OK;
 }
 
@@ -591,6 +624,12 @@ egeria_status egeria_device_status(egeria_ctx *ctx) {
     EG_CUDA(cudaStreamSynchronize(ctx->last_stream));
     int32_t word = 0;
     EG_CUDA(cudaMemcpy(&word, ctx->ws + ctx->L.status, sizeof(word), cudaMemcpyDeviceToHost));
+    if (word != 0) {
+        // a kernel that gave up leaves its progress counters and tickets half-way: start afresh
+        EG_CUDA(cudaMemset(ctx->ws + ctx->L.fin_ctr, 0, (size_t)2 * ctx->M * sizeof(FinCounters)));
+        EG_CUDA(cudaMemset(ctx->ws + ctx->L.tickets, 0, (size_t)ctx->M * sizeof(int32_t)));
+        EG_CUDA(cudaMemset(ctx->ws + ctx->L.status, 0, sizeof(int32_t)));
+    }
     if (word == kStatusTimeout) return EGERIA_ERR_TIMEOUT;
     return word == 0 ? EGERIA_OK : EGERIA_ERR_CUDA;
 }
@@ -632,7 +671,8 @@ static StaticLayout static_layout() {
     L.cta_begin_simt = take((kStaticCtas + 1) * sizeof(int32_t));
     L.sides = take(2 * sizeof(SideInfo));
     L.rowloss = take(kMaxB * sizeof(double));
-    L.ticket = take(2 * sizeof(int32_t));  // [0] finalisation ticket, [1] status word
+    L.ticket = take(2 * sizeof(int32_t) + 2 * sizeof(FinCounters));  // [0] finalisation ticket, [1] status word,
+                                                                     // then two sets of progress counters
     L.slots = take((size_t)max_units(1, kSingle1, kStaticCtas) * slot_floats_of_mode(kSingle1) * sizeof(float));
     L.total = off;
     return L;
@@ -661,10 +701,7 @@ static egeria_status static_setup(int dev, StaticDevice **out) {
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
             qres != cudaDriverEntryPointSuccess || !fn)
             return EGERIA_ERR_CUDA;
-        EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kStacked>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     TcCfg<kStacked>::kSmemBytes));
-        EG_CUDA(cudaFuncSetAttribute(gram_tc_kernel<kSingle1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     TcCfg<kSingle1>::kSmemBytes));
+        EG_CUDA(set_tc_attrs());
         sd.encode = reinterpret_cast<EncodeTiledFn>(fn);
         sd.scratch = static_cast<unsigned char *>(ptr);
     }
@@ -701,7 +738,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     CUtensorMap maps[2];
     memset(maps, 0, sizeof(maps));
     if (tc_ok) {
-        const int box_rows = (P.mode == kStacked) ? 64 : 128;
+        const int box_rows = pitch_of_mode(P.mode);
         const void *bases[2] = {At, Ar};
         for (int side = 0; side < 2; ++side) {
             cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)b};
@@ -715,9 +752,9 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         }
     }
     const ModulePtrs mod{At, Ar, d};
-    // The array keeps whatever the previous call left: the ticket and the status word must
-    // start at zero; everything else is overwritten before it is read.
-    EG_CUDA(cudaMemsetAsync(ws + L.ticket, 0, 2 * sizeof(int32_t), stream));
+    // The array keeps whatever the previous call left: the ticket, the status word and the
+    // progress counters must start at zero; everything else is overwritten before it is read.
+    EG_CUDA(cudaMemsetAsync(ws + L.ticket, 0, 2 * sizeof(int32_t) + 2 * sizeof(FinCounters), stream));
     EG_CUDA(cudaMemcpyAsync(ws + L.tmaps, maps, sizeof(maps), cudaMemcpyHostToDevice, stream));
     EG_CUDA(cudaMemcpyAsync(ws + L.modules, &mod, sizeof(mod), cudaMemcpyHostToDevice, stream));
     EG_CUDA(cudaMemcpyAsync(ws + L.units, P.units.data(), P.units.size() * sizeof(Unit), cudaMemcpyHostToDevice,
@@ -731,19 +768,32 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
 
     const int64_t slot_floats = slot_floats_of_mode(P.mode);
     int32_t *ticket = reinterpret_cast<int32_t *>(ws + L.ticket);
+    FinCommon fc;
+    fc.slots = reinterpret_cast<const float *>(ws + L.slots);
+    fc.slot_floats = slot_floats;
+    fc.sides = reinterpret_cast<const SideInfo *>(ws + L.sides);
+    fc.b = b;
+    fc.out_losses = out_loss;
+    fc.rowloss = reinterpret_cast<double *>(ws + L.rowloss);
+    fc.keep = nullptr;
+    fc.fuse_step = 0;
+    fc.W = 0;
+    fc.signed_test = 0;
+    fc.st = SlopeState{};
+    fc.out_slopes = nullptr;
+    fc.out_mask = nullptr;
     if (P.n_units_tc > 0) {
         TcParams tp;
         tp.tmaps = reinterpret_cast<const CUtensorMap *>(ws + L.tmaps);
         tp.units = reinterpret_cast<const Unit *>(ws + L.units);
         tp.cta_begin = reinterpret_cast<const int32_t *>(ws + L.cta_begin_tc);
         tp.slots = reinterpret_cast<float *>(ws + L.slots);
-        tp.slot_floats = slot_floats;
-        tp.b = b;
         tp.status = ticket + 1;
-        if (P.mode == kStacked)
-            gram_tc_kernel<kStacked><<<kStaticCtas, kTcThreads, TcCfg<kStacked>::kSmemBytes, stream>>>(tp);
-        else
-            gram_tc_kernel<kSingle1><<<kStaticCtas, kTcThreads, TcCfg<kSingle1>::kSmemBytes, stream>>>(tp);
+        tp.ctr = reinterpret_cast<FinCounters *>(ticket + 2);
+        tp.ctr_next = tp.ctr + 1;
+        tp.M = 1;
+        tp.fin = fc;
+        if (launch_tc_mode(P.mode, kStaticCtas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
     } else {
         SimtParams sp;
         sp.modules = reinterpret_cast<const ModulePtrs *>(ws + L.modules);
@@ -754,23 +804,11 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         sp.b = b;
         sp.mode = P.mode;
         gram_simt_kernel<<<kStaticCtas, kSimtThreads, 0, stream>>>(sp);
+        if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+        FinParams fp;
+        fp.c = fc;
+        fp.tickets = ticket;
+        if (launch_finalize(fp, 1, b, stream) != cudaSuccess) return EGERIA_ERR_CUDA;
     }
-    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
-    FinParams fp;
-    fp.slots = reinterpret_cast<const float *>(ws + L.slots);
-    fp.slot_floats = slot_floats;
-    fp.sides = reinterpret_cast<const SideInfo *>(ws + L.sides);
-    fp.b = b;
-    fp.out_losses = out_loss;
-    fp.rowloss = reinterpret_cast<double *>(ws + L.rowloss);
-    fp.tickets = ticket;
-    fp.keep = nullptr;
-    fp.fuse_step = 0;
-    fp.W = 0;
-    fp.signed_test = 0;
-    fp.st = SlopeState{};
-    fp.out_slopes = nullptr;
-    fp.out_mask = nullptr;
-    if (launch_finalize(fp, 1, b, stream) != cudaSuccess) return EGERIA_ERR_CUDA;
     return EGERIA_OK;
 }

@@ -1,9 +1,13 @@
 // Second half of the SP loss (Eq. 1): sum the partial Grams of every (module, side) in a
 // fixed order, scale every row of G to unit L2 norm, and reduce the squared difference
 // of the two normalised matrices to one number per module, divided by b^2.
-// One warp per row of G; the last CTA of a module (ticket) adds the row terms in
-// ascending order, so the result does not depend on scheduling.  Optionally the same
-// warp then advances the module's freezing rule with the new reading (fused step).
+//
+// The work is cut into rows of G, one warp per row (finalize_row, finalize_row_staged), and one last step per
+// module that adds the row terms in a fixed order (finalize_module_total), so the result
+// does not depend on who did which row or when.  The tensor-core Gram kernel calls both
+// from its own epilogue warps; finalize_kernel wraps them for the modules whose partial
+// Grams came from the CUDA-core kernel.  Optionally the warp that finishes a module also
+// advances the module's freezing rule with the new reading (fused step).
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -17,16 +21,14 @@ constexpr int kFinThreads = 256;
 constexpr int kFinRowsPerCta = kFinThreads / 32;
 constexpr int kMaxB = 256;
 constexpr double kNormEps = 1e-12;
-constexpr int kFinBatch = 8;  // partial slots whose loads are issued together
 
-struct FinParams {
+struct FinCommon {
     const float *slots;
     int64_t slot_floats;
     const SideInfo *sides;  // [2 * M]
     int32_t b;
     float *out_losses;      // [M]
     double *rowloss;        // [M][kMaxB] scratch
-    int32_t *tickets;       // [M], zero between calls
     float *keep;            // [M][2][b*b] normalised matrices, or nullptr
     // fused freezing-rule step (fuse_step != 0): Algorithm 1 on the loss just computed
     int32_t fuse_step;
@@ -37,72 +39,220 @@ struct FinParams {
     uint8_t *out_mask;      // [M] or nullptr
 };
 
-// Row i of G for one side: NC columns per lane (column j = lane + 32 c), partial slots added
-// in ascending slot order in float64.  Loads of kFinBatch slots are in flight together.
+// Columns per lane for a given b (column j = lane + 32 c, c < NC).
+__host__ __device__ inline int fin_nc_of_b(int b) { return b <= 32 ? 1 : (b <= 64 ? 2 : (b <= 128 ? 4 : 8)); }
+
+// Column of G that a lane's c-th value belongs to when a lane owns runs of consecutive columns
+// (so that it can fetch them from shared memory with one vector load): 4-column runs, 128
+// columns apart, for NC >= 4; a 2-column run for NC == 2; one column for NC == 1.
 template <int NC>
-__device__ __forceinline__ void sum_row_partials(const float *slots, int64_t slot_floats, const SideInfo si, int i,
-                                                 int b, int lane, double (&g)[NC]) {
+__device__ __forceinline__ int fin_col(int lane, int c) {
+    return NC >= 4 ? 4 * lane + (c & 3) + 128 * (c >> 2) : NC * lane + c;
+}
+
+// Second half of a row, given its two sums gT, gR (this lane's columns: lane + 32 c, or
+// fin_col(lane, c) if kVec): scale each
+// side to unit L2 norm (norm clamped at kNormEps), leave the normalised rows in `keep` if
+// asked, and return sum_j (G~_T[i][j] - G~_R[i][j])^2 (all lanes).  Float64 throughout; one
+// reciprocal per side instead of a division per entry, and the two sides' reductions are
+// interleaved, because this runs at the very end of the kernel with nothing to overlap it.
+template <int NC, bool kVec>
+__device__ __forceinline__ double row_term(const FinCommon &p, int m, int i, int lane, double (&gT)[NC],
+                                           double (&gR)[NC]) {
+    const int b = p.b;
+    double ssT = 0.0, ssR = 0.0;
 #pragma unroll
-    for (int c = 0; c < NC; ++c) g[c] = 0.0;
-    const float *row0 = slots + (int64_t)si.first_slot * slot_floats + si.side_off + (int64_t)i * si.pitch;
-    for (int u0 = 0; u0 < si.n_slots; u0 += kFinBatch) {
-        float v[kFinBatch][NC];
+    for (int c = 0; c < NC; ++c) {
+        ssT = fma(gT[c], gT[c], ssT);
+        ssR = fma(gR[c], gR[c], ssR);
+    }
 #pragma unroll
-        for (int k = 0; k < kFinBatch; ++k) {
-            const bool live = (u0 + k < si.n_slots);
-            const float *row = row0 + (int64_t)(u0 + k) * slot_floats;
+    for (int o = 16; o > 0; o >>= 1) {
+        ssT += __shfl_xor_sync(0xffffffffu, ssT, o);
+        ssR += __shfl_xor_sync(0xffffffffu, ssR, o);
+    }
+    double nT = sqrt(ssT), nR = sqrt(ssR);
+    if (nT < kNormEps) nT = kNormEps;
+    if (nR < kNormEps) nR = kNormEps;
+    const double invT = 1.0 / nT, invR = 1.0 / nR;
+    double s = 0.0;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        gT[c] *= invT;
+        gR[c] *= invR;
+        const double diff = gT[c] - gR[c];
+        s = fma(diff, diff, s);
+    }
+    if (p.keep) {
+        float *dT = p.keep + ((int64_t)(2 * m) * b + i) * b, *dR = dT + (int64_t)b * b;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const int j = kVec ? fin_col<NC>(lane, c) : lane + 32 * c;
+            if (j < b) {
+                dT[j] = (float)gT[c];
+                dR[j] = (float)gR[c];
+            }
+        }
+    }
+    return warp_sum_f64(s);
+}
+
+// One warp: row i of module m with the partials read straight into registers.  Partial slots
+// are added in ascending slot order in float64; the loads of KB slots per side go together.
+template <int NC>
+__device__ __forceinline__ double finalize_row(const FinCommon &p, const SideInfo sT, const SideInfo sR, int m, int i,
+                                               int lane) {
+    constexpr int KB = (32 / (2 * NC)) > 0 ? (32 / (2 * NC)) : 1;
+    const int b = p.b;
+    double gT[NC], gR[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) gT[c] = gR[c] = 0.0;
+    const float *rowT = p.slots + (int64_t)sT.first_slot * p.slot_floats + sT.side_off + (int64_t)i * sT.pitch;
+    const float *rowR = p.slots + (int64_t)sR.first_slot * p.slot_floats + sR.side_off + (int64_t)i * sR.pitch;
+    const int n_max = sT.n_slots > sR.n_slots ? sT.n_slots : sR.n_slots;
+    for (int u0 = 0; u0 < n_max; u0 += KB) {
+        float vT[KB][NC], vR[KB][NC];
+#pragma unroll
+        for (int k = 0; k < KB; ++k) {
+            const bool liveT = (u0 + k < sT.n_slots), liveR = (u0 + k < sR.n_slots);
+            const float *pT = rowT + (int64_t)(u0 + k) * p.slot_floats;
+            const float *pR = rowR + (int64_t)(u0 + k) * p.slot_floats;
 #pragma unroll
             for (int c = 0; c < NC; ++c) {
                 const int j = lane + 32 * c;
-                v[k][c] = (live && j < b) ? __ldcg(row + j) : 0.f;
+                vT[k][c] = (liveT && j < b) ? __ldcg(pT + j) : 0.f;
+                vR[k][c] = (liveR && j < b) ? __ldcg(pR + j) : 0.f;
             }
         }
 #pragma unroll
-        for (int k = 0; k < kFinBatch; ++k)
+        for (int k = 0; k < KB; ++k)
 #pragma unroll
-            for (int c = 0; c < NC; ++c) g[c] += (double)v[k][c];
+            for (int c = 0; c < NC; ++c) {
+                gT[c] += (double)vT[k][c];
+                gR[c] += (double)vR[k][c];
+            }
     }
+    return row_term<NC, false>(p, m, i, lane, gT, gR);
 }
 
+constexpr int kFinStageBytes = 16384;  // warp-private shared memory of the staged variant
+
+// The same row with the partials staged through `stage` (kFinStageBytes of shared memory that
+// only this warp touches): every 16-byte piece of the row in every partial slot is fetched with
+// cp.async, all in flight together whatever the register budget, then added from shared memory
+// in ascending slot order (A_T's partials, then A_R's).  A lane owns the columns fin_col(lane, c).
+// The partial slots of the tensor-core modes have a row pitch of exactly 32 * NC floats.
+template <int NC>
+__device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const SideInfo sT, const SideInfo sR, int m,
+                                                      int i, int lane, float *stage) {
+    constexpr int kPitch = 32 * NC;                          // floats per row of a partial
+    constexpr int kPieces = kPitch / 4;                      // 16-byte pieces per row: 8, 16, 32, 64
+    constexpr int kCap = kFinStageBytes / (kPitch * 4);      // rows of partials the stage holds
+    constexpr int kLanesPerRow = kPieces < 32 ? kPieces : 32;
+    constexpr int kRowsPerIssue = 32 / kLanesPerRow;         // rows one cp.async of the warp covers
+    constexpr int kIssuesPerRow = (kPieces + 31) / 32;
+    const int b = p.b;
+    double gT[NC], gR[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) gT[c] = gR[c] = 0.0;
+    const float *rowT = p.slots + (int64_t)sT.first_slot * p.slot_floats + sT.side_off + (int64_t)i * kPitch;
+    const float *rowR = p.slots + (int64_t)sR.first_slot * p.slot_floats + sR.side_off + (int64_t)i * kPitch;
+    const int nT = sT.n_slots, n_tot = sT.n_slots + sR.n_slots;
+    const uint32_t stage_addr = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
+    const int sub = lane / kLanesPerRow, piece = lane % kLanesPerRow;
+    for (int s0 = 0; s0 < n_tot; s0 += kCap) {
+        const int G = (n_tot - s0 < kCap) ? n_tot - s0 : kCap;
+        for (int sl0 = 0; sl0 < G; sl0 += kRowsPerIssue) {
+            const int sl = sl0 + sub;
+            if (sl < G) {
+                const int s = s0 + sl;
+                const float *src = (s < nT) ? rowT + (int64_t)s * p.slot_floats : rowR + (int64_t)(s - nT) * p.slot_floats;
+#pragma unroll
+                for (int q = 0; q < kIssuesPerRow; ++q) {
+                    const int off = 4 * (piece + 32 * q);
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_addr + (sl * kPitch + off) * 4),
+                                 "l"(src + off)
+                                 : "memory");
+                }
+            }
+        }
+        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+        for (int sl = 0; sl < G; ++sl) {
+            const float *row = stage + sl * kPitch;
+            float v[NC];
+            if (NC >= 4) {
+#pragma unroll
+                for (int h = 0; h < NC / 4; ++h) {
+                    const float4 t = *reinterpret_cast<const float4 *>(row + 128 * h + 4 * lane);
+                    v[4 * h] = t.x;
+                    v[4 * h + 1] = t.y;
+                    v[4 * h + 2] = t.z;
+                    v[4 * h + 3] = t.w;
+                }
+            } else if (NC == 2) {
+                const float2 t = *reinterpret_cast<const float2 *>(row + 2 * lane);
+                v[0] = t.x;
+                v[NC - 1] = t.y;
+            } else {
+                v[0] = row[lane];
+            }
+            if (s0 + sl < nT) {  // uniform over the warp
+#pragma unroll
+                for (int c = 0; c < NC; ++c) gT[c] += (double)v[c];
+            } else {
+#pragma unroll
+                for (int c = 0; c < NC; ++c) gR[c] += (double)v[c];
+            }
+        }
+        __syncwarp();  // everyone has read the stage before the next pass overwrites it
+    }
+    // columns beyond b were never written by anyone: whatever was added there is dropped
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+        if (fin_col<NC>(lane, c) >= b) gT[c] = gR[c] = 0.0;
+    return row_term<NC, true>(p, m, i, lane, gT, gR);
+}
+
+// One warp, once every row term of module m is in p.rowloss and visible: the loss (Eq. 1),
+// then optionally one evaluation of the freezing rule.
+__device__ __forceinline__ void finalize_module_total(const FinCommon &p, int m, int lane) {
+    const int b = p.b;
+    double v[kMaxB / 32];
+#pragma unroll
+    for (int j = 0; j < kMaxB / 32; ++j) {
+        const int r = lane + 32 * j;
+        v[j] = (r < b) ? __ldcg(&p.rowloss[(int64_t)m * kMaxB + r]) : 0.0;
+    }
+    StepLoaded L;
+    if (p.fuse_step) L = plasticity_step_load(p.st, m, p.W, lane);  // in flight together with the row terms
+    double s = 0.0;
+#pragma unroll
+    for (int j = 0; j < kMaxB / 32; ++j) s += v[j];
+    s = warp_sum_f64(s);
+    const float loss = (float)(s / ((double)b * (double)b));
+    if (lane == 0) p.out_losses[m] = loss;
+    if (p.fuse_step) plasticity_step_apply(p.st, L, m, p.W, p.signed_test, loss, p.out_slopes, p.out_mask, lane);
+}
+
+struct FinParams {
+    FinCommon c;
+    int32_t *tickets;  // [M], zero between calls
+};
+
+// Modules whose partial Grams came from the CUDA-core kernel.  grid = (M, ceil(b / 8)).
 template <int NC>
 __global__ void __launch_bounds__(kFinThreads) finalize_kernel(const FinParams p) {
     const int m = blockIdx.x;
+    if (p.c.sides[2 * m].tensor_core) return;  // finished inside the tensor-core kernel
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = p.b;
+    const int b = p.c.b;
     const int i = blockIdx.y * kFinRowsPerCta + warp;
     __shared__ int is_last;
 
     if (i < b) {
-        double g[2][NC];
-        sum_row_partials<NC>(p.slots, p.slot_floats, p.sides[2 * m], i, b, lane, g[0]);
-        sum_row_partials<NC>(p.slots, p.slot_floats, p.sides[2 * m + 1], i, b, lane, g[1]);
-#pragma unroll
-        for (int side = 0; side < 2; ++side) {
-            double ss = 0.0;
-#pragma unroll
-            for (int c = 0; c < NC; ++c) ss += g[side][c] * g[side][c];
-            ss = warp_sum_f64(ss);
-            double n = sqrt(ss);
-            if (n < kNormEps) n = kNormEps;
-#pragma unroll
-            for (int c = 0; c < NC; ++c) g[side][c] = g[side][c] / n;
-            if (p.keep) {
-                float *dst = p.keep + ((int64_t)(2 * m + side) * b + i) * b;
-#pragma unroll
-                for (int c = 0; c < NC; ++c) {
-                    const int j = lane + 32 * c;
-                    if (j < b) dst[j] = (float)g[side][c];
-                }
-            }
-        }
-        double s = 0.0;
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-            const double diff = g[0][c] - g[1][c];
-            s += diff * diff;
-        }
-        s = warp_sum_f64(s);
-        if (lane == 0) p.rowloss[(int64_t)m * kMaxB + i] = s;
+        const double s = finalize_row<NC>(p.c, p.c.sides[2 * m], p.c.sides[2 * m + 1], m, i, lane);
+        if (lane == 0) p.c.rowloss[(int64_t)m * kMaxB + i] = s;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -113,15 +263,8 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(const FinParams p
     __syncthreads();
     if (is_last && warp == 0) {
         __threadfence();
-        double s = 0.0;
-        for (int r = lane; r < b; r += 32) s += __ldcg(&p.rowloss[(int64_t)m * kMaxB + r]);
-        s = warp_sum_f64(s);
-        const float loss = (float)(s / ((double)b * (double)b));
-        if (lane == 0) {
-            p.out_losses[m] = loss;
-            p.tickets[m] = 0;
-        }
-        if (p.fuse_step) plasticity_step_module(p.st, m, p.W, p.signed_test, loss, p.out_slopes, p.out_mask, lane);
+        if (lane == 0) p.tickets[m] = 0;
+        finalize_module_total(p.c, m, lane);
     }
 }
 

@@ -45,7 +45,7 @@ __global__ void __launch_bounds__(kSimtThreads) gram_simt_kernel(const SimtParam
         for (int side = 0; side < 2; ++side) {
             if (u.side != 2 && u.side != side) continue;
             const __nv_bfloat16 *A = static_cast<const __nv_bfloat16 *>(side == 0 ? mp.At : mp.Ar);
-            float *out = slot + ((p.mode == kStacked) ? side * 64 * 64 : 0);
+            float *out = slot + (mode_is_stacked(p.mode) ? side * pitch * pitch : 0);
             for (int bi = 0; bi < nblk; ++bi) {
                 for (int bj = bi; bj < nblk; ++bj) {
                     float acc[4][4];

@@ -1,40 +1,66 @@
-// Partial Gram matrices G = A A^T on the 5th-generation tensor cores (sm_100a).
+// The SP loss (Eq. 1) of all tensor-core modules in ONE launch on sm_100a: partial Gram
+// matrices G = A A^T on the 5th-generation tensor cores, then row normalisation, difference
+// and Frobenius reduction by the same kernel.
 //
 // One persistent CTA per SM walks its static list of work units (a K-range of one
 // (module, side) tile).  Per 64-element block of the feature axis, one TMA box load
 // brings all b rows into a 128-byte-swizzled shared-memory slab; the same slab is
 // both the A and the B operand of tcgen05.mma (row block i against row block j,
 // i <= j), accumulating in fp32 in tensor memory.  At the end of a unit the
-// accumulator is drained to the unit's partial slot in the workspace.
+// accumulator is drained to the unit's partial slot in the workspace (L2-resident).
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
-// owner, warps 2..5 = epilogue (TMEM -> registers -> global).
-// Every mbarrier wait is bounded; on expiry the CTA raises its abort flag, records
+// A module is finished by the CTAs that worked on it.  Every unit bumps the module's
+// units_done counter.  A CTA that has done all its units goes through the modules it worked
+// on: where all units of the module are in (for the module of its last unit it waits briefly),
+// its epilogue warps claim rows of G one by one from the module's row cursor, fetch the row
+// of every partial into shared memory (the operand ring is idle by then), add them in a
+// fixed order, normalise, take the difference, square, and reduce with warp shuffles.  The
+// warp that delivers the module's last row adds the row terms in a fixed order and writes the
+// loss (and, if asked, advances the freezing rule).  Whoever delivers a module's last unit
+// always gets to this point after it, so every module is finished; and the result never
+// depends on which warp did what.
+//
+// Warp roles (448 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
+// owner, warps 2..13 = epilogue (TMEM -> registers -> global, then the finalisation); a warp
+// may read only the TMEM lane quarter (warp index mod 4), so three warps share each quarter
+// and split its columns.
+// Every wait is bounded; on expiry the CTA raises its abort flag, records
 // EGERIA_ERR_TIMEOUT in the status word, drains what is in flight and returns.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "finalize.cuh"
 #include "plan.h"
 #include "ptx_sm100.cuh"
 
 namespace egeria {
 
-constexpr int kTcThreads = 192;
+constexpr int kEpiWarps = 12;                     // three per TMEM lane quarter
+constexpr int kEpiThreads = 32 * kEpiWarps;
+constexpr int kTcThreads = 64 + kEpiThreads;      // + TMA producer warp + MMA warp
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s per wait
+constexpr uint64_t kHelpWaitNs = 1000000ull;      // 1 ms: how long a finished CTA waits to help
 constexpr int kStatusTimeout = 6;                 // == EGERIA_ERR_TIMEOUT
 
 template <int MODE>
 struct TcCfg {
-    static constexpr int kSlabRows = (MODE == kSingle2) ? 256 : 128;
-    static constexpr int kStageBytes = kSlabRows * 128;          // one 64-element block of all rows
-    static constexpr int kStages = (MODE == kSingle2) ? 6 : 12;  // 192 KB of loads in flight
-    static constexpr int kAccCols = (MODE == kSingle2) ? 384 : 128;
+    static constexpr bool kStacked = (MODE == kStacked32 || MODE == kStacked64);
+    static constexpr int kBoxRows = (MODE == kStacked32) ? 32 : (MODE == kStacked64 ? 64 : (MODE == kSingle1 ? 128 : 256));
+    static constexpr int kSlabRows = kStacked ? 2 * kBoxRows : kBoxRows;   // rows of one 64-column slab
+    static constexpr int kSlabBytes = kSlabRows * 128;
+    static constexpr int kKbPerStage = (MODE == kStacked32) ? 2 : 1;       // slabs per pipeline stage
+    static constexpr int kStageBytes = kSlabBytes * kKbPerStage;           // 16 KB (32 KB for b > 128)
+    static constexpr int kStages = (MODE == kSingle2) ? 6 : 12;            // 192 KB of loads in flight
+    // kStacked32 issues M = 128 MMAs over a 64-row slab: the A operand reaches one slab further.
+    static constexpr int kPadBytes = (MODE == kStacked32) ? kSlabBytes : 0;
+    static constexpr int kAccCols = (MODE == kStacked32) ? 64 : (MODE == kSingle2 ? 384 : 128);
     static constexpr int kAccStages = (MODE == kSingle2) ? 1 : 2;
-    static constexpr int kTmemCols = (MODE == kSingle2) ? 512 : 256;
-    static constexpr int kBoxRows = (MODE == kStacked) ? 64 : kSlabRows;  // rows of one TMA box
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
+    static constexpr int kTmemCols = (MODE == kStacked32) ? 128 : (MODE == kSingle2 ? 512 : 256);
+    static constexpr int kNC = (MODE == kStacked32) ? 1 : (MODE == kStacked64 ? 2 : (MODE == kSingle1 ? 4 : 8));
+    static constexpr int kSmemBytes =
+        kStages * kStageBytes + kPadBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
 };
 
 struct TcParams {
@@ -42,10 +68,156 @@ struct TcParams {
     const Unit *units;         // tensor-core units
     const int32_t *cta_begin;  // [gridDim.x + 1]
     float *slots;              // partial Gram slots
-    int64_t slot_floats;
-    int32_t b;
     int32_t *status;           // device status word
+    FinCounters *ctr;          // [M] progress counters of this launch (all zero at launch)
+    FinCounters *ctr_next;     // [M] the set the next launch will use: cleared here
+    int32_t M;
+    FinCommon fin;             // slots, sides, b, outputs, freezing-rule state
 };
+
+namespace detail {
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+// All epilogue threads: AND of `pred` over them.
+__device__ __forceinline__ bool epi_bar_and(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t"
+        "}"
+        : "=r"(out)
+        : "r"((uint32_t)pred), "n"(kEpiThreads)
+        : "memory");
+    return out != 0;
+}
+__device__ __forceinline__ int ld_acquire(const int32_t *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// One 32-row x 32-column piece of an accumulator, as one epilogue warp sees it: where it is in
+// tensor memory and where this lane's row of it goes in the partial slot.
+struct Chunk {
+    uint32_t col;      // first TMEM column
+    float *dst;        // this lane's 32 floats in the slot
+    bool valid;        // this lane's row is a row of G
+    int mirror_c0;     // kSingle2: first column of a G01 chunk that is also written transposed, else -1
+};
+
+// Chunk k of the accumulator of one unit, for the warp of TMEM lane quarter q.  False if there
+// is no such chunk (warp-uniform).  Layouts per mode:
+//   kStacked32: rows 0..31 x cols 0..31 = G_T, rows 32..63 x cols 32..63 = G_R
+//   kStacked64: rows 0..63 x cols 0..63 = G_T, rows 64..127 x cols 64..127 = G_R
+//   kSingle1:   rows 0..127 x cols 0..127 = G
+//   kSingle2:   cols 0..255 = rows 0..127 of G (all 256 columns); cols 256..383 = G11
+template <int MODE>
+__device__ __forceinline__ bool chunk_of(int k, int q, int lane, int b, float *slot, Chunk &ch) {
+    ch.mirror_c0 = -1;
+    if (MODE == kStacked32) {
+        if (k != 0 || q >= 2) return false;
+        ch.col = q * 32;
+        ch.dst = slot + q * 32 * 32 + lane * 32;
+        ch.valid = lane < b;
+        return true;
+    } else if (MODE == kStacked64) {
+        const int side = q >> 1, r = (q & 1) * 32 + lane, c0 = 32 * k;
+        if (k >= 2 || c0 >= b || (q & 1) * 32 >= b) return false;
+        ch.col = side * 64 + c0;
+        ch.dst = slot + side * 64 * 64 + r * 64 + c0;
+        ch.valid = r < b;
+        return true;
+    } else if (MODE == kSingle1) {
+        const int r = q * 32 + lane, c0 = 32 * k;
+        if (k >= 4 || c0 >= b || q * 32 >= b) return false;
+        ch.col = c0;
+        ch.dst = slot + r * 128 + c0;
+        ch.valid = r < b;
+        return true;
+    } else {
+        const int r = q * 32 + lane;  // 0..127, always < b in this mode
+        if (k < 8) {
+            const int c0 = 32 * k;
+            if (c0 >= b) return false;
+            ch.col = c0;
+            ch.dst = slot + r * 256 + c0;
+            ch.valid = true;
+            if (c0 >= 128) ch.mirror_c0 = c0;
+            return true;
+        }
+        const int l = 32 * (k - 8);
+        if (k >= 12 || 128 + l >= b || 128 + q * 32 >= b) return false;
+        ch.col = 256 + l;
+        ch.dst = slot + (128 + r) * 256 + 128 + l;
+        ch.valid = 128 + r < b;
+        return true;
+    }
+}
+
+// First existing chunk among k, k + 3, k + 6, ... (k is advanced to it).  Warp-uniform.
+template <int MODE>
+__device__ __forceinline__ bool next_chunk(int &k, int q, int lane, int b, float *slot, Chunk &ch) {
+    constexpr int kChunks = (MODE == kStacked32) ? 1 : (MODE == kStacked64 ? 2 : (MODE == kSingle1 ? 4 : 12));
+    for (; k < kChunks; k += 3)
+        if (chunk_of<MODE>(k, q, lane, b, slot, ch)) return true;
+    return false;
+}
+
+// One warp: wait until `total` units of the module are complete, to help finish it.  The
+// wait is a courtesy, not a dependency: the CTA that delivers the module's last unit finishes
+// every row nobody else has claimed, so a warp that stops waiting (false) loses nothing but
+// parallelism.  That keeps the kernel correct when not all of its CTAs are resident together.
+__device__ __forceinline__ bool wait_units_done(const int32_t *units_done, int total, volatile int *abort_flag,
+                                                int lane) {
+    int ok = 1;
+    if (lane == 0) {
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ld_acquire(units_done) < total) {
+            if (*abort_flag || ptx::globaltimer_ns() - t0 > kHelpWaitNs) {
+                ok = 0;
+                break;
+            }
+            __nanosleep(40);
+        }
+    }
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+// One warp: take rows of module m from its cursor until none is left.  The claim of the next
+// row is in flight while the current one is worked on; the rows are published together.
+// `stage` is kFinStageBytes of shared memory for this warp alone.
+template <int NC>
+__device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int lane, float *stage) {
+    const int b = p.fin.b;
+    FinCounters *c = p.ctr + m;
+    int mine = 0;
+    int r = 0;
+    if (lane == 0) r = atomicAdd(&c->row_cursor, 1);
+    const SideInfo sT = p.fin.sides[2 * m], sR = p.fin.sides[2 * m + 1];  // in flight with the claim
+    r = __shfl_sync(0xffffffffu, r, 0);
+    while (r < b) {
+        int r_next = 0;
+        if (lane == 0) r_next = atomicAdd(&c->row_cursor, 1);
+        const double term = finalize_row_staged<NC>(p.fin, sT, sR, m, r, lane, stage);
+        if (lane == 0) p.fin.rowloss[(int64_t)m * kMaxB + r] = term;
+        ++mine;
+        r = __shfl_sync(0xffffffffu, r_next, 0);
+    }
+    if (mine == 0) return;
+    int before = 0;
+    if (lane == 0) {
+        __threadfence();
+        before = atomicAdd(&c->rows_done, mine);
+    }
+    before = __shfl_sync(0xffffffffu, before, 0);
+    if (before + mine == b) {
+        __threadfence();
+        finalize_module_total(p.fin, m, lane);
+    }
+}
+}  // namespace detail
 
 template <int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p) {
@@ -54,7 +226,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     // 1024-byte alignment: the 128-byte swizzle pattern is a function of address bits 4..9.
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_aligned = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_aligned + Cfg::kStages * Cfg::kStageBytes);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_aligned + Cfg::kStages * Cfg::kStageBytes + Cfg::kPadBytes);
     // bars: full[kStages], empty[kStages], acc_full[kAccStages], acc_empty[kAccStages]
     const uint32_t full0 = ptx::smem_u32(bars);
     const uint32_t empty0 = full0 + 8 * Cfg::kStages;
@@ -69,6 +241,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     const int u_begin = p.cta_begin[blockIdx.x];
     const int u_end = p.cta_begin[blockIdx.x + 1];
 
+    // The counters of the next launch start at zero (nobody reads that set during this launch).
+    {
+        int32_t *z = reinterpret_cast<int32_t *>(p.ctr_next);
+        const int n = p.M * (int)(sizeof(FinCounters) / sizeof(int32_t));
+        for (int i = blockIdx.x * kTcThreads + threadIdx.x; i < n; i += gridDim.x * kTcThreads) z[i] = 0;
+    }
+
     if (threadIdx.x == 0) {
         for (int s = 0; s < Cfg::kStages; ++s) {
             ptx::mbar_init(full0 + 8 * s, 1);
@@ -76,7 +255,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         }
         for (int s = 0; s < Cfg::kAccStages; ++s) {
             ptx::mbar_init(accfull0 + 8 * s, 1);
-            ptx::mbar_init(accempty0 + 8 * s, 4);  // one arrival per epilogue warp
+            ptx::mbar_init(accempty0 + 8 * s, kEpiWarps);  // one arrival per epilogue warp
         }
         *abort_flag = 0;
         ptx::fence_barrier_init();
@@ -109,19 +288,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                     last_module = u.module;
                 }
                 const CUtensorMap *tm_side = (u.side == 1) ? tm_r : tm_t;
-                for (int kb = u.kb0; kb < u.kb0 + u.nkb; ++kb) {
+                const int kb_end = u.kb0 + u.nkb;
+                for (int kb = u.kb0; kb < kb_end; kb += Cfg::kKbPerStage) {
                     if (!ptx::mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u, abort_flag, kWaitLimitNs)) {
                         ok = false;
                         break;
                     }
                     const uint32_t dst = smem_base + stage * Cfg::kStageBytes;
                     const uint32_t bar = full0 + 8 * stage;
-                    ptx::mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
-                    if (MODE == kStacked) {
-                        ptx::tma_load_2d(dst, tm_t, kb * kKBlock, 0, bar, policy);
-                        ptx::tma_load_2d(dst + 64 * 128, tm_r, kb * kKBlock, 0, bar, policy);
-                    } else {
-                        ptx::tma_load_2d(dst, tm_side, kb * kKBlock, 0, bar, policy);
+                    const int nk = (kb_end - kb < Cfg::kKbPerStage) ? kb_end - kb : Cfg::kKbPerStage;
+                    ptx::mbar_arrive_expect_tx(bar, (uint32_t)nk * Cfg::kSlabBytes);
+#pragma unroll
+                    for (int j = 0; j < Cfg::kKbPerStage; ++j) {
+                        if (j >= nk) break;
+                        const uint32_t slab = dst + j * Cfg::kSlabBytes;
+                        if (Cfg::kStacked) {
+                            ptx::tma_load_2d(slab, tm_t, (kb + j) * kKBlock, 0, bar, policy);
+                            ptx::tma_load_2d(slab + Cfg::kBoxRows * 128, tm_r, (kb + j) * kKBlock, 0, bar, policy);
+                        } else {
+                            ptx::tma_load_2d(slab, tm_side, (kb + j) * kKBlock, 0, bar, policy);
+                        }
                     }
                     ++issued;
                     if (++stage == Cfg::kStages) {
@@ -147,6 +333,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
+            constexpr uint32_t idesc64 = ptx::make_idesc_bf16_f32(128, 64);
             constexpr uint32_t idesc128 = ptx::make_idesc_bf16_f32(128, 128);
             constexpr uint32_t idesc256 = ptx::make_idesc_bf16_f32(128, 256);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
@@ -160,29 +347,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 }
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * Cfg::kAccCols;
-                for (int kb = 0; kb < u.nkb; ++kb) {
+                for (int kb = 0; kb < u.nkb; kb += Cfg::kKbPerStage) {
                     if (!ptx::mbar_wait_bounded(full0 + 8 * stage, phase, abort_flag, kWaitLimitNs)) {
                         ok = false;
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    const uint32_t slab = smem_base + stage * Cfg::kStageBytes;
+                    const int nk = (u.nkb - kb < Cfg::kKbPerStage) ? u.nkb - kb : Cfg::kKbPerStage;
 #pragma unroll
-                    for (int k = 0; k < kKBlock / 16; ++k) {
-                        const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
-                        const uint64_t lo = ptx::make_desc_k_sw128(slab + k * 32);
-                        if (MODE == kSingle2) {
-                            const uint64_t hi = ptx::make_desc_k_sw128(slab + 128 * 128 + k * 32);
-                            // [G00 | G01] = rows 0..127 against rows 0..255
-                            ptx::mma_bf16_ss(d_tmem, lo, lo, idesc256, accum);
-                            // G11 = rows 128..255 against themselves
-                            ptx::mma_bf16_ss(d_tmem + 256, hi, hi, idesc128, accum);
-                        } else {
-                            ptx::mma_bf16_ss(d_tmem, lo, lo, idesc128, accum);
+                    for (int j = 0; j < Cfg::kKbPerStage; ++j) {
+                        if (j >= nk) break;
+                        const uint32_t slab = smem_base + stage * Cfg::kStageBytes + j * Cfg::kSlabBytes;
+#pragma unroll
+                        for (int k = 0; k < kKBlock / 16; ++k) {
+                            const uint32_t accum = (kb > 0 || j > 0 || k > 0) ? 1u : 0u;
+                            const uint64_t lo = ptx::make_desc_k_sw128(slab + k * 32);
+                            if (MODE == kSingle2) {
+                                const uint64_t hi = ptx::make_desc_k_sw128(slab + 128 * 128 + k * 32);
+                                // [G00 | G01] = rows 0..127 against rows 0..255
+                                ptx::mma_bf16_ss(d_tmem, lo, lo, idesc256, accum);
+                                // G11 = rows 128..255 against themselves
+                                ptx::mma_bf16_ss(d_tmem + 256, hi, hi, idesc128, accum);
+                            } else if (MODE == kStacked32) {
+                                // 128 operand rows, of which only 0..63 (this slab) matter
+                                ptx::mma_bf16_ss(d_tmem, lo, lo, idesc64, accum);
+                            } else {
+                                ptx::mma_bf16_ss(d_tmem, lo, lo, idesc128, accum);
+                            }
                         }
                     }
                     any_mma = true;
-                    ptx::mma_commit(empty0 + 8 * stage);  // slab free once these MMAs have read it
+                    ptx::mma_commit(empty0 + 8 * stage);  // stage free once these MMAs have read it
                     if (++stage == Cfg::kStages) {
                         stage = 0;
                         phase ^= 1u;
@@ -206,86 +401,116 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         __syncwarp();
     } else {
         // ------------------------------------------------------------ epilogue warps
-        const int q = warp & 3;  // TMEM lane quarter this warp may read
-        const int b = p.b;
+        const int q = warp & 3;           // TMEM lane quarter this warp may read
+        const int part = (warp - 2) >> 2;  // which third of the quarter's columns this warp drains
+        const int b = p.fin.b;
+        const bool epi_leader = (threadIdx.x == 64);
         uint32_t acc = 0, acc_phase = 0;
-        bool ok = true;
-        for (int ui = u_begin; ui < u_end && ok; ++ui) {
+        bool aborted = false;
+        for (int ui = u_begin; ui < u_end; ++ui) {
             const Unit u = p.units[ui];
-            if (!ptx::mbar_wait_bounded(accfull0 + 8 * acc, acc_phase, abort_flag, kWaitLimitNs)) {
-                ok = false;
+            const bool got = ptx::mbar_wait_bounded(accfull0 + 8 * acc, acc_phase, abort_flag, kWaitLimitNs);
+            if (!detail::epi_bar_and(got)) {  // the epilogue warps leave together
+                aborted = true;
                 break;
             }
             ptx::tc_fence_after_sync();
-            float *slot = p.slots + (int64_t)u.slot * p.slot_floats;
+            float *slot = p.slots + (int64_t)u.slot * p.fin.slot_floats;
             const uint32_t t_row = tmem_base + acc * Cfg::kAccCols + ((uint32_t)(q * 32) << 16);
-            uint32_t v[32];
-            if (MODE == kStacked) {
-                // rows 0..63 x cols 0..63 = G_T, rows 64..127 x cols 64..127 = G_R
-                const int side = q >> 1;
-                const int r = (q & 1) * 32 + lane;
-                if ((q & 1) * 32 < b) {
-                    float *dst = slot + side * 64 * 64 + r * 64;
-                    for (int c0 = 0; c0 < 64 && c0 < b; c0 += 32) {
-                        ptx::tmem_ld_32x32(t_row + side * 64 + c0, v);
-                        ptx::tmem_ld_wait();
-                        if (r < b) {
+            // This warp's share of the accumulator: 32 x 32 chunks part, part + 3, ...; the load of
+            // the next chunk is in flight while the current one is stored.
+            detail::Chunk ch, nx;
+            int k = part;
+            bool have = detail::next_chunk<MODE>(k, q, lane, b, slot, ch);
+            uint32_t v[32], w[32];
+            if (have) ptx::tmem_ld_32x32(t_row + ch.col, w);
+            while (have) {
+                ptx::tmem_ld_wait();
 #pragma unroll
-                            for (int c = 0; c < 32; c += 4)
-                                *reinterpret_cast<uint4 *>(dst + c0 + c) = make_uint4(v[c], v[c + 1], v[c + 2], v[c + 3]);
-                        }
-                    }
+                for (int c = 0; c < 32; ++c) v[c] = w[c];
+                k += 3;
+                const bool have_next = detail::next_chunk<MODE>(k, q, lane, b, slot, nx);
+                if (have_next) ptx::tmem_ld_32x32(t_row + nx.col, w);
+                if (ch.valid) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) ptx::st_global_v8(ch.dst + c, v + c);
                 }
-            } else if (MODE == kSingle1) {
-                const int r = q * 32 + lane;
-                if (q * 32 < b) {
-                    float *dst = slot + r * 128;
-                    for (int c0 = 0; c0 < 128 && c0 < b; c0 += 32) {
-                        ptx::tmem_ld_32x32(t_row + c0, v);
-                        ptx::tmem_ld_wait();
-                        if (r < b) {
+                if (MODE == kSingle2 && ch.mirror_c0 >= 0) {
+                    // mirror G01 into the lower-left block: lanes write consecutive floats
+                    const int r = q * 32 + lane;
 #pragma unroll
-                            for (int c = 0; c < 32; c += 4)
-                                *reinterpret_cast<uint4 *>(dst + c0 + c) = make_uint4(v[c], v[c + 1], v[c + 2], v[c + 3]);
-                        }
-                    }
+                    for (int c = 0; c < 32; ++c)
+                        if (ch.mirror_c0 + c < b) slot[(ch.mirror_c0 + c) * 256 + r] = __uint_as_float(v[c]);
                 }
-            } else {
-                // TMEM cols 0..255: rows 0..127 of G (all 256 columns); cols 256..383: G11.
-                const int r = q * 32 + lane;  // 0..127, always < b in this mode
-                float *dst = slot + r * 256;
-                for (int c0 = 0; c0 < 256 && c0 < b; c0 += 32) {
-                    ptx::tmem_ld_32x32(t_row + c0, v);
-                    ptx::tmem_ld_wait();
-#pragma unroll
-                    for (int c = 0; c < 32; c += 4)
-                        *reinterpret_cast<uint4 *>(dst + c0 + c) = make_uint4(v[c], v[c + 1], v[c + 2], v[c + 3]);
-                    if (c0 >= 128) {
-                        // mirror G01 into the lower-left block: lanes write consecutive floats
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (c0 + c < b) slot[(c0 + c) * 256 + r] = __uint_as_float(v[c]);
-                    }
-                }
-                if (128 + q * 32 < b) {
-                    float *dst2 = slot + (128 + r) * 256 + 128;
-                    for (int c0 = 0; c0 < 128 && 128 + c0 < b; c0 += 32) {
-                        ptx::tmem_ld_32x32(t_row + 256 + c0, v);
-                        ptx::tmem_ld_wait();
-                        if (128 + r < b) {
-#pragma unroll
-                            for (int c = 0; c < 32; c += 4)
-                                *reinterpret_cast<uint4 *>(dst2 + c0 + c) = make_uint4(v[c], v[c + 1], v[c + 2], v[c + 3]);
-                        }
-                    }
-                }
+                ch = nx;
+                have = have_next;
             }
+            // Hand the accumulator back before anything else: the next unit's MMAs can start.
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(accempty0 + 8 * acc);
             if (++acc == Cfg::kAccStages) {
                 acc = 0;
                 acc_phase ^= 1u;
+            }
+
+            // Publish the partial: every thread's stores, then one count for the unit.
+            __threadfence();
+            detail::epi_bar_sync();
+            if (epi_leader) atomicAdd(&p.ctr[u.module].units_done, 1);
+        }
+        if (!aborted) {
+            // All of this CTA's units are in and its pipeline is idle, so the operand ring is free:
+            // each epilogue warp takes kFinStageBytes of it as its staging area and helps finish the
+            // modules this CTA worked on, as far as they are complete.
+            static_assert(kEpiWarps * kFinStageBytes <= Cfg::kStages * Cfg::kStageBytes, "ring too small to stage");
+            float *stage = reinterpret_cast<float *>(smem_aligned + (warp - 2) * kFinStageBytes);
+            ptx::fence_proxy_async();  // the ring was last touched by TMA and the tensor cores
+            const int m_last = (u_end > u_begin) ? p.units[u_end - 1].module : -1;
+            int prev_m = -1;
+            for (int ui = u_begin; ui < u_end; ++ui) {
+                const int m = p.units[ui].module;
+                if (m == prev_m) continue;
+                prev_m = m;
+                const int total = p.fin.sides[2 * m].module_units;
+                int done = 0;
+                if (lane == 0) done = detail::ld_acquire(&p.ctr[m].units_done);
+                bool ready = (__shfl_sync(0xffffffffu, done, 0) >= total);
+                if (!ready && m == m_last)
+                    ready = detail::wait_units_done(&p.ctr[m].units_done, total, abort_flag, lane);
+                if (ready) {
+                    __threadfence();
+                    detail::finish_module_rows<Cfg::kNC>(p, m, lane, stage);
+                }
+            }
+            // Then look at all the other modules, a few times: where one is complete and still has
+            // many rows nobody has claimed (few CTAs worked on it, so its rows go slowly), lend a
+            // hand to the one with the most rows left.
+            for (int round = 0; round < 3; ++round) {
+                int best_left = 0, best_m = -1;
+                for (int mm = lane; mm < p.M; mm += 32) {
+                    const SideInfo si = p.fin.sides[2 * mm];
+                    if (!si.tensor_core) continue;
+                    const int done = detail::ld_acquire(&p.ctr[mm].units_done);
+                    const int cur = detail::ld_acquire(&p.ctr[mm].row_cursor);
+                    const int left = (done >= si.module_units) ? b - cur : 0;
+                    if (left > best_left) {
+                        best_left = left;
+                        best_m = mm;
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const int ol = __shfl_xor_sync(0xffffffffu, best_left, o);
+                    const int om = __shfl_xor_sync(0xffffffffu, best_m, o);
+                    if (ol > best_left || (ol == best_left && om > best_m)) {
+                        best_left = ol;
+                        best_m = om;
+                    }
+                }
+                if (best_left < 2 * kEpiWarps) break;  // not worth a round trip: its own CTAs are about done
+                __threadfence();
+                detail::finish_module_rows<Cfg::kNC>(p, best_m, lane, stage);
             }
         }
     }

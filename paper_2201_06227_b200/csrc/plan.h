@@ -16,24 +16,34 @@ namespace egeria {
 constexpr int kKBlock = 64;
 
 // How the b rows of A_T / A_R are laid into MMA tiles.
-//   kStacked : b <= 64.  One tile per module: A_T in rows 0..63 and A_R in rows 64..127 of a
-//              128-row slab, one 128x128 MMA; the two diagonal 64x64 blocks are G_T and G_R.
-//   kSingle1 : b <= 128. One tile per (module, side): 128-row slab, one 128x128 MMA.
-//   kSingle2 : b <= 256. One tile per (module, side): 256-row slab, the upper triangle of
-//              2x2 blocks of 128 (G00|G01 as one 128x256 MMA, G11 as one 128x128 MMA).
-enum Mode : int { kStacked = 0, kSingle1 = 1, kSingle2 = 2 };
+//   kStacked32 : b <= 32.  One tile per module: A_T in rows 0..31 and A_R in rows 32..63 of a
+//                64-row slab, one 128x64 MMA (the upper 64 accumulator rows are unused); the
+//                two diagonal 32x32 blocks are G_T and G_R.
+//   kStacked64 : b <= 64.  Same with 64 rows per side: 128-row slab, one 128x128 MMA.
+//   kSingle1   : b <= 128. One tile per (module, side): 128-row slab, one 128x128 MMA.
+//   kSingle2   : b <= 256. One tile per (module, side): 256-row slab, the upper triangle of
+//                2x2 blocks of 128 (G00|G01 as one 128x256 MMA, G11 as one 128x128 MMA).
+enum Mode : int { kStacked32 = 0, kStacked64 = 1, kSingle1 = 2, kSingle2 = 3 };
+constexpr int kNumModes = 4;
 
-__host__ __device__ inline int mode_of_b(int b) { return b <= 64 ? kStacked : (b <= 128 ? kSingle1 : kSingle2); }
-__host__ __device__ inline int pitch_of_mode(int mode) { return mode == kStacked ? 64 : (mode == kSingle1 ? 128 : 256); }
-// fp32 values of one partial-Gram slot.
+__host__ __device__ inline int mode_of_b(int b) {
+    return b <= 32 ? kStacked32 : (b <= 64 ? kStacked64 : (b <= 128 ? kSingle1 : kSingle2));
+}
+__host__ __device__ inline bool mode_is_stacked(int mode) { return mode <= kStacked64; }
+// Row pitch (floats) of a partial Gram; for the stacked modes also the rows per side.
+__host__ __device__ inline int pitch_of_mode(int mode) {
+    return mode == kStacked32 ? 32 : (mode == kStacked64 ? 64 : (mode == kSingle1 ? 128 : 256));
+}
+// fp32 values of one partial-Gram slot ([2][h][h] when stacked, else [pitch][pitch]).
 __host__ __device__ inline int64_t slot_floats_of_mode(int mode) {
-    return mode == kStacked ? 2 * 64 * 64 : (mode == kSingle1 ? 128 * 128 : 256 * 256);
+    const int64_t p = pitch_of_mode(mode);
+    return mode_is_stacked(mode) ? 2 * p * p : p * p;
 }
 
 // One work unit: a K-range of one tile, done by one CTA, leaving one partial Gram in `slot`.
 struct Unit {
     int32_t module;
-    int32_t side;  // 0 = A_T, 1 = A_R, 2 = both (kStacked)
+    int32_t side;  // 0 = A_T, 1 = A_R, 2 = both (stacked modes)
     int32_t kb0;   // first 64-element block
     int32_t nkb;   // number of blocks
     int32_t slot;  // partial slot index
@@ -44,8 +54,20 @@ struct Unit {
 struct SideInfo {
     int32_t first_slot;
     int32_t n_slots;
-    int32_t side_off;  // float offset of this side inside a slot (kStacked: side * 64 * 64)
-    int32_t pitch;     // row pitch of the partial, in floats
+    int32_t side_off;      // float offset of this side inside a slot (stacked: side * h * h)
+    int32_t pitch;         // row pitch of the partial, in floats
+    int32_t tensor_core;   // 1: the module's units belong to the tensor-core kernel, which also
+                           //    finishes the module; 0: CUDA-core kernel + finalisation kernel
+    int32_t module_units;  // work units of the whole module (both sides)
+    int32_t pad[2];
+};
+
+// Progress counters of one module inside the tensor-core kernel (zero before a launch).
+struct FinCounters {
+    int32_t units_done;  // work units whose partial Gram is complete and visible
+    int32_t row_cursor;  // next row of G nobody has claimed yet
+    int32_t rows_done;   // rows whose term of the loss is in the row scratch
+    int32_t pad;
 };
 
 // Per-module pointers for the CUDA-core kernel.
@@ -70,7 +92,7 @@ inline int64_t kblocks_of(int64_t d) { return (d + kKBlock - 1) / kKBlock; }
 // Upper bound on the number of units (hence slots) for any b of one mode: every tile, plus
 // one extra unit per CTA boundary in each of the two splits (tensor-core and CUDA-core).
 inline int64_t max_units(int M, int mode, int n_ctas) {
-    int64_t tiles = (mode == kStacked) ? M : 2 * (int64_t)M;
+    int64_t tiles = mode_is_stacked(mode) ? M : 2 * (int64_t)M;
     return tiles + 2 * (int64_t)n_ctas;
 }
 
@@ -130,11 +152,11 @@ inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t
     plan.mode = mode_of_b(b);
     plan.n_ctas = n_ctas;
     plan.units.clear();
-    plan.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0});
+    plan.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, {0, 0}});
     std::vector<detail::Tile> tc, simt;
     for (int m = 0; m < M; ++m) {
         std::vector<detail::Tile> &dst = tc_ok[m] ? tc : simt;
-        if (plan.mode == kStacked) {
+        if (mode_is_stacked(plan.mode)) {
             dst.push_back({m, 2, kblocks_of(d[m])});
         } else {
             dst.push_back({m, 0, kblocks_of(d[m])});
@@ -151,9 +173,15 @@ inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t
             SideInfo &si = plan.sides[2 * (size_t)u.module + s];
             if (si.n_slots == 0) si.first_slot = u.slot;
             si.n_slots += 1;
-            si.side_off = (plan.mode == kStacked) ? s * 64 * 64 : 0;
+            si.side_off = mode_is_stacked(plan.mode) ? s * pitch * pitch : 0;
             si.pitch = pitch;
         }
+    }
+    for (int m = 0; m < M; ++m) {
+        SideInfo &t = plan.sides[2 * (size_t)m], &r = plan.sides[2 * (size_t)m + 1];
+        const int32_t units = mode_is_stacked(plan.mode) ? t.n_slots : t.n_slots + r.n_slots;
+        t.tensor_core = r.tensor_core = tc_ok[m] ? 1 : 0;
+        t.module_units = r.module_units = units;
     }
 }
 

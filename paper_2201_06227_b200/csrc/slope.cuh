@@ -9,8 +9,8 @@
 namespace egeria {
 
 struct SlopeState {     // per-module arrays (device)
-    double *raw;        // [M][W_cap] ring of raw readings P_i
-    double *plist;      // [M][W_cap] ring of smoothed readings (the last W of pList)
+    double *raw;        // [M][W_cap] the last min(n_evals, W) raw readings P_i, oldest first
+    double *plist;      // [M][W_cap] the last min(n_evals, W) smoothed readings (tail of pList), oldest first
     int32_t *n_evals;   // [M] readings taken so far (== len(pList))
     int32_t *counter;   // [M] consecutive stale evaluations
     int32_t *freeze_eval;  // [M] evaluation index at which the counter reached W, or -1
@@ -68,19 +68,155 @@ __device__ __forceinline__ double plasticity_advance(double *raw, double *plist,
     return slope;
 }
 
+// Smoothing (Eq. 2), window fit and counter update of Algorithm 1 for one new reading, given
+// the module's two windows AFTER the new values are in place.  `val(k)` returns element k of
+// the smoothed window (k = 0 oldest) for the k this lane owns (k = lane, lane + 32, ...).
+template <class F>
+__device__ __forceinline__ double window_slope(int n2, int lane, F val) {
+    if (n2 < 2) return INFINITY;
+    const double xm = 0.5 * (double)(n2 - 1);
+    double sy = 0.0;
+    for (int k = lane; k < n2; k += 32) sy += val(k);
+    const double ym = warp_sum_f64(sy) / (double)n2;
+    double sxy = 0.0, sxx = 0.0;
+    for (int k = lane; k < n2; k += 32) {
+        const double dx = (double)k - xm;
+        sxy += dx * (val(k) - ym);
+        sxx += dx * dx;
+    }
+    sxy = warp_sum_f64(sxy);
+    sxx = warp_sum_f64(sxx);
+    return sxy / sxx;
+}
+
+constexpr int kStepRegs = 4;  // window elements a lane keeps in registers: W <= 128 takes the fast path
+
+// The same fit with the window in registers: this lane holds elements lane + 32 j in y[j].
+__device__ __forceinline__ double window_slope_regs(int n2, int lane, const double (&y)[kStepRegs]) {
+    if (n2 < 2) return INFINITY;
+    const double xm = 0.5 * (double)(n2 - 1);
+    double sy = 0.0;
+#pragma unroll
+    for (int j = 0; j < kStepRegs; ++j)
+        if (lane + 32 * j < n2) sy += y[j];
+    const double ym = warp_sum_f64(sy) / (double)n2;
+    double sxy = 0.0, sxx = 0.0;
+#pragma unroll
+    for (int j = 0; j < kStepRegs; ++j)
+        if (lane + 32 * j < n2) {
+            const double dx = (double)(lane + 32 * j) - xm;
+            sxy += dx * (y[j] - ym);
+            sxx += dx * dx;
+        }
+    sxy = warp_sum_f64(sxy);
+    sxx = warp_sum_f64(sxx);
+    return sxy / sxx;
+}
+
 // One new reading for module m, by one warp: Algorithm 1 on the context's state.
-__device__ __forceinline__ void plasticity_step_module(const SlopeState &st, int m, int W, int signed_test,
-                                                       float reading, double *out_slopes, uint8_t *out_mask,
-                                                       int lane) {
-    int n_evals = st.n_evals[m], counter = st.counter[m], freeze_eval = st.freeze_eval[m];
-    double slope = st.last_slope[m];
+// The two windows are kept oldest-first at fixed addresses, so for W <= 128 every load of the
+// step (counters, both windows, and both windows shifted by one for the case that the oldest
+// entry drops out) is issued at once: one memory round trip, then arithmetic in registers.
+struct StepLoaded {
+    double ra[kStepRegs], rb[kStepRegs], pa[kStepRegs], pb[kStepRegs];
+    double slope, T;
+    int i, counter, freeze_eval;
+};
+
+// Issue every load of one step of module m (nothing here depends on the new reading).
+__device__ __forceinline__ StepLoaded plasticity_step_load(const SlopeState &st, int m, int W, int lane) {
+    StepLoaded L;
+    const double *raw = st.raw + (int64_t)m * st.W_cap, *plist = st.plist + (int64_t)m * st.W_cap;
+    if (W <= 32 * kStepRegs) {
+#pragma unroll
+        for (int j = 0; j < kStepRegs; ++j) {
+            const int k = lane + 32 * j;
+            L.ra[j] = (k < W) ? raw[k] : 0.0;
+            L.pa[j] = (k < W) ? plist[k] : 0.0;
+            L.rb[j] = (k + 1 < W) ? raw[k + 1] : 0.0;
+            L.pb[j] = (k + 1 < W) ? plist[k + 1] : 0.0;
+        }
+    }
+    L.i = st.n_evals[m];  // readings taken before this one == index of this evaluation
+    L.counter = st.counter[m];
+    L.freeze_eval = st.freeze_eval[m];
+    L.slope = st.last_slope[m];
+    L.T = (double)st.T[m];
+    return L;
+}
+
+__device__ __forceinline__ void plasticity_step_apply(const SlopeState &st, StepLoaded &L, int m, int W,
+                                                      int signed_test, float reading, double *out_slopes,
+                                                      uint8_t *out_mask, int lane) {
+    double *raw = st.raw + (int64_t)m * st.W_cap, *plist = st.plist + (int64_t)m * st.W_cap;
+    const bool fast = (W <= 32 * kStepRegs);
+    double(&ra)[kStepRegs] = L.ra, (&rb)[kStepRegs] = L.rb, (&pa)[kStepRegs] = L.pa, (&pb)[kStepRegs] = L.pb;
+    const int i = L.i;
+    int counter = L.counter, freeze_eval = L.freeze_eval;
+    double slope = L.slope;
+    const double T = L.T;
     __syncwarp();
     if (counter < W) {
-        slope = plasticity_advance(st.raw + (int64_t)m * st.W_cap, st.plist + (int64_t)m * st.W_cap, n_evals,
-                                   counter, freeze_eval, (double)reading, W, (double)st.T[m], signed_test != 0,
-                                   lane);
+        const int len = (i < W) ? i : W;       // entries in the windows now
+        const bool drop = (len == W);          // the oldest entry leaves
+        const int n = drop ? W : len + 1;      // entries after this reading: min(i + 1, W)
+        const double P = (double)reading;
+        if (fast) {
+            // windows after the update, in registers: element k = lane + 32 j
+#pragma unroll
+            for (int j = 0; j < kStepRegs; ++j) {
+                const int k = lane + 32 * j;
+                ra[j] = (k == n - 1) ? P : (drop ? rb[j] : ra[j]);
+                pa[j] = drop ? pb[j] : pa[j];
+            }
+            double s = 0.0;  // Eq. 2: mean of the last min(i + 1, W) raw readings
+#pragma unroll
+            for (int j = 0; j < kStepRegs; ++j)
+                if (lane + 32 * j < n) s += ra[j];
+            const double pbar = warp_sum_f64(s) / (double)n;
+#pragma unroll
+            for (int j = 0; j < kStepRegs; ++j)
+                if (lane + 32 * j == n - 1) pa[j] = pbar;
+            slope = window_slope_regs(n, lane, pa);
+#pragma unroll
+            for (int j = 0; j < kStepRegs; ++j) {
+                const int k = lane + 32 * j;
+                if (k < n && (drop || k == n - 1)) {
+                    raw[k] = ra[j];
+                    plist[k] = pa[j];
+                }
+            }
+        } else {
+            if (drop) {  // shift both windows left by one, 32 entries at a time
+                for (int k0 = 0; k0 < W - 1; k0 += 32) {
+                    const int k = k0 + lane;
+                    double r = 0.0, q = 0.0;
+                    if (k < W - 1) {
+                        r = raw[k + 1];
+                        q = plist[k + 1];
+                    }
+                    __syncwarp();
+                    if (k < W - 1) {
+                        raw[k] = r;
+                        plist[k] = q;
+                    }
+                    __syncwarp();
+                }
+            }
+            if (lane == 0) raw[n - 1] = P;
+            __syncwarp();
+            double s = 0.0;
+            for (int k = lane; k < n; k += 32) s += raw[k];
+            const double pbar = warp_sum_f64(s) / (double)n;
+            if (lane == 0) plist[n - 1] = pbar;
+            __syncwarp();
+            slope = window_slope(n, lane, [&](int k) { return plist[k]; });
+        }
+        const bool stale = signed_test ? (slope < T) : (fabs(slope) < T);  // NaN compares false
+        counter = stale ? counter + 1 : 0;
+        if (counter >= W && freeze_eval < 0) freeze_eval = i;
         if (lane == 0) {
-            st.n_evals[m] = n_evals;
+            st.n_evals[m] = i + 1;
             st.counter[m] = counter;
             st.freeze_eval[m] = freeze_eval;
             st.last_slope[m] = slope;
@@ -90,6 +226,13 @@ __device__ __forceinline__ void plasticity_step_module(const SlopeState &st, int
         if (out_slopes) out_slopes[m] = slope;
         if (out_mask) out_mask[m] = (counter >= W) ? 1 : 0;
     }
+}
+
+__device__ __forceinline__ void plasticity_step_module(const SlopeState &st, int m, int W, int signed_test,
+                                                       float reading, double *out_slopes, uint8_t *out_mask,
+                                                       int lane) {
+    StepLoaded L = plasticity_step_load(st, m, W, lane);
+    plasticity_step_apply(st, L, m, W, signed_test, reading, out_slopes, out_mask, lane);
 }
 
 // One new reading per module.  grid = M warps (one 32-thread block each).
