@@ -14,7 +14,8 @@
  *   - "device" pointers are CUDA device memory owned by the caller; "host"
  *     pointers are ordinary host memory.  The library allocates no device
  *     memory: all scratch lives in the caller's workspace (see
- *     egeria_workspace_bytes).
+ *     egeria_workspace_bytes).  (A context also holds a few KB of pinned host
+ *     memory unless EGERIA_FLAG_EQUAL_SPLIT is given.)
  *   - cuda_stream is a cudaStream_t passed as void* (NULL = default stream).
  *     Calls enqueue work on it and return without synchronising, unless the
  *     call's comment says otherwise.
@@ -59,7 +60,19 @@ enum {
     EGERIA_FLAG_HOST_STAGING = 8u,
     /* Record a CUDA event before and after the Gram kernel(s) of every
      * egeria_sp_loss_batch call, for egeria_gram_kernel_time. */
-    EGERIA_FLAG_TIME_GRAM = 16u
+    EGERIA_FLAG_TIME_GRAM = 16u,
+    /* Always cut the work into equal shares.  Without this flag the first
+     * evaluations of a context that keep every SM busy report how fast each
+     * thread block streamed, and the shares then follow those rates (the SMs of
+     * a B200 do not all get the same share of HBM bandwidth, and the placement of
+     * thread blocks on SMs repeats from launch to launch): three evaluations are
+     * measured, the shares are set, and this is repeated twice under the new
+     * shares; after the ninth such evaluation the shares stay.  The shares decide
+     * how the fp32 partial sums are grouped, so with the adaptive split the
+     * low-order bits of a loss can differ between evaluations across a change of
+     * shares and from run to run; with this flag every evaluation of the same
+     * inputs gives the same bits. */
+    EGERIA_FLAG_EQUAL_SPLIT = 32u
 };
 
 #define EGERIA_MAX_B 256          /* largest supported mini-batch size */
@@ -159,6 +172,13 @@ egeria_status egeria_plasticity_reset(egeria_ctx *ctx, void *cuda_stream, int ha
 /* Current window of the context (changes only through egeria_plasticity_reset). */
 int egeria_plasticity_window(const egeria_ctx *ctx);
 
+/* The per-thread-block shares of the adaptive split (see EGERIA_FLAG_EQUAL_SPLIT).
+ * Copies up to max_weights of them to out_weights (host, may be NULL; 1.0 = the
+ * equal share) and returns how many thread blocks the split is over once measured
+ * rates are in use, 0 while the split is still (or for good) the equal one, -1 for
+ * a NULL context.  Never waits for the device. */
+int egeria_split_weights(egeria_ctx *ctx, float *out_weights, int max_weights);
+
 /* Test hook: copy the row-normalised similarity matrices of one module, as
  * left by the last egeria_sp_loss_batch, to device float [b, b] buffers.
  * Needs EGERIA_FLAG_KEEP_GRAMS. */
@@ -171,6 +191,12 @@ egeria_status egeria_debug_dump_gram(egeria_ctx *ctx, void *cuda_stream, int mod
  * n_units.  n_ctas is the number of persistent CTAs to split over. */
 egeria_status egeria_debug_plan(int M, const int64_t *d, int b, int n_ctas, int32_t *out_units,
                                 int max_units, int *n_units);
+
+/* Test hook: the same with one weight per CTA (host float [n_ctas], positive;
+ * NULL = equal shares): CTA c's share of the blocks is weights[c] / sum. */
+egeria_status egeria_debug_plan_weighted(int M, const int64_t *d, int b, int n_ctas,
+                                         const float *weights, int32_t *out_units, int max_units,
+                                         int *n_units);
 
 /* Synchronise the stream of the last call and report the device status word:
  * EGERIA_OK, or EGERIA_ERR_TIMEOUT if a bounded wait inside a kernel ran out

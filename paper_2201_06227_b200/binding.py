@@ -18,6 +18,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libegeria.so"
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 FLAG_SIGNED_SLOPE, FLAG_FORCE_SIMT, FLAG_KEEP_GRAMS, FLAG_HOST_STAGING, FLAG_TIME_GRAM = 1, 2, 4, 8, 16
+FLAG_EQUAL_SPLIT = 32
 MAX_B = 256
 WORKSPACE_ALIGN = 1024
 
@@ -25,9 +26,10 @@ EXPORTS = [
     "egeria_workspace_bytes", "egeria_plasticity_create", "egeria_plasticity_destroy",
     "egeria_sp_loss_batch", "egeria_sp_loss_batch_host", "egeria_plasticity_step",
     "egeria_plasticity_replay", "egeria_plasticity_reset", "egeria_plasticity_window",
-    "egeria_debug_dump_gram", "egeria_debug_plan", "egeria_device_status", "egeria_launch_count",
+    "egeria_debug_dump_gram", "egeria_debug_plan", "egeria_debug_plan_weighted", "egeria_device_status",
+    "egeria_launch_count",
     "egeria_gram_kernel_time", "egeria_sp_loss_static", "egeria_plasticity_evaluate",
-    "egeria_status_string",
+    "egeria_split_weights", "egeria_status_string",
 ]
 
 
@@ -66,6 +68,10 @@ def lib() -> ctypes.CDLL:
     L.egeria_debug_dump_gram.argtypes = [vp, vp, ctypes.c_int, vp, vp]
     L.egeria_debug_plan.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int,
                                     ctypes.POINTER(ctypes.c_int32), ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+    L.egeria_debug_plan_weighted.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int,
+                                             ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32),
+                                             ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+    L.egeria_split_weights.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.c_int]
     L.egeria_device_status.argtypes = [vp]
     L.egeria_gram_kernel_time.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
     L.egeria_sp_loss_static.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_int64, vp]
@@ -110,6 +116,23 @@ def egeria_debug_plan(d: Sequence[int], b: int, n_ctas: int) -> np.ndarray:
     st = lib().egeria_debug_plan(M, _i64(d), int(b), int(n_ctas),
                                  out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), cap, ctypes.byref(n))
     _check(st, "egeria_debug_plan")
+    return out[: n.value].copy()
+
+
+def egeria_debug_plan_weighted(d: Sequence[int], b: int, n_ctas: int, weights) -> np.ndarray:
+    """The same split with one weight per CTA (None = equal shares)."""
+    M = len(d)
+    cap = 2 * M + n_ctas + 8
+    out = np.zeros((cap, 5), dtype=np.int32)
+    n = ctypes.c_int(0)
+    wp = None
+    if weights is not None:
+        w = np.ascontiguousarray(weights, dtype=np.float32)
+        assert w.shape == (n_ctas,)
+        wp = w.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
+    st = lib().egeria_debug_plan_weighted(M, _i64(d), int(b), int(n_ctas), wp,
+                                          out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), cap, ctypes.byref(n))
+    _check(st, "egeria_debug_plan_weighted")
     return out[: n.value].copy()
 
 
@@ -286,6 +309,12 @@ class Context:
         ms, n = ctypes.c_double(), ctypes.c_int64()
         _check(lib().egeria_gram_kernel_time(self._h, ctypes.byref(ms), ctypes.byref(n)), "egeria_gram_kernel_time")
         return ms.value, n.value
+
+    def egeria_split_weights(self):
+        """(n, weights): n > 0 once the split follows measured streaming rates."""
+        w = np.ones(256, dtype=np.float32)
+        n = int(lib().egeria_split_weights(self._h, w.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), 256))
+        return n, w[: max(n, 0)].copy()
 
     def egeria_launch_count(self) -> int:
         return int(lib().egeria_launch_count(self._h))

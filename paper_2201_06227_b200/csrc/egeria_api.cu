@@ -20,12 +20,14 @@ namespace egeria {
 constexpr int kMaxCtas = 160;  // sizing bound for the work split (a B200 has 148 SMs)
 constexpr int kMaxW = 2048;    // replay keeps 2 * W doubles in shared memory
 constexpr int kPlanSlots = 16; // device-side plans kept, keyed by (b, activation pointers)
+constexpr int kCalibLaunches = 3;  // launches whose per-CTA streaming rates set the split weights
+constexpr int kCalibRounds = 3;    // times the weights are re-measured under the split they produced
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Offsets of everything the library keeps in the caller's workspace.
 struct Layout {
-    size_t status, rowloss, tickets, fin_ctr, T, raw, plist, n_evals, counter, freeze_eval, last_slope, losses, keep,
+    size_t status, cta_log, rowloss, tickets, fin_ctr, T, raw, plist, n_evals, counter, freeze_eval, last_slope, losses, keep,
         slots, staging, total;
     size_t slot_bytes_cap;  // bytes reserved for partial slots
     // Device-side plans (tensor maps, pointers, unit table, per-CTA ranges, slot ranges): kPlanSlots
@@ -51,6 +53,7 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
         return o;
     };
     L.status = take(256);
+    L.cta_log = take(kMaxCtas * sizeof(CtaLog));
     {
         size_t saved = off;
         off = 0;
@@ -129,6 +132,7 @@ struct egeria_ctx {
     // device-side plans, least recently used one is replaced
     struct PlanEntry {
         int b = -1;
+        int weights_version = 0;
         std::vector<const void *> At, Ar;
         Plan plan;
         uint64_t last_use = 0;
@@ -142,6 +146,15 @@ struct egeria_ctx {
     cudaStream_t last_stream = nullptr;
     int64_t launches = 0;
     uint32_t tc_launches = 0;  // selects the set of progress counters the next tensor-core launch uses
+    // Split weights: one per CTA, from the streaming rates the CTAs report (SMs do not all get
+    // the same share of HBM bandwidth; the CTA -> SM placement repeats from launch to launch).
+    std::vector<float> weights;
+    int weights_version = 0;
+    bool calibrated = false;   // no more measuring
+    int calib_round = 0;
+    int calib_enqueued = 0;
+    uint32_t calib_serial[kCalibLaunches] = {};
+    CtaLog *host_log = nullptr;  // pinned, kCalibLaunches x kMaxCtas
     std::vector<void *> staging_t, staging_r;
     // EGERIA_FLAG_TIME_GRAM: event pairs around the Gram kernel launches since the last query
     std::vector<cudaEvent_t> ev_pool;
@@ -164,6 +177,10 @@ struct egeria_ctx {
         return st;
     }
 };
+
+namespace egeria {
+static void poll_calibration(egeria_ctx *ctx);
+}
 
 #define EG_CUDA(call)                                   \
     do {                                                \
@@ -195,13 +212,18 @@ size_t egeria_workspace_bytes(int M, const int64_t *d, int b_max, int W, uint32_
 
 egeria_status egeria_debug_plan(int M, const int64_t *d, int b, int n_ctas, int32_t *out_units, int max_units_out,
                                 int *n_units) {
+    return egeria_debug_plan_weighted(M, d, b, n_ctas, nullptr, out_units, max_units_out, n_units);
+}
+
+egeria_status egeria_debug_plan_weighted(int M, const int64_t *d, int b, int n_ctas, const float *weights,
+                                         int32_t *out_units, int max_units_out, int *n_units) {
     if (!out_units || !n_units || n_ctas < 1 || max_units_out < 0) return EGERIA_ERR_INVALID_ARG;
     egeria_status s = check_shapes(M, d, b, 1);
     if (s != EGERIA_OK) return s;
     std::vector<uint8_t> tc_ok(M);
     for (int m = 0; m < M; ++m) tc_ok[m] = (d[m] % 8 == 0);
     Plan plan;
-    build_plan(M, d, b, n_ctas, tc_ok.data(), plan);
+    build_plan(M, d, b, n_ctas, tc_ok.data(), plan, weights);
     *n_units = (int)plan.units.size();
     for (int i = 0; i < (int)plan.units.size() && i < max_units_out; ++i) {
         const Unit &u = plan.units[i];
@@ -267,7 +289,18 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
 
     std::vector<float> Th(M);
     for (int m = 0; m < M; ++m) Th[m] = T ? T[m] : T_all;
+    ctx->weights.assign(ctx->n_ctas, 1.0f);
+    if (!(flags & EGERIA_FLAG_EQUAL_SPLIT)) {
+        void *hp = nullptr;
+        if (cudaHostAlloc(&hp, sizeof(CtaLog) * kCalibLaunches * kMaxCtas, cudaHostAllocDefault) == cudaSuccess) {
+            memset(hp, 0, sizeof(CtaLog) * kCalibLaunches * kMaxCtas);
+            ctx->host_log = static_cast<CtaLog *>(hp);
+        } else {
+            (void)cudaGetLastError();  // no pinned memory: keep the equal split
+        }
+    }
     cudaError_t e = cudaMemset(ctx->ws + L.status, 0, 256);
+    if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.cta_log, 0, kMaxCtas * sizeof(CtaLog));
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.tickets, 0, (size_t)M * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.fin_ctr, 0, (size_t)2 * M * sizeof(FinCounters));
     if (e == cudaSuccess) e = cudaMemcpy(ctx->ws + L.T, Th.data(), (size_t)M * sizeof(float), cudaMemcpyHostToDevice);
@@ -277,6 +310,7 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
         e = cudaDeviceSynchronize();
     }
     if (e != cudaSuccess) {
+        if (ctx->host_log) cudaFreeHost(ctx->host_log);
         delete ctx;
         return EGERIA_ERR_CUDA;
     }
@@ -287,11 +321,20 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
 egeria_status egeria_plasticity_destroy(egeria_ctx *ctx) {
     if (!ctx) return EGERIA_ERR_INVALID_ARG;
     for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+    if (ctx->host_log) cudaFreeHost(ctx->host_log);
     delete ctx;
     return EGERIA_OK;
 }
 
 int egeria_plasticity_window(const egeria_ctx *ctx) { return ctx ? ctx->W : 0; }
+
+int egeria_split_weights(egeria_ctx *ctx, float *out_weights, int max_weights) {
+    if (!ctx) return -1;
+    poll_calibration(ctx);
+    if (out_weights)
+        for (int c = 0; c < ctx->n_ctas && c < max_weights; ++c) out_weights[c] = ctx->weights[c];
+    return (ctx->weights_version > 0) ? ctx->n_ctas : 0;
+}
 int64_t egeria_launch_count(const egeria_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
 }  // extern "C"
@@ -309,6 +352,41 @@ static egeria_status encode_map(egeria_ctx *ctx, CUtensorMap *tm, const void *ba
     return r == CUDA_SUCCESS ? EGERIA_OK : EGERIA_ERR_CUDA;
 }
 
+// If the logs of all calibration launches have arrived on the host, turn them into split
+// weights: CTA c gets work in proportion to the blocks per nanosecond it managed.  Never waits.
+static void poll_calibration(egeria_ctx *ctx) {
+    if (ctx->calibrated || !ctx->host_log || ctx->calib_enqueued < kCalibLaunches) return;
+    const int n = ctx->n_ctas;
+    std::vector<double> rate(n, 0.0);
+    for (int k = 0; k < kCalibLaunches; ++k) {
+        const volatile CtaLog *log = ctx->host_log + (size_t)k * kMaxCtas;
+        for (int c = 0; c < n; ++c) {
+            if (log[c].serial != ctx->calib_serial[k]) return;  // this copy has not landed yet
+            const uint32_t ns = log[c].duration_ns, blocks = log[c].blocks;
+            if (ns == 0 || blocks == 0) {  // a launch that gave up: stay with the equal split
+                ctx->calibrated = true;
+                return;
+            }
+            rate[c] += (double)blocks / (double)ns;
+        }
+    }
+    double mean = 0.0;
+    for (int c = 0; c < n; ++c) mean += rate[c];
+    mean /= n;
+    for (int c = 0; c < n; ++c) {
+        double w = rate[c] / mean;
+        if (w < 0.5) w = 0.5;
+        if (w > 2.0) w = 2.0;
+        ctx->weights[c] = (float)w;
+    }
+    ctx->weights_version++;  // plans made with the previous shares are rebuilt on their next use
+    // Under the equal split the fast CTAs finish early and leave the slow ones more bandwidth, which
+    // flatters the slow ones: measure again under the new shares, a few times.
+    ctx->calib_round++;
+    ctx->calib_enqueued = 0;
+    if (ctx->calib_round >= kCalibRounds) ctx->calibrated = true;
+}
+
 // Select (or build and upload) the device-side plan for this (b, pointers).
 static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const void *const *At, const void *const *Ar,
                                   int b) {
@@ -317,7 +395,8 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
     int lru = 0;
     for (int i = 0; i < kPlanSlots; ++i) {
         egeria_ctx::PlanEntry &e = ctx->plans[i];
-        if (e.b == b && memcmp(e.At.data(), At, pbytes) == 0 && memcmp(e.Ar.data(), Ar, pbytes) == 0) {
+        if (e.b == b && e.weights_version == ctx->weights_version && memcmp(e.At.data(), At, pbytes) == 0 &&
+            memcmp(e.Ar.data(), Ar, pbytes) == 0) {
             e.last_use = ++ctx->use_clock;
             ctx->cur = i;
             ctx->plan_b = b;
@@ -334,7 +413,8 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
                              (reinterpret_cast<uintptr_t>(Ar[m]) % 16 == 0) && (ctx->d[m] % 8 == 0);
         tc_ok[m] = aligned && !(ctx->flags & EGERIA_FLAG_FORCE_SIMT);
     }
-    build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), e.plan);
+    build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), e.plan,
+               ctx->weights_version > 0 ? ctx->weights.data() : nullptr);
     const Plan &P = e.plan;
     const Layout &L = ctx->L;
     if ((size_t)P.units.size() * slot_floats_of_mode(P.mode) * sizeof(float) > L.slot_bytes_cap ||
@@ -360,6 +440,7 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
     // One copy from pageable memory: the runtime stages it before returning, so `pack` may be reused.
     EG_CUDA(cudaMemcpyAsync(ctx->plan_region(lru), img, L.plan_stride, cudaMemcpyHostToDevice, stream));
     e.b = b;
+    e.weights_version = ctx->weights_version;
     e.At.assign(At, At + M);
     e.Ar.assign(Ar, Ar + M);
     e.last_use = ++ctx->use_clock;
@@ -435,6 +516,7 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
     ctx->last_stream = stream;
     egeria_status s = set_attrs(ctx);
     if (s != EGERIA_OK) return s;
+    poll_calibration(ctx);
     s = refresh_plan(ctx, stream, At, Ar, b);
     if (s != EGERIA_OK) return s;
 
@@ -483,7 +565,18 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         tp.ctr_next = sets + (size_t)(set ^ 1u) * ctx->M;
         tp.M = ctx->M;
         tp.fin = fc;
+        const bool log_it = !ctx->calibrated && ctx->host_log && ctx->calib_enqueued < kCalibLaunches &&
+                            P.all_ctas_busy_tc;
+        tp.log = log_it ? ctx->at<CtaLog>(L.cta_log) : nullptr;
+        tp.serial = ctx->tc_launches + 1;
         if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
+        if (log_it) {
+            const int k = ctx->calib_enqueued;
+            EG_CUDA(cudaMemcpyAsync(ctx->host_log + (size_t)k * kMaxCtas, tp.log, (size_t)ctx->n_ctas * sizeof(CtaLog),
+                                    cudaMemcpyDeviceToHost, stream));
+            ctx->calib_serial[k] = tp.serial;
+            ctx->calib_enqueued = k + 1;
+        }
         ctx->tc_launches++;
         ctx->launches++;
     }
@@ -791,6 +884,8 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         tp.status = ticket + 1;
         tp.ctr = reinterpret_cast<FinCounters *>(ticket + 2);
         tp.ctr_next = tp.ctr + 1;
+        tp.log = nullptr;
+        tp.serial = 0;
         tp.M = 1;
         tp.fin = fc;
         if (launch_tc_mode(P.mode, kStaticCtas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;

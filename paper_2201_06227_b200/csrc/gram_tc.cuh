@@ -71,6 +71,8 @@ struct TcParams {
     int32_t *status;           // device status word
     FinCounters *ctr;          // [M] progress counters of this launch (all zero at launch)
     FinCounters *ctr_next;     // [M] the set the next launch will use: cleared here
+    CtaLog *log;               // [gridDim.x] what each CTA reports about this launch, or nullptr
+    uint32_t serial;           // tag of this launch in the log
     int32_t M;
     FinCommon fin;             // slots, sides, b, outputs, freezing-rule state
 };
@@ -165,24 +167,28 @@ __device__ __forceinline__ bool next_chunk(int &k, int q, int lane, int b, float
     return false;
 }
 
-// One warp: wait until `total` units of the module are complete, to help finish it.  The
-// wait is a courtesy, not a dependency: the CTA that delivers the module's last unit finishes
-// every row nobody else has claimed, so a warp that stops waiting (false) loses nothing but
-// parallelism.  That keeps the kernel correct when not all of its CTAs are resident together.
+// All epilogue warps: wait until `total` units of the module are complete, to help finish it.
+// One lane of the CTA polls (a counter that every waiting warp of every CTA polled would be a
+// hot spot); the others wait for it at a barrier.  The wait is a courtesy, not a dependency:
+// the CTA that delivers the module's last unit finishes every row nobody else has claimed, so a
+// CTA that stops waiting (false) loses nothing but parallelism.  That keeps the kernel correct
+// when not all of its CTAs are resident together.
 __device__ __forceinline__ bool wait_units_done(const int32_t *units_done, int total, volatile int *abort_flag,
-                                                int lane) {
-    int ok = 1;
-    if (lane == 0) {
+                                                volatile int *verdict, bool poller) {
+    if (poller) {
+        int ok = 1;
         const uint64_t t0 = ptx::globaltimer_ns();
         while (ld_acquire(units_done) < total) {
             if (*abort_flag || ptx::globaltimer_ns() - t0 > kHelpWaitNs) {
                 ok = 0;
                 break;
             }
-            __nanosleep(40);
+            __nanosleep(100);
         }
+        *verdict = ok;
     }
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+    epi_bar_sync();
+    return *verdict != 0;
 }
 
 // One warp: take rows of module m from its cursor until none is left.  The claim of the next
@@ -235,6 +241,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     volatile uint32_t *tmem_holder =
         reinterpret_cast<volatile uint32_t *>(bars + 2 * Cfg::kStages + 2 * Cfg::kAccStages);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+    volatile int *wait_verdict = reinterpret_cast<volatile int *>(tmem_holder + 2);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -336,6 +343,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             constexpr uint32_t idesc64 = ptx::make_idesc_bf16_f32(128, 64);
             constexpr uint32_t idesc128 = ptx::make_idesc_bf16_f32(128, 128);
             constexpr uint32_t idesc256 = ptx::make_idesc_bf16_f32(128, 256);
+            const uint64_t t_entry = ptx::globaltimer_ns();
+            uint32_t blocks_done = 0;
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
             bool any_mma = false;
@@ -384,11 +393,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                     }
                 }
                 if (!ok) break;
+                blocks_done += (uint32_t)u.nkb;
                 ptx::mma_commit(accfull0 + 8 * acc);  // accumulator complete
                 if (++acc == Cfg::kAccStages) {
                     acc = 0;
                     acc_phase ^= 1u;
                 }
+            }
+            if (p.log) {
+                CtaLog e;
+                e.serial = p.serial;
+                e.duration_ns = (uint32_t)(ptx::globaltimer_ns() - t_entry);
+                e.blocks = ok ? blocks_done : 0u;
+                e.pad = 0;
+                p.log[blockIdx.x] = e;
             }
             if (!ok && any_mma) {
                 // Gave up: give the MMAs already issued time to finish before TMEM is freed
@@ -473,11 +491,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 if (m == prev_m) continue;
                 prev_m = m;
                 const int total = p.fin.sides[2 * m].module_units;
-                int done = 0;
-                if (lane == 0) done = detail::ld_acquire(&p.ctr[m].units_done);
-                bool ready = (__shfl_sync(0xffffffffu, done, 0) >= total);
-                if (!ready && m == m_last)
-                    ready = detail::wait_units_done(&p.ctr[m].units_done, total, abort_flag, lane);
+                bool ready;
+                if (m == m_last) {
+                    // every warp of the CTA gets here (same units, same order): wait together
+                    ready = detail::wait_units_done(&p.ctr[m].units_done, total, abort_flag, wait_verdict, epi_leader);
+                } else {
+                    int done = 0;
+                    if (lane == 0) done = detail::ld_acquire(&p.ctr[m].units_done);
+                    ready = (__shfl_sync(0xffffffffu, done, 0) >= total);
+                }
                 if (ready) {
                     __threadfence();
                     detail::finish_module_rows<Cfg::kNC>(p, m, lane, stage);

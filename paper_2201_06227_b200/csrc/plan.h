@@ -62,12 +62,24 @@ struct SideInfo {
     int32_t pad[2];
 };
 
-// Progress counters of one module inside the tensor-core kernel (zero before a launch).
+// What one CTA of the tensor-core kernel reports about a launch: how long it streamed and how
+// much.  The host turns the blocks-per-nanosecond of a few launches into the split weights.
+struct CtaLog {
+    uint32_t serial;       // launch this entry belongs to
+    uint32_t duration_ns;  // kernel entry to last MMA issued
+    uint32_t blocks;       // 64-element blocks it processed
+    uint32_t pad;
+};
+
+// Progress counters of one module inside the tensor-core kernel (zero before a launch).  Each
+// is polled or bumped by many CTAs at the end of a launch, so each has a 128-byte line of its own.
 struct FinCounters {
     int32_t units_done;  // work units whose partial Gram is complete and visible
+    int32_t pad0[31];
     int32_t row_cursor;  // next row of G nobody has claimed yet
+    int32_t pad1[31];
     int32_t rows_done;   // rows whose term of the loss is in the row scratch
-    int32_t pad;
+    int32_t pad2[31];
 };
 
 // Per-module pointers for the CUDA-core kernel.
@@ -82,6 +94,7 @@ struct Plan {
     int n_ctas = 0;
     std::vector<Unit> units;        // tensor-core units first, then CUDA-core units
     int n_units_tc = 0;
+    bool all_ctas_busy_tc = false;        // every CTA of the tensor-core kernel has at least one unit
     std::vector<int32_t> cta_begin_tc;    // [n_ctas + 1] into units[0 .. n_units_tc)
     std::vector<int32_t> cta_begin_simt;  // [n_ctas + 1] into units[n_units_tc ..), relative to 0
     std::vector<SideInfo> sides;    // [2 * M]
@@ -109,8 +122,11 @@ struct Tile {
 // and only adds partial slots for the finaliser to read.
 constexpr int kMinBlocksPerCta = 8;
 
+// `weights` (optional, [n_ctas], positive): CTA c's range is proportional to weights[c] instead
+// of equal -- the caller's estimate of how fast each CTA streams.  Ignored when fewer CTAs than
+// n_ctas are used.
 inline void split_tiles(const std::vector<Tile> &tiles, int n_ctas, int slot0, std::vector<Unit> &units,
-                        std::vector<int32_t> &cta_begin) {
+                        std::vector<int32_t> &cta_begin, const float *weights = nullptr) {
     int64_t total = 0;
     for (const Tile &t : tiles) total += t.nkb;
     cta_begin.assign(n_ctas + 1, 0);
@@ -120,10 +136,31 @@ inline void split_tiles(const std::vector<Tile> &tiles, int n_ctas, int slot0, s
     int64_t used = (total + kMinBlocksPerCta - 1) / kMinBlocksPerCta;
     if (used > n_ctas) used = n_ctas;
     if (used < 1) used = 1;
+    // cut[c] .. cut[c + 1]: the blocks of CTA c
+    std::vector<int64_t> cut(used + 1);
+    bool weighted = (weights != nullptr && used == n_ctas);
+    double wsum = 0.0;
+    if (weighted)
+        for (int c = 0; c < n_ctas; ++c) {
+            if (!(weights[c] > 0.f) || weights[c] > 1e30f) weighted = false;  // also rejects NaN
+            wsum += weights[c];
+        }
+    double acc = 0.0;
+    for (int64_t c = 0; c <= used; ++c) {
+        if (weighted) {
+            int64_t v = (c == used) ? total : (int64_t)((double)total * (acc / wsum) + 0.5);
+            if (c > 0 && v < cut[c - 1]) v = cut[c - 1];
+            if (v > total) v = total;
+            cut[c] = v;
+            if (c < used) acc += weights[c];
+        } else {
+            cut[c] = total * c / used;
+        }
+    }
     for (int c = 0; c < n_ctas; ++c) {
         cta_begin[c] = (int)units.size() - base;
         if (c >= used) continue;  // idle CTA: empty range
-        const int64_t lo = total * c / used, hi = total * (c + 1) / used;
+        const int64_t lo = cut[c], hi = cut[c + 1];
         int64_t pos = lo;
         while (pos < hi) {
             while (ti < tiles.size() && tile_start + tiles[ti].nkb <= pos) {
@@ -147,8 +184,10 @@ inline void split_tiles(const std::vector<Tile> &tiles, int n_ctas, int slot0, s
 }
 }  // namespace detail
 
-// tc_ok[m] != 0: module m may use the TMA + tcgen05 kernel.
-inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t *tc_ok, Plan &plan) {
+// tc_ok[m] != 0: module m may use the TMA + tcgen05 kernel.  weights: see split_tiles (applies to
+// the tensor-core split only).
+inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t *tc_ok, Plan &plan,
+                       const float *weights = nullptr) {
     plan.mode = mode_of_b(b);
     plan.n_ctas = n_ctas;
     plan.units.clear();
@@ -163,8 +202,11 @@ inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t
             dst.push_back({m, 1, kblocks_of(d[m])});
         }
     }
-    detail::split_tiles(tc, n_ctas, 0, plan.units, plan.cta_begin_tc);
+    detail::split_tiles(tc, n_ctas, 0, plan.units, plan.cta_begin_tc, weights);
     plan.n_units_tc = (int)plan.units.size();
+    plan.all_ctas_busy_tc = true;
+    for (int c = 0; c < n_ctas; ++c)
+        if (plan.cta_begin_tc[c + 1] == plan.cta_begin_tc[c]) plan.all_ctas_busy_tc = false;
     detail::split_tiles(simt, n_ctas, plan.n_units_tc, plan.units, plan.cta_begin_simt);
     const int pitch = pitch_of_mode(plan.mode);
     for (const Unit &u : plan.units) {

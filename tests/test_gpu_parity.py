@@ -217,7 +217,7 @@ def test_host_entry_matches_device_entry():
         t, r = wl.make_pair(b, d, "relu", 0.2, seed=40 + m, device="cpu")
         at.append(t.pin_memory())
         ar.append(r.pin_memory())
-    ctx = eg.Context(ds, b, 5, 1e-3, eg.FLAG_HOST_STAGING, device=DEV)
+    ctx = eg.Context(ds, b, 5, 1e-3, eg.FLAG_HOST_STAGING | eg.FLAG_EQUAL_SPLIT, device=DEV)
     host = ctx.egeria_sp_loss_batch_host(at, ar).numpy().copy()
     dev = ctx.egeria_sp_loss_batch([t.to(DEV) for t in at], [r.to(DEV) for r in ar]).cpu().numpy()
     assert host.tobytes() == dev.tobytes()
@@ -330,8 +330,8 @@ def test_step_matches_replay_and_oracle(signed):
 def test_evaluate_equals_separate_calls():
     """egeria_plasticity_evaluate = egeria_sp_loss_batch + egeria_plasticity_step, bit for bit."""
     ds, b, W, T = [4096, 520, 1001, 8192], 72, 3, float(np.float32(5e-4))
-    fused = eg.Context(ds, b, W, T, device=DEV)
-    split = eg.Context(ds, b, W, T, device=DEV)
+    fused = eg.Context(ds, b, W, T, eg.FLAG_EQUAL_SPLIT, device=DEV)
+    split = eg.Context(ds, b, W, T, eg.FLAG_EQUAL_SPLIT, device=DEV)
     for k in range(8):
         at, ar = [], []
         for m, d in enumerate(ds):
@@ -349,6 +349,59 @@ def test_evaluate_equals_separate_calls():
     fused.check_device_status()
     fused.close()
     split.close()
+
+
+@pytest.mark.parametrize("b,ds", [(64, [401408, 200704, 100352, 802816]), (256, [131072] * 5), (128, [65536] * 7)])
+def test_adaptive_split_keeps_the_result(b, ds):
+    """After three evaluations that fill every SM the shares follow the measured streaming
+    rates; the losses stay within the tolerance of the equal split's, and with
+    EGERIA_FLAG_EQUAL_SPLIT every evaluation gives the same bits."""
+    at, ar = [], []
+    for m, d in enumerate(ds):
+        t, r = wl.make_pair(b, d, "relu", 0.05 + 0.05 * m, seed=7000 + m, device=DEV)
+        at.append(t)
+        ar.append(r)
+    fixed = eg.Context(ds, b, 5, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
+    ref = [fixed.egeria_sp_loss_batch(at, ar).cpu().numpy().copy() for _ in range(3)]
+    assert ref[0].tobytes() == ref[1].tobytes() == ref[2].tobytes()
+    assert fixed.egeria_split_weights()[0] == 0
+    fixed.close()
+    ctx = eg.Context(ds, b, 5, 1e-3, device=DEV)
+    outs = []
+    for k in range(14):
+        outs.append(ctx.egeria_sp_loss_batch(at, ar).cpu().numpy().copy())   # .cpu() waits: the logs have landed
+    n, w = ctx.egeria_split_weights()
+    assert n > 0 and len(w) == n
+    assert np.all(w >= 0.5) and np.all(w <= 2.0) and abs(float(w.mean()) - 1.0) < 0.05
+    assert outs[0].tobytes() == ref[0].tobytes()          # the first evaluations use the equal split
+    for o in outs:
+        assert_loss_close(o, ref[0].astype(np.float64), "adaptive split")
+    assert outs[-1].tobytes() == outs[-2].tobytes() == outs[-3].tobytes()   # and the shares settle
+    ctx.check_device_status()
+    ctx.close()
+
+
+def test_step_with_a_window_too_long_for_registers():
+    """W > 128 takes the freezing rule's loop path; it must agree with the oracle too."""
+    M, W, T, H = 3, 150, np.float32(1e-4), 400
+    k = np.arange(H)
+    hist = np.stack([0.02 * np.exp(-k / (20.0 + 30 * m)) + 0.003 + 1e-5 * np.cos(0.7 * k + m)
+                     for m in range(M)]).astype(np.float32)
+    ctx = eg.Context([64] * M, 8, W, float(T), device=DEV)
+    hist_dev = torch.from_numpy(hist).to(DEV)
+    slopes = np.empty((M, H))
+    masks = np.empty((M, H), dtype=np.uint8)
+    for i in range(H):
+        s, mk = ctx.egeria_plasticity_step(hist_dev[:, i].contiguous())
+        slopes[:, i], masks[:, i] = s.cpu().numpy(), mk.cpu().numpy()
+    for m in range(M):
+        ref = oracle.plasticity_replay(hist[m], W, float(T))
+        live = np.isfinite(ref["slopes"])
+        np.testing.assert_allclose(slopes[m][live], ref["slopes"][live], rtol=1e-9, atol=1e-15)
+        sl = ref["slopes"][live]
+        if not np.any(np.abs(np.abs(sl) - T) <= 1e-6):
+            assert bool(masks[m, -1]) == ref["converged"]
+    ctx.close()
 
 
 def test_alg1_hand_traces_on_gpu():

@@ -133,6 +133,47 @@ def test_plan_odd_shapes(d, b, n):
     _check_plan(d, b, n)
 
 
+@pytest.mark.parametrize("name", ["resnet50", "gpt2_medium", "resnet56"])
+def test_weighted_plan_gives_shares_in_proportion(name):
+    w = wl.WORKLOADS[name]
+    d, n = list(w.d), 148
+    rng = np.random.default_rng(7)
+    weights = (1.0 + 0.08 * rng.standard_normal(n)).astype(np.float32)
+    units = eg.egeria_debug_plan_weighted(d, w.b, n, weights)
+    # still an exact cover, in order
+    sides = [2] if w.b <= 64 else [0, 1]
+    for m in range(len(d)):
+        for s in sides:
+            rows = units[(units[:, 0] == m) & (units[:, 1] == s)]
+            pos = 0
+            for r in rows:
+                assert r[2] == pos and r[3] >= 1
+                pos += r[3]
+            assert pos == (d[m] + 63) // 64
+    assert np.all(np.diff(units[:, 4]) >= 0)
+    assert len(units) <= len(sides) * len(d) + 2 * n
+    per = np.bincount(units[:, 4], weights=units[:, 3], minlength=n)
+    want = per.sum() * weights.astype(np.float64) / weights.astype(np.float64).sum()
+    assert np.max(np.abs(per - want)) <= 1.0 + 1e-6 * per.sum()
+    # equal weights and no weights are the same split
+    eq = eg.egeria_debug_plan_weighted(d, w.b, n, np.ones(n, dtype=np.float32))
+    per_eq = np.bincount(eq[:, 4], weights=eq[:, 3], minlength=n)
+    assert per_eq.max() - per_eq.min() <= 1
+    assert np.array_equal(eg.egeria_debug_plan_weighted(d, w.b, n, None), eg.egeria_debug_plan(d, w.b, n))
+
+
+def test_weighted_plan_ignores_bad_weights_and_small_problems():
+    d, b, n = [802816, 401408], 64, 148
+    base = eg.egeria_debug_plan(d, b, n)
+    for bad in (np.zeros(n), np.full(n, np.nan), -np.ones(n), np.full(n, np.inf)):
+        got = eg.egeria_debug_plan_weighted(d, b, n, bad.astype(np.float32))
+        assert np.array_equal(got, base)
+    # a problem that does not fill every CTA keeps the equal split
+    small = eg.egeria_debug_plan([4096], 8, n)
+    w = np.linspace(0.5, 1.5, n).astype(np.float32)
+    assert np.array_equal(eg.egeria_debug_plan_weighted([4096], 8, n, w), small)
+
+
 def test_plan_rejects_bad_arguments():
     out = np.zeros((4, 5), dtype=np.int32)
     n = ctypes.c_int()
