@@ -167,28 +167,41 @@ __device__ __forceinline__ bool next_chunk(int &k, int q, int lane, int b, float
     return false;
 }
 
-// All epilogue warps: wait until `total` units of the module are complete, to help finish it.
-// One lane of the CTA polls (a counter that every waiting warp of every CTA polled would be a
-// hot spot); the others wait for it at a barrier.  The wait is a courtesy, not a dependency:
+// One warp: wait until `total` units of the module are complete, to help finish it.  The first
+// warp of the CTA to get here polls the counter (a counter that every waiting warp of every CTA
+// polled would be a hot spot); the others watch its verdict in shared memory (*state: 0 nobody
+// polls yet, 1 being polled, 2 complete, 3 gave up).  The wait is a courtesy, not a dependency:
 // the CTA that delivers the module's last unit finishes every row nobody else has claimed, so a
 // CTA that stops waiting (false) loses nothing but parallelism.  That keeps the kernel correct
 // when not all of its CTAs are resident together.
 __device__ __forceinline__ bool wait_units_done(const int32_t *units_done, int total, volatile int *abort_flag,
-                                                volatile int *verdict, bool poller) {
-    if (poller) {
-        int ok = 1;
-        const uint64_t t0 = ptx::globaltimer_ns();
-        while (ld_acquire(units_done) < total) {
-            if (*abort_flag || ptx::globaltimer_ns() - t0 > kHelpWaitNs) {
-                ok = 0;
-                break;
+                                                int *state, int lane) {
+    int v = 0;
+    if (lane == 0) {
+        if (atomicCAS(state, 0, 1) == 0) {
+            v = 2;
+            const uint64_t t0 = ptx::globaltimer_ns();
+            while (ld_acquire(units_done) < total) {
+                if (*abort_flag || ptx::globaltimer_ns() - t0 > kHelpWaitNs) {
+                    v = 3;
+                    break;
+                }
+                __nanosleep(100);
             }
-            __nanosleep(100);
+            __threadfence_block();
+            *reinterpret_cast<volatile int *>(state) = v;
+        } else {
+            const uint64_t t0 = ptx::globaltimer_ns();
+            while ((v = *reinterpret_cast<volatile int *>(state)) == 1) {
+                if (ptx::globaltimer_ns() - t0 > 2 * kHelpWaitNs) {
+                    v = 3;
+                    break;
+                }
+                __nanosleep(50);
+            }
         }
-        *verdict = ok;
     }
-    epi_bar_sync();
-    return *verdict != 0;
+    return __shfl_sync(0xffffffffu, v, 0) == 2;
 }
 
 // One warp: take rows of module m from its cursor until none is left.  The claim of the next
@@ -241,7 +254,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     volatile uint32_t *tmem_holder =
         reinterpret_cast<volatile uint32_t *>(bars + 2 * Cfg::kStages + 2 * Cfg::kAccStages);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
-    volatile int *wait_verdict = reinterpret_cast<volatile int *>(tmem_holder + 2);
+    int *wait_state = reinterpret_cast<int *>(const_cast<uint32_t *>(tmem_holder) + 2);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -265,6 +278,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             ptx::mbar_init(accempty0 + 8 * s, kEpiWarps);  // one arrival per epilogue warp
         }
         *abort_flag = 0;
+        *wait_state = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
     }
@@ -491,10 +505,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 if (m == prev_m) continue;
                 prev_m = m;
                 const int total = p.fin.sides[2 * m].module_units;
+                // With many CTAs on a module and few rows, most claims would find nothing and only
+                // crowd the cursor: as many warps of this CTA as its share of the rows, plus one.
+                const int ctas_on_m = Cfg::kStacked ? total : (total + 1) / 2;
+                if (warp - 2 > (b + ctas_on_m - 1) / ctas_on_m) continue;
                 bool ready;
                 if (m == m_last) {
-                    // every warp of the CTA gets here (same units, same order): wait together
-                    ready = detail::wait_units_done(&p.ctr[m].units_done, total, abort_flag, wait_verdict, epi_leader);
+                    ready = detail::wait_units_done(&p.ctr[m].units_done, total, abort_flag, wait_state, lane);
                 } else {
                     int done = 0;
                     if (lane == 0) done = detail::ld_acquire(&p.ctr[m].units_done);
