@@ -67,6 +67,15 @@ def lib() -> ctypes.CDLL:
             ctypes.POINTER(ctypes.c_float), i64, i64, ctypes.c_double, ctypes.c_int,
             f64p, f64p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
         L.egeria_oracle_plasticity_replay.restype = ctypes.c_int
+        i32p = ctypes.POINTER(ctypes.c_int32)
+        L.egeria_oracle_plasticity_replay_auto.argtypes = [
+            ctypes.POINTER(ctypes.c_float), i64, i64, ctypes.c_int, f64p, i32p, f64p]
+        L.egeria_oracle_plasticity_replay_auto.restype = ctypes.c_int
+        L.egeria_oracle_frontmost_replay.argtypes = [
+            ctypes.POINTER(ctypes.c_float), i64, i64, i64, f64p, ctypes.c_int, ctypes.c_int, i32p, i32p, f64p]
+        L.egeria_oracle_frontmost_replay.restype = ctypes.c_int
+        L.egeria_oracle_bootstrap_replay.argtypes = [ctypes.POINTER(ctypes.c_float), i64, i64, ctypes.c_double, f64p]
+        L.egeria_oracle_bootstrap_replay.restype = ctypes.c_int64
         _lib = L
     return _lib
 
@@ -174,3 +183,51 @@ def plasticity_replay(hist, W: int, T: float, signed_test: bool = False):
         raise RuntimeError(f"oracle replay failed ({rc})")
     return dict(smoothed=sm[:H], slopes=sl[:H], counter=cnt.value, freeze_eval=fe.value,
                 converged=bool(rc))
+
+
+def plasticity_replay_auto(hist, W: int, signed_test: bool = False):
+    """Algorithm 1 with the per-module tolerance of Sec. 4.2.2: 20 % of the largest |slope| in
+    the module's initial 3 readings.  Returns dict(slopes[H], freeze_eval, converged, T)."""
+    h = np.ascontiguousarray(hist, dtype=np.float32)
+    H = h.shape[0]
+    sl = np.empty(max(H, 1), dtype=np.float64)
+    fe = ctypes.c_int32()
+    T = ctypes.c_double()
+    rc = lib().egeria_oracle_plasticity_replay_auto(_p(h, ctypes.c_float), H, int(W), int(bool(signed_test)),
+                                                    _p(sl, ctypes.c_double), ctypes.byref(fe), ctypes.byref(T))
+    if rc < 0:
+        raise RuntimeError(f"oracle replay_auto failed ({rc})")
+    return dict(slopes=sl[:H], freeze_eval=fe.value, converged=bool(rc), T=T.value)
+
+
+def frontmost_replay(hist, W: int, T=None, signed_test: bool = False):
+    """Frontmost-active policy (Sec. 4.2.2, Algorithm 1 `l <- l + 1`) over [M, H] raw readings.
+    T: per-module tolerances, or None for the automatic one.
+    Returns dict(freeze_eval[M], monitored[H], slopes[H], frozen)."""
+    h = np.ascontiguousarray(hist, dtype=np.float32)
+    M, H = h.shape
+    auto = T is None
+    Tarr = np.zeros(M, dtype=np.float64) if auto else np.ascontiguousarray(np.broadcast_to(T, (M,)), dtype=np.float64)
+    fe = np.empty(M, dtype=np.int32)
+    mon = np.empty(max(H, 1), dtype=np.int32)
+    sl = np.empty(max(H, 1), dtype=np.float64)
+    rc = lib().egeria_oracle_frontmost_replay(_p(h, ctypes.c_float), M, H, int(W), _p(Tarr, ctypes.c_double),
+                                              int(bool(signed_test)), int(auto), _p(fe, ctypes.c_int32),
+                                              _p(mon, ctypes.c_int32), _p(sl, ctypes.c_double))
+    if rc < 0:
+        raise RuntimeError(f"oracle frontmost_replay failed ({rc})")
+    return dict(freeze_eval=fe, monitored=mon[:H], slopes=sl[:H], frozen=int(rc))
+
+
+def bootstrap_replay(loss_hist, W: int, rate_tol: float = 0.1):
+    """End of the bootstrapping stage (Sec. 3, Sec. 4.2.2): first evaluation with a full window
+    whose changing rate |slope| (W - 1) / |window mean| of the smoothed training loss is below
+    rate_tol.  Returns dict(end, rates[H])."""
+    h = np.ascontiguousarray(loss_hist, dtype=np.float32)
+    H = h.shape[0]
+    rates = np.empty(max(H, 1), dtype=np.float64)
+    end = lib().egeria_oracle_bootstrap_replay(_p(h, ctypes.c_float), H, int(W), float(rate_tol),
+                                               _p(rates, ctypes.c_double))
+    if end < -1:
+        raise RuntimeError("oracle bootstrap_replay: bad sizes")
+    return dict(end=int(end), rates=rates[:H])

@@ -234,3 +234,137 @@ int egeria_oracle_plasticity_replay(const float *hist, int64_t H, int64_t W, dou
     free(pl);
     return counter >= W ? 1 : 0;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Policies around Algorithm 1 that the paper states in prose.
+ * ------------------------------------------------------------------------------------------ */
+
+/* State of Algorithm 1 for one monitored module, advanced one reading at a time. */
+typedef struct {
+    double *P;        /* raw readings taken so far */
+    double *pl;       /* pList: smoothed readings */
+    int64_t len;      /* readings taken */
+    int64_t counter;  /* staleCounter */
+    double T;         /* tolerance in use (NaN while the automatic one is not set yet) */
+    double smax;      /* automatic tolerance: largest |slope| seen in the initial readings */
+} module_state;
+
+/* One call of checkPlasticity for a new raw reading [Algorithm 1], with the optional
+ * per-module tolerance of Sec. 4.2.2 ("Hyperparameters guideline"): T = 20% of the maximal
+ * |slope| in the module's initial 3 readings.  A slope exists from the 2nd reading on, so
+ * these are the slopes of evaluations 1 and 2; up to and including evaluation 2 no tolerance
+ * is known and the evaluation is never stale.  Returns the slope of this evaluation. */
+static double module_advance(module_state *st, double reading, int64_t W, int signed_test, int auto_T) {
+    int64_t i = st->len;
+    st->P[i] = reading;
+    double pbar = egeria_oracle_smooth(st->P, i, W);
+    st->pl[i] = pbar;
+    st->len = i + 1;
+    int64_t n = (st->len < W) ? st->len : W;
+    double s = egeria_oracle_ols_slope(st->pl + (st->len - n), n);
+    int stale;
+    if (auto_T && i <= 2) {
+        if (i >= 1 && fabs(s) > st->smax) st->smax = fabs(s);
+        if (i == 2) st->T = 0.2 * st->smax;
+        stale = 0;
+    } else {
+        stale = signed_test ? (s < st->T) : (fabs(s) < st->T);
+    }
+    st->counter = stale ? st->counter + 1 : 0;
+    return s;
+}
+
+/* Algorithm 1 for one module with the automatic tolerance.  Same outputs as
+ * egeria_oracle_plasticity_replay plus the tolerance that was derived (NaN if the history
+ * has fewer than 3 readings). */
+int egeria_oracle_plasticity_replay_auto(const float *hist, int64_t H, int64_t W, int signed_test,
+                                         double *slopes, int32_t *freeze_eval_out, double *T_out) {
+    if (H < 0 || W < 1) return -2;
+    module_state st;
+    st.P = (double *)malloc(sizeof(double) * (size_t)(H > 0 ? H : 1));
+    st.pl = (double *)malloc(sizeof(double) * (size_t)(H > 0 ? H : 1));
+    if (!st.P || !st.pl) { free(st.P); free(st.pl); return -1; }
+    st.len = 0; st.counter = 0; st.T = NAN; st.smax = 0.0;
+    int32_t freeze_eval = -1;
+    for (int64_t i = 0; i < H; ++i) if (slopes) slopes[i] = NAN;
+    for (int64_t i = 0; i < H && st.counter < W; ++i) {
+        double s = module_advance(&st, (double)hist[i], W, signed_test, 1);
+        if (slopes) slopes[i] = s;
+        if (st.counter >= W) freeze_eval = (int32_t)i;
+    }
+    if (freeze_eval_out) *freeze_eval_out = freeze_eval;
+    if (T_out) *T_out = st.T;
+    int conv = st.counter >= W;
+    free(st.P); free(st.pl);
+    return conv;
+}
+
+/* The frontmost-active policy [Sec. 4.2.2: "monitors the frontmost active layer module l to
+ * avoid a fragmented frozen model"; Algorithm 1: freeze, then l <- l + 1].  Modules are ordered
+ * front to back.  Only module l = (number of frozen modules) is monitored: evaluation i feeds
+ * it hist[l][i]; when its counter reaches W it is frozen at that evaluation and the next
+ * evaluation starts module l + 1 from a cleared state.  hist is [M][H] row-major.
+ * Outputs: freeze_eval[M] (-1 = not frozen within the history), monitored[H] (module fed at
+ * evaluation i, or M when all are frozen), slopes[H] (its slope, NaN when none was fed).
+ * T is [M] (ignored when auto_T).  Returns the number of frozen modules, negative on error. */
+int egeria_oracle_frontmost_replay(const float *hist, int64_t M, int64_t H, int64_t W, const double *T,
+                                   int signed_test, int auto_T, int32_t *freeze_eval,
+                                   int32_t *monitored, double *slopes) {
+    if (M < 1 || H < 0 || W < 1) return -2;
+    module_state st;
+    st.P = (double *)malloc(sizeof(double) * (size_t)(H > 0 ? H : 1));
+    st.pl = (double *)malloc(sizeof(double) * (size_t)(H > 0 ? H : 1));
+    if (!st.P || !st.pl) { free(st.P); free(st.pl); return -1; }
+    for (int64_t m = 0; m < M; ++m) freeze_eval[m] = -1;
+    int64_t l = 0;
+    st.len = 0; st.counter = 0; st.smax = 0.0;
+    st.T = auto_T ? NAN : T[0];
+    for (int64_t i = 0; i < H; ++i) {
+        if (monitored) monitored[i] = (int32_t)l;
+        if (slopes) slopes[i] = NAN;
+        if (l >= M) continue;
+        double s = module_advance(&st, (double)hist[l * H + i], W, signed_test, auto_T);
+        if (slopes) slopes[i] = s;
+        if (st.counter >= W) {
+            freeze_eval[l] = (int32_t)i;
+            ++l;
+            st.len = 0; st.counter = 0; st.smax = 0.0;
+            st.T = (auto_T || l >= M) ? NAN : T[l];
+        }
+    }
+    free(st.P); free(st.pl);
+    return (int)l;
+}
+
+/* End of the bootstrapping stage [Sec. 3 "Bootstrapping stage": the changing rate of the
+ * training loss is monitored "in line with the later plasticity monitoring"; Sec. 4.2.2: the
+ * changing rate that ends the stage is 10%].  The training-loss readings are smoothed [Eq. 2]
+ * and fitted like the plasticity; with a full window of W smoothed values, slope s and window
+ * mean ybar, the changing rate is |s| (W - 1) / |ybar|: the relative change of the fitted line
+ * across the window.  The stage ends at the first evaluation with a full window whose rate is
+ * below rate_tol.  rates[H] gets the rate (NaN before the window is full and after the end).
+ * Returns the evaluation index at which the stage ended, -1 if it did not, -2 on bad sizes. */
+int64_t egeria_oracle_bootstrap_replay(const float *loss, int64_t H, int64_t W, double rate_tol,
+                                       double *rates) {
+    if (H < 0 || W < 2) return -2;
+    double *P = (double *)malloc(sizeof(double) * (size_t)(H > 0 ? H : 1));
+    double *pl = (double *)malloc(sizeof(double) * (size_t)(H > 0 ? H : 1));
+    if (!P || !pl) { free(P); free(pl); return -2; }
+    int64_t end = -1;
+    for (int64_t i = 0; i < H; ++i) if (rates) rates[i] = NAN;
+    for (int64_t i = 0; i < H && end < 0; ++i) {
+        P[i] = (double)loss[i];
+        pl[i] = egeria_oracle_smooth(P, i, W);
+        if (i + 1 < W) continue;
+        const double *y = pl + (i + 1 - W);
+        double s = egeria_oracle_ols_slope(y, W);
+        double ybar = 0.0;
+        for (int64_t k = 0; k < W; ++k) ybar += y[k];
+        ybar /= (double)W;
+        double rate = fabs(s) * (double)(W - 1) / fabs(ybar);
+        if (rates) rates[i] = rate;
+        if (rate < rate_tol) end = i;
+    }
+    free(P); free(pl);
+    return end;
+}

@@ -326,3 +326,144 @@ def test_larger_T_or_smaller_W_freezes_earlier():
     assert a != -1 and b_ != -1 and b_ < a
     assert c != -1 and c < a
     assert f(10, 1e-12) == -1
+
+
+# ----------------------------------------------------------------------------- policies around Algorithm 1
+
+def _policy_lines(kind):
+    for line in (GOLDEN / "policy_traces.txt").read_text().splitlines():
+        if line.startswith("#") or not line.strip():
+            continue
+        f = [x.strip() for x in line.split("|")]
+        if f[0] == kind:
+            yield f
+
+
+def _frac_list(txt):
+    out = []
+    for tok in txt.split():
+        out.append(np.nan if tok == "x" else (np.inf if tok == "inf" else float(Fraction(tok))))
+    return np.array(out)
+
+
+@pytest.mark.parametrize("f", list(_policy_lines("auto")))
+def test_auto_tolerance_hand_traces(f):
+    W, hist = int(f[1]), np.array([float(v) for v in f[2].split()], dtype=np.float32)
+    want = _frac_list(f[3])
+    got = oracle.plasticity_replay_auto(hist, W)
+    assert got["T"] == pytest.approx(float(Fraction(f[4])), rel=1e-12)
+    assert got["freeze_eval"] == int(f[5])
+    live = ~np.isnan(want)
+    assert np.array_equal(np.isnan(got["slopes"]), ~live)
+    fin = live & np.isfinite(want)
+    np.testing.assert_allclose(got["slopes"][fin], want[fin], rtol=1e-12, atol=1e-15)
+    assert np.all(np.isinf(got["slopes"][live & ~fin]))
+
+
+def test_auto_tolerance_of_a_straight_line_is_a_tenth_of_its_slope():
+    # raw readings a + beta i: the first three smoothed values are a, a + beta/2, a + beta, so both
+    # early slopes are beta/2 and T = |beta|/10; once the window is full the slope is beta: never stale
+    for beta in (0.3, -2.0):
+        hist = (5.0 + beta * np.arange(40)).astype(np.float32)
+        got = oracle.plasticity_replay_auto(hist, 6)
+        assert got["T"] == pytest.approx(abs(beta) / 10, rel=1e-6)
+        assert got["freeze_eval"] == -1
+    # a constant history gives T = 0, and |0| < 0 is false: it never freezes either
+    got = oracle.plasticity_replay_auto(np.full(30, 2.5, dtype=np.float32), 4)
+    assert got["T"] == 0.0 and got["freeze_eval"] == -1
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_auto_tolerance_equals_fixed_tolerance_after_the_initial_readings(seed):
+    # with T known the rule is the plain Algorithm 1, except that evaluations 0..2 cannot be stale:
+    # replay with the derived T and compare wherever the fixed-T run was not stale before evaluation 3
+    rng = np.random.default_rng(seed)
+    k = np.arange(80)
+    hist = (np.exp(-k / rng.uniform(3, 15)) + 0.05 + 0.002 * rng.standard_normal(80)).astype(np.float32)
+    W = int(rng.integers(3, 8))
+    a = oracle.plasticity_replay_auto(hist, W)
+    early = [abs(oracle.ols_slope([oracle.smooth(hist, j, W) for j in range(i + 1)][-W:])) for i in (1, 2)]
+    assert a["T"] == pytest.approx(0.2 * max(early), rel=1e-12)
+    b = oracle.plasticity_replay(hist, W, a["T"])
+    stale_early = np.abs(b["slopes"][1:3]) < a["T"]
+    if not stale_early.any():
+        assert a["freeze_eval"] == b["freeze_eval"]
+        np.testing.assert_array_equal(a["slopes"], b["slopes"])
+
+
+@pytest.mark.parametrize("f", list(_policy_lines("front")))
+def test_frontmost_hand_traces(f):
+    W = int(f[1])
+    T = [float(v) for v in f[2].split()]
+    hist = np.array([[float(v) for v in row.split()] for row in f[3].split(";")], dtype=np.float32)
+    got = oracle.frontmost_replay(hist, W, T)
+    assert got["monitored"].tolist() == [int(v) for v in f[4].split()]
+    assert got["freeze_eval"].tolist() == [int(v) for v in f[5].split()]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_frontmost_is_single_module_replays_chained(seed):
+    # the policy only decides WHICH module is fed: module l's run must be the plain Algorithm 1 on
+    # its own readings from the evaluation after module l - 1 froze
+    rng = np.random.default_rng(100 + seed)
+    M, H, W = 4, 120, int(rng.integers(2, 6))
+    k = np.arange(H)
+    hist = np.stack([0.3 * np.exp(-k / rng.uniform(2, 10)) + 0.01 * (m + 1) + 1e-4 * rng.standard_normal(H)
+                     for m in range(M)]).astype(np.float32)
+    T = rng.uniform(2e-3, 2e-2, size=M)
+    got = oracle.frontmost_replay(hist, W, T)
+    start, frozen = 0, 0
+    for m in range(M):
+        if start >= H:
+            assert got["freeze_eval"][m] == -1
+            continue
+        single = oracle.plasticity_replay(hist[m, start:], W, float(T[m]))
+        if single["converged"]:
+            assert got["freeze_eval"][m] == start + single["freeze_eval"]
+            n = single["freeze_eval"] + 1
+            np.testing.assert_array_equal(got["slopes"][start:start + n], single["slopes"][:n])
+            assert np.all(got["monitored"][start:start + n] == m)
+            start += n
+            frozen += 1
+        else:
+            assert got["freeze_eval"][m] == -1
+            assert np.all(got["monitored"][start:] == m)
+            start = H
+    assert got["frozen"] == frozen
+    fe = got["freeze_eval"]
+    assert np.all(fe[:frozen] >= 0) and np.all(fe[frozen:] == -1) and np.all(np.diff(fe[:frozen]) > 0)
+    # one module: the policy changes nothing
+    one = oracle.frontmost_replay(hist[:1], W, T[:1])
+    assert one["freeze_eval"][0] == oracle.plasticity_replay(hist[0], W, float(T[0]))["freeze_eval"]
+
+
+@pytest.mark.parametrize("f", list(_policy_lines("boot")))
+def test_bootstrap_hand_traces(f):
+    W, tol = int(f[1]), float(f[2])
+    hist = np.array([float(v) for v in f[3].split()], dtype=np.float32)
+    want = _frac_list(f[4])
+    got = oracle.bootstrap_replay(hist, W, tol)
+    assert got["end"] == int(f[5])
+    assert np.array_equal(np.isnan(got["rates"]), np.isnan(want))
+    np.testing.assert_allclose(got["rates"][~np.isnan(want)], want[~np.isnan(want)], rtol=1e-6)
+
+
+def test_bootstrap_closed_forms():
+    # a constant loss changes by 0 %: the stage ends with the first full window
+    assert oracle.bootstrap_replay(np.full(20, 3.0, dtype=np.float32), 5)["end"] == 4
+    # a straight line a - beta i: once every smoothed value in the window is a full average
+    # (i >= 2W - 2) the fitted slope is -beta and the window mean a - beta (i - W + 1)
+    a, beta, W = 100.0, 0.5, 6
+    got = oracle.bootstrap_replay((a - beta * np.arange(60)).astype(np.float32), W, 1e-9)
+    for i in range(2 * W - 2, 60):
+        assert got["rates"][i] == pytest.approx(beta * (W - 1) / (a - beta * (i - W + 1)), rel=1e-6)
+    assert got["end"] == -1
+    # the rate is relative: scaling the loss by any positive constant changes nothing
+    rng = np.random.default_rng(3)
+    base = (2.0 * np.exp(-np.arange(50) / 7.0) + 0.3 + 0.01 * rng.random(50)).astype(np.float32)
+    r1 = oracle.bootstrap_replay(base, 5, 0.1)
+    r2 = oracle.bootstrap_replay(base * np.float32(8.0), 5, 0.1)   # exact in float32
+    assert r1["end"] == r2["end"] and r1["end"] > 5
+    np.testing.assert_allclose(r1["rates"][4:r1["end"] + 1], r2["rates"][4:r1["end"] + 1], rtol=1e-12)
+    # a looser tolerance can only end the stage earlier
+    assert oracle.bootstrap_replay(base, 5, 0.3)["end"] <= r1["end"]
