@@ -72,7 +72,22 @@ enum {
      * low-order bits of a loss can differ between evaluations across a change of
      * shares and from run to run; with this flag every evaluation of the same
      * inputs gives the same bits. */
-    EGERIA_FLAG_EQUAL_SPLIT = 32u
+    EGERIA_FLAG_EQUAL_SPLIT = 32u,
+    /* Per-module tolerance [Sec. 4.2.2, "Hyperparameters guideline"]: T of a
+     * module is 20 % of the largest |slope| in its initial 3 readings (a slope
+     * exists from the 2nd reading on, so these are evaluations 1 and 2).  The T
+     * given at creation is ignored; evaluations 0..2 of a module only set its
+     * tolerance and are never stale. */
+    EGERIA_FLAG_AUTO_T = 64u,
+    /* Frontmost-active policy [Sec. 4.2.2 "monitors the frontmost active layer
+     * module l to avoid a fragmented frozen model"; Algorithm 1: freeze, then
+     * l <- l + 1].  Modules are ordered front to back.  Only module l = (number
+     * of frozen modules) is advanced by an evaluation; when its counter reaches
+     * W it is frozen, and the NEXT evaluation starts module l + 1 from a cleared
+     * state.  out_mask is then a prefix mask (1 for the frozen modules) and
+     * out_slopes holds this evaluation's slope for the monitored module, the
+     * final slope of every frozen one and +inf for those not monitored yet. */
+    EGERIA_FLAG_FRONTMOST = 128u
 };
 
 #define EGERIA_MAX_B 256          /* largest supported mini-batch size */
@@ -168,6 +183,45 @@ egeria_status egeria_plasticity_replay(egeria_ctx *ctx, void *cuda_stream, const
  * is non-zero the window is halved first (never below 2), as the paper does
  * for refreezing. */
 egeria_status egeria_plasticity_reset(egeria_ctx *ctx, void *cuda_stream, int halve_W);
+
+/* End of the bootstrapping stage [Sec. 3 "Bootstrapping stage": the changing rate
+ * of the training loss is monitored in line with the plasticity; Sec. 4.2.2: the
+ * changing rate that ends the stage is 10 %].  The training-loss readings are
+ * smoothed (Eq. 2) and fitted like a plasticity series, with the window W given
+ * at creation (>= 2); with a full window of W smoothed values, slope s and window
+ * mean ybar, the changing rate is |s| (W - 1) / |ybar| -- the relative change of
+ * the fitted line across the window -- and the stage ends at the first evaluation
+ * whose rate is below rate_tol (the paper's value: 0.1).  The state is separate
+ * from the modules' and is not touched by egeria_plasticity_reset.
+ *   train_loss  device float [1]: the new reading
+ *   out_rate    device double [1]: rate of this evaluation, NaN while the window
+ *               is not full and once the stage has ended; may be NULL
+ *   out_done    device uint8 [1]: 1 once the stage has ended; may be NULL */
+egeria_status egeria_bootstrap_step(egeria_ctx *ctx, void *cuda_stream, const float *train_loss,
+                                    float rate_tol, double *out_rate, uint8_t *out_done);
+
+/* The same over a whole history, from a cleared state private to the call.
+ *   loss_hist  device float [H]     out_rates  device double [H], may be NULL
+ *   out_end    device int32 [1]: evaluation at which the stage ended, -1 if not */
+egeria_status egeria_bootstrap_replay(egeria_ctx *ctx, void *cuda_stream, const float *loss_hist,
+                                      int H, float rate_tol, double *out_rates, int32_t *out_end);
+
+/* Start the bootstrapping detector of the context afresh. */
+egeria_status egeria_bootstrap_reset(egeria_ctx *ctx, void *cuda_stream);
+
+/* Checkpointing of the freezing-rule state (windows, counters, tolerances, the
+ * front, the bootstrapping detector; not the work split).  export copies it,
+ * with a small header, to a HOST buffer of at least
+ * egeria_plasticity_state_bytes() bytes and synchronises the stream; import
+ * restores it into a context created with the same M, W and rule flags (else
+ * EGERIA_ERR_INVALID_ARG) and synchronises the stream.  A too small buffer gives
+ * EGERIA_ERR_WORKSPACE.  The paper has no counterpart: it is what a training job
+ * that checkpoints needs to resume with the same freezing decisions. */
+size_t egeria_plasticity_state_bytes(const egeria_ctx *ctx);
+egeria_status egeria_plasticity_export(egeria_ctx *ctx, void *cuda_stream, void *host_buffer,
+                                       size_t buffer_bytes);
+egeria_status egeria_plasticity_import(egeria_ctx *ctx, void *cuda_stream, const void *host_buffer,
+                                       size_t buffer_bytes);
 
 /* Current window of the context (changes only through egeria_plasticity_reset). */
 int egeria_plasticity_window(const egeria_ctx *ctx);

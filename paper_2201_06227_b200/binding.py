@@ -18,7 +18,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libegeria.so"
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 FLAG_SIGNED_SLOPE, FLAG_FORCE_SIMT, FLAG_KEEP_GRAMS, FLAG_HOST_STAGING, FLAG_TIME_GRAM = 1, 2, 4, 8, 16
-FLAG_EQUAL_SPLIT = 32
+FLAG_EQUAL_SPLIT, FLAG_AUTO_T, FLAG_FRONTMOST = 32, 64, 128
 MAX_B = 256
 WORKSPACE_ALIGN = 1024
 
@@ -29,7 +29,8 @@ EXPORTS = [
     "egeria_debug_dump_gram", "egeria_debug_plan", "egeria_debug_plan_weighted", "egeria_device_status",
     "egeria_launch_count",
     "egeria_gram_kernel_time", "egeria_sp_loss_static", "egeria_plasticity_evaluate",
-    "egeria_split_weights", "egeria_status_string",
+    "egeria_split_weights", "egeria_status_string", "egeria_bootstrap_step", "egeria_bootstrap_replay",
+    "egeria_bootstrap_reset", "egeria_plasticity_state_bytes", "egeria_plasticity_export", "egeria_plasticity_import",
 ]
 
 
@@ -72,6 +73,13 @@ def lib() -> ctypes.CDLL:
                                              ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32),
                                              ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
     L.egeria_split_weights.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.c_int]
+    L.egeria_bootstrap_step.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp]
+    L.egeria_bootstrap_replay.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_float, vp, vp]
+    L.egeria_bootstrap_reset.argtypes = [vp, vp]
+    L.egeria_plasticity_state_bytes.argtypes = [vp]
+    L.egeria_plasticity_state_bytes.restype = ctypes.c_size_t
+    L.egeria_plasticity_export.argtypes = [vp, vp, vp, ctypes.c_size_t]
+    L.egeria_plasticity_import.argtypes = [vp, vp, vp, ctypes.c_size_t]
     L.egeria_device_status.argtypes = [vp]
     L.egeria_gram_kernel_time.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
     L.egeria_sp_loss_static.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_int64, vp]
@@ -287,6 +295,46 @@ class Context:
     def egeria_plasticity_reset(self, halve_W: bool = False, stream: Optional[torch.cuda.Stream] = None) -> None:
         _check(lib().egeria_plasticity_reset(self._h, _stream_ptr(stream), int(bool(halve_W))),
                "egeria_plasticity_reset")
+
+    def egeria_bootstrap_step(self, train_loss: torch.Tensor, rate_tol: float = 0.1,
+                              stream: Optional[torch.cuda.Stream] = None):
+        """One more training-loss reading for the bootstrapping detector: (rate, done) device tensors."""
+        assert train_loss.is_cuda and train_loss.dtype == torch.float32 and train_loss.numel() == 1
+        rate = torch.empty(1, dtype=torch.float64, device=self.device)
+        done = torch.empty(1, dtype=torch.uint8, device=self.device)
+        _check(lib().egeria_bootstrap_step(self._h, _stream_ptr(stream), train_loss.data_ptr(), ctypes.c_float(rate_tol),
+                                           rate.data_ptr(), done.data_ptr()), "egeria_bootstrap_step")
+        return rate, done
+
+    def egeria_bootstrap_replay(self, loss_hist: torch.Tensor, rate_tol: float = 0.1,
+                                stream: Optional[torch.cuda.Stream] = None):
+        assert loss_hist.is_cuda and loss_hist.dtype == torch.float32 and loss_hist.dim() == 1
+        loss_hist = loss_hist.contiguous()
+        H = int(loss_hist.shape[0])
+        rates = torch.empty(max(H, 1), dtype=torch.float64, device=self.device)
+        end = torch.empty(1, dtype=torch.int32, device=self.device)
+        _check(lib().egeria_bootstrap_replay(self._h, _stream_ptr(stream), loss_hist.data_ptr(), H,
+                                             ctypes.c_float(rate_tol), rates.data_ptr(), end.data_ptr()),
+               "egeria_bootstrap_replay")
+        return rates[:H], end
+
+    def egeria_bootstrap_reset(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        _check(lib().egeria_bootstrap_reset(self._h, _stream_ptr(stream)), "egeria_bootstrap_reset")
+
+    def egeria_plasticity_state_bytes(self) -> int:
+        return int(lib().egeria_plasticity_state_bytes(self._h))
+
+    def egeria_plasticity_export(self, stream: Optional[torch.cuda.Stream] = None) -> np.ndarray:
+        """The freezing-rule state as host bytes (synchronises the stream)."""
+        buf = np.zeros(self.egeria_plasticity_state_bytes(), dtype=np.uint8)
+        _check(lib().egeria_plasticity_export(self._h, _stream_ptr(stream), buf.ctypes.data, buf.nbytes),
+               "egeria_plasticity_export")
+        return buf
+
+    def egeria_plasticity_import(self, buf: np.ndarray, stream: Optional[torch.cuda.Stream] = None) -> None:
+        buf = np.ascontiguousarray(buf, dtype=np.uint8)
+        _check(lib().egeria_plasticity_import(self._h, _stream_ptr(stream), buf.ctypes.data, buf.nbytes),
+               "egeria_plasticity_import")
 
     def egeria_plasticity_window(self) -> int:
         return int(lib().egeria_plasticity_window(self._h))

@@ -27,8 +27,10 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Offsets of everything the library keeps in the caller's workspace.
 struct Layout {
-    size_t status, cta_log, rowloss, tickets, fin_ctr, T, raw, plist, n_evals, counter, freeze_eval, last_slope, losses, keep,
-        slots, staging, total;
+    size_t status, cta_log, rowloss, tickets, fin_ctr, T, losses, keep, slots, staging, total;
+    // the freezing-rule state, one contiguous region [rule0, rule_end) (what export / import copy)
+    size_t rule0, raw, plist, n_evals, counter, freeze_eval, last_slope, Tauto, smax, front, boot_raw, boot_plist,
+        boot_ints, rule_end;
     size_t slot_bytes_cap;  // bytes reserved for partial slots
     // Device-side plans (tensor maps, pointers, unit table, per-CTA ranges, slot ranges): kPlanSlots
     // regions of plan_stride bytes from plan0; the offsets below are relative to a region.
@@ -71,12 +73,20 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
     L.tickets = take((size_t)M * sizeof(int32_t));
     L.fin_ctr = take((size_t)2 * M * sizeof(FinCounters));  // two sets, used by alternate launches
     L.T = take((size_t)M * sizeof(float));
+    L.rule0 = off;
     L.raw = take((size_t)M * W * sizeof(double));
     L.plist = take((size_t)M * W * sizeof(double));
     L.n_evals = take((size_t)M * sizeof(int32_t));
     L.counter = take((size_t)M * sizeof(int32_t));
     L.freeze_eval = take((size_t)M * sizeof(int32_t));
     L.last_slope = take((size_t)M * sizeof(double));
+    L.Tauto = take((size_t)M * sizeof(double));
+    L.smax = take((size_t)M * sizeof(double));
+    L.front = take(2 * sizeof(int32_t));
+    L.boot_raw = take((size_t)W * sizeof(double));
+    L.boot_plist = take((size_t)W * sizeof(double));
+    L.boot_ints = take(2 * sizeof(int32_t));
+    L.rule_end = off;
     L.losses = take((size_t)M * sizeof(float));
     L.keep = off;
     if (flags & EGERIA_FLAG_KEEP_GRAMS) take((size_t)M * 2 * b_max * b_max * sizeof(float));
@@ -146,6 +156,7 @@ struct egeria_ctx {
     cudaStream_t last_stream = nullptr;
     int64_t launches = 0;
     uint32_t tc_launches = 0;  // selects the set of progress counters the next tensor-core launch uses
+    uint32_t rule_evals = 0;   // evaluations of the freezing rule enqueued: its parity selects the front counter
     // Split weights: one per CTA, from the streaming rates the CTAs report (SMs do not all get
     // the same share of HBM bandwidth; the CTA -> SM placement repeats from launch to launch).
     std::vector<float> weights;
@@ -164,6 +175,18 @@ struct egeria_ctx {
     T *at(size_t off) const {
         return reinterpret_cast<T *>(ws + off);
     }
+    int rule_flags() const {
+        return ((flags & EGERIA_FLAG_SIGNED_SLOPE) ? kRuleSigned : 0) | ((flags & EGERIA_FLAG_AUTO_T) ? kRuleAutoT : 0) |
+               ((flags & EGERIA_FLAG_FRONTMOST) ? kRuleFrontmost : 0);
+    }
+    BootState boot_state() const {
+        BootState bs;
+        bs.raw = at<double>(L.boot_raw);
+        bs.plist = at<double>(L.boot_plist);
+        bs.n_evals = at<int32_t>(L.boot_ints);
+        bs.end = at<int32_t>(L.boot_ints) + 1;
+        return bs;
+    }
     SlopeState slope_state() const {
         SlopeState st;
         st.raw = at<double>(L.raw);
@@ -172,6 +195,9 @@ struct egeria_ctx {
         st.counter = at<int32_t>(L.counter);
         st.freeze_eval = at<int32_t>(L.freeze_eval);
         st.last_slope = at<double>(L.last_slope);
+        st.Tauto = at<double>(L.Tauto);
+        st.smax = at<double>(L.smax);
+        st.front = at<int32_t>(L.front);
         st.T = at<float>(L.T);
         st.W_cap = W_cap;
         return st;
@@ -306,7 +332,8 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     if (e == cudaSuccess) e = cudaMemcpy(ctx->ws + L.T, Th.data(), (size_t)M * sizeof(float), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) {
         plasticity_clear_kernel<<<(M + 127) / 128, 128>>>(ctx->slope_state(), M);
-        ctx->launches++;
+        bootstrap_clear_kernel<<<1, 1>>>(ctx->boot_state());
+        ctx->launches += 2;
         e = cudaDeviceSynchronize();
     }
     if (e != cudaSuccess) {
@@ -548,7 +575,10 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
     fc.keep = (ctx->flags & EGERIA_FLAG_KEEP_GRAMS) ? ctx->at<float>(L.keep) : nullptr;
     fc.fuse_step = fuse_step ? 1 : 0;
     fc.W = ctx->W;
-    fc.signed_test = (ctx->flags & EGERIA_FLAG_SIGNED_SLOPE) ? 1 : 0;
+    fc.rule_flags = ctx->rule_flags();
+    fc.rule_parity = (int)(ctx->rule_evals & 1u);
+    fc.M = ctx->M;
+    if (fuse_step) ctx->rule_evals++;
     fc.st = ctx->slope_state();
     fc.out_slopes = out_slopes;
     fc.out_mask = out_mask;
@@ -646,9 +676,9 @@ egeria_status egeria_plasticity_step(egeria_ctx *ctx, void *cuda_stream, const f
     if (!ctx || !losses) return EGERIA_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     ctx->last_stream = stream;
-    plasticity_step_kernel<<<ctx->M, 32, 0, stream>>>(ctx->slope_state(), ctx->M, ctx->W,
-                                                      (ctx->flags & EGERIA_FLAG_SIGNED_SLOPE) ? 1 : 0, losses,
-                                                      out_slopes, out_mask);
+    plasticity_step_kernel<<<ctx->M, 32, 0, stream>>>(ctx->slope_state(), ctx->M, ctx->W, ctx->rule_flags(),
+                                                      (int)(ctx->rule_evals & 1u), losses, out_slopes, out_mask);
+    ctx->rule_evals++;
     if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
     ctx->launches++;
     return EGERIA_OK;
@@ -659,9 +689,9 @@ egeria_status egeria_plasticity_replay(egeria_ctx *ctx, void *cuda_stream, const
     if (!ctx || !hist || H < 0 || !out_mask) return EGERIA_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     ctx->last_stream = stream;
-    plasticity_replay_kernel<<<ctx->M, 32, 2 * (size_t)ctx->W * sizeof(double), stream>>>(
-        ctx->at<float>(ctx->L.T), ctx->M, ctx->W, (ctx->flags & EGERIA_FLAG_SIGNED_SLOPE) ? 1 : 0, hist, H,
-        out_slopes, out_mask, out_freeze_eval);
+    const int grid = (ctx->flags & EGERIA_FLAG_FRONTMOST) ? 1 : ctx->M;
+    plasticity_replay_kernel<<<grid, 32, 2 * (size_t)ctx->W * sizeof(double), stream>>>(
+        ctx->at<float>(ctx->L.T), ctx->M, ctx->W, ctx->rule_flags(), hist, H, out_slopes, out_mask, out_freeze_eval);
     if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
     ctx->launches++;
     return EGERIA_OK;
@@ -678,6 +708,94 @@ egeria_status egeria_plasticity_reset(egeria_ctx *ctx, void *cuda_stream, int ha
     plasticity_clear_kernel<<<(ctx->M + 127) / 128, 128, 0, stream>>>(ctx->slope_state(), ctx->M);
     if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
     ctx->launches++;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_bootstrap_step(egeria_ctx *ctx, void *cuda_stream, const float *train_loss, float rate_tol,
+                                    double *out_rate, uint8_t *out_done) {
+    if (!ctx || !train_loss || !(rate_tol > 0.f)) return EGERIA_ERR_INVALID_ARG;
+    if (ctx->W_cap < 2) return EGERIA_ERR_INVALID_ARG;  // no line through one point
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    bootstrap_step_kernel<<<1, 32, 0, stream>>>(ctx->boot_state(), ctx->W_cap, (double)rate_tol, train_loss, out_rate,
+                                                out_done);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_bootstrap_replay(egeria_ctx *ctx, void *cuda_stream, const float *loss_hist, int H, float rate_tol,
+                                      double *out_rates, int32_t *out_end) {
+    if (!ctx || !loss_hist || H < 0 || !(rate_tol > 0.f) || !out_end) return EGERIA_ERR_INVALID_ARG;
+    if (ctx->W_cap < 2) return EGERIA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    bootstrap_replay_kernel<<<1, 32, 2 * (size_t)ctx->W_cap * sizeof(double), stream>>>(
+        ctx->W_cap, (double)rate_tol, loss_hist, H, out_rates, out_end);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_bootstrap_reset(egeria_ctx *ctx, void *cuda_stream) {
+    if (!ctx) return EGERIA_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    bootstrap_clear_kernel<<<1, 1, 0, stream>>>(ctx->boot_state());
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
+// What export writes in front of the raw state: enough to refuse a buffer from another set-up.
+struct StateHeader {
+    uint32_t magic;
+    int32_t M, W_cap, W;
+    uint32_t rule_evals, flags;
+    uint64_t state_bytes;
+};
+constexpr uint32_t kStateMagic = 0x45474552u;  // "EGER"
+
+size_t egeria_plasticity_state_bytes(const egeria_ctx *ctx) {
+    return ctx ? sizeof(StateHeader) + (ctx->L.rule_end - ctx->L.rule0) : 0;
+}
+
+egeria_status egeria_plasticity_export(egeria_ctx *ctx, void *cuda_stream, void *host_buffer, size_t buffer_bytes) {
+    if (!ctx || !host_buffer) return EGERIA_ERR_INVALID_ARG;
+    if (buffer_bytes < egeria_plasticity_state_bytes(ctx)) return EGERIA_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    StateHeader h;
+    h.magic = kStateMagic;
+    h.M = ctx->M;
+    h.W_cap = ctx->W_cap;
+    h.W = ctx->W;
+    h.rule_evals = ctx->rule_evals;
+    h.flags = ctx->flags & (EGERIA_FLAG_SIGNED_SLOPE | EGERIA_FLAG_AUTO_T | EGERIA_FLAG_FRONTMOST);
+    h.state_bytes = ctx->L.rule_end - ctx->L.rule0;
+    memcpy(host_buffer, &h, sizeof(h));
+    EG_CUDA(cudaMemcpyAsync(static_cast<uint8_t *>(host_buffer) + sizeof(h), ctx->ws + ctx->L.rule0, h.state_bytes,
+                            cudaMemcpyDeviceToHost, stream));
+    EG_CUDA(cudaStreamSynchronize(stream));
+    return EGERIA_OK;
+}
+
+egeria_status egeria_plasticity_import(egeria_ctx *ctx, void *cuda_stream, const void *host_buffer, size_t buffer_bytes) {
+    if (!ctx || !host_buffer || buffer_bytes < sizeof(StateHeader)) return EGERIA_ERR_INVALID_ARG;
+    StateHeader h;
+    memcpy(&h, host_buffer, sizeof(h));
+    const uint32_t rule_bits = ctx->flags & (EGERIA_FLAG_SIGNED_SLOPE | EGERIA_FLAG_AUTO_T | EGERIA_FLAG_FRONTMOST);
+    if (h.magic != kStateMagic || h.M != ctx->M || h.W_cap != ctx->W_cap || h.flags != rule_bits ||
+        h.state_bytes != ctx->L.rule_end - ctx->L.rule0 || h.W < 1 || h.W > ctx->W_cap)
+        return EGERIA_ERR_INVALID_ARG;
+    if (buffer_bytes < sizeof(h) + h.state_bytes) return EGERIA_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    EG_CUDA(cudaMemcpyAsync(ctx->ws + ctx->L.rule0, static_cast<const uint8_t *>(host_buffer) + sizeof(h), h.state_bytes,
+                            cudaMemcpyHostToDevice, stream));
+    EG_CUDA(cudaStreamSynchronize(stream));  // the buffer may be pageable: it is free again on return
+    ctx->W = h.W;
+    ctx->rule_evals = h.rule_evals;
     return EGERIA_OK;
 }
 
@@ -871,7 +989,9 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     fc.keep = nullptr;
     fc.fuse_step = 0;
     fc.W = 0;
-    fc.signed_test = 0;
+    fc.rule_flags = 0;
+    fc.rule_parity = 0;
+    fc.M = 1;
     fc.st = SlopeState{};
     fc.out_slopes = nullptr;
     fc.out_mask = nullptr;

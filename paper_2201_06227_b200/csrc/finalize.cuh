@@ -33,7 +33,9 @@ struct FinCommon {
     // fused freezing-rule step (fuse_step != 0): Algorithm 1 on the loss just computed
     int32_t fuse_step;
     int32_t W;
-    int32_t signed_test;
+    int32_t rule_flags;     // RuleFlags
+    int32_t rule_parity;    // which front counter this evaluation reads (frontmost policy)
+    int32_t M;
     SlopeState st;
     double *out_slopes;     // [M] or nullptr
     uint8_t *out_mask;      // [M] or nullptr
@@ -232,7 +234,8 @@ __device__ __forceinline__ void finalize_module_total(const FinCommon &p, int m,
     s = warp_sum_f64(s);
     const float loss = (float)(s / ((double)b * (double)b));
     if (lane == 0) p.out_losses[m] = loss;
-    if (p.fuse_step) plasticity_step_apply(p.st, L, m, p.W, p.signed_test, loss, p.out_slopes, p.out_mask, lane);
+    if (p.fuse_step)
+        plasticity_rule_step(p.st, L, m, p.M, p.W, p.rule_flags, p.rule_parity, loss, p.out_slopes, p.out_mask, lane);
 }
 
 struct FinParams {

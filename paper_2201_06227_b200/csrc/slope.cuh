@@ -1,12 +1,21 @@
 // The freezing rule (Sec. 4.2.2, Eq. 2, Algorithm 1) for all modules: moving average
 // of the raw plasticity readings, least-squares slope of the last W smoothed values,
-// tolerance test, consecutive-stale counter.  One warp per module, float64 throughout.
+// tolerance test, consecutive-stale counter; and the policies the paper states around it:
+// the per-module automatic tolerance (Sec. 4.2.2 "Hyperparameters guideline"), the
+// frontmost-active policy (Sec. 4.2.2; Algorithm 1 "l <- l + 1") and the end of the
+// bootstrapping stage (Sec. 3).  One warp per module, float64 throughout.
 #pragma once
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
 
 namespace egeria {
+
+enum RuleFlags : int {
+    kRuleSigned = 1,     // the literal test of Algorithm 1, slope < T, instead of |slope| < T
+    kRuleAutoT = 2,      // T = 20 % of the largest |slope| in the module's initial 3 readings
+    kRuleFrontmost = 4,  // only the frontmost module that is not frozen is monitored
+};
 
 struct SlopeState {     // per-module arrays (device)
     double *raw;        // [M][W_cap] the last min(n_evals, W) raw readings P_i, oldest first
@@ -15,8 +24,11 @@ struct SlopeState {     // per-module arrays (device)
     int32_t *counter;   // [M] consecutive stale evaluations
     int32_t *freeze_eval;  // [M] evaluation index at which the counter reached W, or -1
     double *last_slope; // [M]
-    const float *T;     // [M] tolerance
-    int32_t W_cap;      // ring pitch
+    double *Tauto;      // [M] automatic tolerance (NaN until the third reading)
+    double *smax;       // [M] largest |slope| of the initial readings
+    int32_t *front;     // [2] number of frozen modules (frontmost policy): read [parity], write [parity ^ 1]
+    const float *T;     // [M] tolerance given at creation
+    int32_t W_cap;      // window pitch
 };
 
 __device__ __forceinline__ double warp_sum_f64(double v) {
@@ -25,52 +37,8 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
     return v;
 }
 
-// One evaluation of one module by one warp.  raw/plist are this module's rings of pitch
-// >= W (global or shared memory).  Returns the slope of this evaluation (all lanes).
-__device__ __forceinline__ double plasticity_advance(double *raw, double *plist, int &n_evals, int &counter,
-                                                     int &freeze_eval, double reading, int W, double T,
-                                                     bool signed_test, int lane) {
-    const int i = n_evals;
-    if (lane == 0) raw[i % W] = reading;
-    __syncwarp();
-    // Eq. 2: mean of the last min(i + 1, W) raw readings
-    const int n = (i + 1 < W) ? i + 1 : W;
-    double s = 0.0;
-    for (int k = lane; k < n; k += 32) s += raw[(i - n + 1 + k) % W];
-    const double pbar = warp_sum_f64(s) / (double)n;
-    if (lane == 0) plist[i % W] = pbar;
-    __syncwarp();
-    // windowLinearFit: least squares over the last min(len, W) entries of pList, x = 0..n2-1
-    const int len = i + 1;
-    const int n2 = (len < W) ? len : W;
-    double slope;
-    if (n2 < 2) {
-        slope = INFINITY;
-    } else {
-        const double xm = 0.5 * (double)(n2 - 1);
-        double sy = 0.0;
-        for (int k = lane; k < n2; k += 32) sy += plist[(len - n2 + k) % W];
-        const double ym = warp_sum_f64(sy) / (double)n2;
-        double sxy = 0.0, sxx = 0.0;
-        for (int k = lane; k < n2; k += 32) {
-            const double dx = (double)k - xm;
-            sxy += dx * (plist[(len - n2 + k) % W] - ym);
-            sxx += dx * dx;
-        }
-        sxy = warp_sum_f64(sxy);
-        sxx = warp_sum_f64(sxx);
-        slope = sxy / sxx;
-    }
-    const bool stale = signed_test ? (slope < T) : (fabs(slope) < T);  // NaN compares false
-    counter = stale ? counter + 1 : 0;
-    if (counter >= W && freeze_eval < 0) freeze_eval = i;
-    n_evals = i + 1;
-    return slope;
-}
-
-// Smoothing (Eq. 2), window fit and counter update of Algorithm 1 for one new reading, given
-// the module's two windows AFTER the new values are in place.  `val(k)` returns element k of
-// the smoothed window (k = 0 oldest) for the k this lane owns (k = lane, lane + 32, ...).
+// windowLinearFit: least-squares slope of y(0..n2-1) against x = 0..n2-1; `val(k)` returns
+// element k for the k this lane owns (k = lane, lane + 32, ...).  Fewer than 2 points: +inf.
 template <class F>
 __device__ __forceinline__ double window_slope(int n2, int lane, F val) {
     if (n2 < 2) return INFINITY;
@@ -113,13 +81,63 @@ __device__ __forceinline__ double window_slope_regs(int n2, int lane, const doub
     return sxy / sxx;
 }
 
-// One new reading for module m, by one warp: Algorithm 1 on the context's state.
+// One warp: append reading P to a pair of windows kept oldest-first in memory (global or
+// shared), `len` entries each before the call, capacity W.  Eq. 2: the smoothed value is the
+// mean of the raw window after the append.  Returns the number of entries after the call and
+// the smoothed value and slope of this evaluation.
+__device__ __forceinline__ int window_push(double *raw, double *plist, int len, int W, double P, int lane,
+                                           double &pbar, double &slope) {
+    const bool drop = (len >= W);
+    const int n = drop ? W : len + 1;
+    if (drop) {  // the oldest entry leaves: shift both windows left by one, 32 entries at a time
+        for (int k0 = 0; k0 < W - 1; k0 += 32) {
+            const int k = k0 + lane;
+            double r = 0.0, q = 0.0;
+            if (k < W - 1) {
+                r = raw[k + 1];
+                q = plist[k + 1];
+            }
+            __syncwarp();
+            if (k < W - 1) {
+                raw[k] = r;
+                plist[k] = q;
+            }
+            __syncwarp();
+        }
+    }
+    if (lane == 0) raw[n - 1] = P;
+    __syncwarp();
+    double s = 0.0;
+    for (int k = lane; k < n; k += 32) s += raw[k];
+    pbar = warp_sum_f64(s) / (double)n;
+    if (lane == 0) plist[n - 1] = pbar;
+    __syncwarp();
+    slope = window_slope(n, lane, [&](int k) { return plist[k]; });
+    return n;
+}
+
+// Is evaluation i with this slope stale?  With the automatic tolerance the module's initial 3
+// readings (evaluations 0..2) only set it and are never stale.  NaN compares false: never stale.
+__device__ __forceinline__ bool rule_is_stale(double slope, int i, int flags, double T_fixed, double &Tauto,
+                                              double &smax) {
+    double T = T_fixed;
+    if (flags & kRuleAutoT) {
+        if (i <= 2) {
+            if (i >= 1 && fabs(slope) > smax) smax = fabs(slope);
+            if (i == 2) Tauto = 0.2 * smax;
+            return false;
+        }
+        T = Tauto;
+    }
+    return (flags & kRuleSigned) ? (slope < T) : (fabs(slope) < T);
+}
+
 // The two windows are kept oldest-first at fixed addresses, so for W <= 128 every load of the
 // step (counters, both windows, and both windows shifted by one for the case that the oldest
 // entry drops out) is issued at once: one memory round trip, then arithmetic in registers.
 struct StepLoaded {
     double ra[kStepRegs], rb[kStepRegs], pa[kStepRegs], pb[kStepRegs];
-    double slope, T;
+    double slope, T, Tauto, smax;
     int i, counter, freeze_eval;
 };
 
@@ -141,27 +159,30 @@ __device__ __forceinline__ StepLoaded plasticity_step_load(const SlopeState &st,
     L.counter = st.counter[m];
     L.freeze_eval = st.freeze_eval[m];
     L.slope = st.last_slope[m];
+    L.Tauto = st.Tauto[m];
+    L.smax = st.smax[m];
     L.T = (double)st.T[m];
     return L;
 }
 
-__device__ __forceinline__ void plasticity_step_apply(const SlopeState &st, StepLoaded &L, int m, int W,
-                                                      int signed_test, float reading, double *out_slopes,
-                                                      uint8_t *out_mask, int lane) {
+// One new reading for module m, by one warp: Algorithm 1 on the context's state.  Returns
+// whether the module is converged after this evaluation; `slope_out` is the slope of this
+// evaluation (the last one if the module had converged before).
+__device__ __forceinline__ bool plasticity_step_apply(const SlopeState &st, StepLoaded &L, int m, int W, int flags,
+                                                      float reading, int lane, double &slope_out) {
     double *raw = st.raw + (int64_t)m * st.W_cap, *plist = st.plist + (int64_t)m * st.W_cap;
     const bool fast = (W <= 32 * kStepRegs);
     double(&ra)[kStepRegs] = L.ra, (&rb)[kStepRegs] = L.rb, (&pa)[kStepRegs] = L.pa, (&pb)[kStepRegs] = L.pb;
     const int i = L.i;
     int counter = L.counter, freeze_eval = L.freeze_eval;
     double slope = L.slope;
-    const double T = L.T;
     __syncwarp();
     if (counter < W) {
         const int len = (i < W) ? i : W;       // entries in the windows now
-        const bool drop = (len == W);          // the oldest entry leaves
-        const int n = drop ? W : len + 1;      // entries after this reading: min(i + 1, W)
         const double P = (double)reading;
         if (fast) {
+            const bool drop = (len == W);      // the oldest entry leaves
+            const int n = drop ? W : len + 1;  // entries after this reading: min(i + 1, W)
             // windows after the update, in registers: element k = lane + 32 j
 #pragma unroll
             for (int j = 0; j < kStepRegs; ++j) {
@@ -187,32 +208,10 @@ __device__ __forceinline__ void plasticity_step_apply(const SlopeState &st, Step
                 }
             }
         } else {
-            if (drop) {  // shift both windows left by one, 32 entries at a time
-                for (int k0 = 0; k0 < W - 1; k0 += 32) {
-                    const int k = k0 + lane;
-                    double r = 0.0, q = 0.0;
-                    if (k < W - 1) {
-                        r = raw[k + 1];
-                        q = plist[k + 1];
-                    }
-                    __syncwarp();
-                    if (k < W - 1) {
-                        raw[k] = r;
-                        plist[k] = q;
-                    }
-                    __syncwarp();
-                }
-            }
-            if (lane == 0) raw[n - 1] = P;
-            __syncwarp();
-            double s = 0.0;
-            for (int k = lane; k < n; k += 32) s += raw[k];
-            const double pbar = warp_sum_f64(s) / (double)n;
-            if (lane == 0) plist[n - 1] = pbar;
-            __syncwarp();
-            slope = window_slope(n, lane, [&](int k) { return plist[k]; });
+            double pbar;
+            window_push(raw, plist, len, W, P, lane, pbar, slope);
         }
-        const bool stale = signed_test ? (slope < T) : (fabs(slope) < T);  // NaN compares false
+        const bool stale = rule_is_stale(slope, i, flags, L.T, L.Tauto, L.smax);
         counter = stale ? counter + 1 : 0;
         if (counter >= W && freeze_eval < 0) freeze_eval = i;
         if (lane == 0) {
@@ -220,48 +219,111 @@ __device__ __forceinline__ void plasticity_step_apply(const SlopeState &st, Step
             st.counter[m] = counter;
             st.freeze_eval[m] = freeze_eval;
             st.last_slope[m] = slope;
+            if (flags & kRuleAutoT) {
+                st.Tauto[m] = L.Tauto;
+                st.smax[m] = L.smax;
+            }
         }
     }
-    if (lane == 0) {
-        if (out_slopes) out_slopes[m] = slope;
-        if (out_mask) out_mask[m] = (counter >= W) ? 1 : 0;
-    }
+    slope_out = slope;
+    return counter >= W;
 }
 
-__device__ __forceinline__ void plasticity_step_module(const SlopeState &st, int m, int W, int signed_test,
-                                                       float reading, double *out_slopes, uint8_t *out_mask,
-                                                       int lane) {
-    StepLoaded L = plasticity_step_load(st, m, W, lane);
-    plasticity_step_apply(st, L, m, W, signed_test, reading, out_slopes, out_mask, lane);
+// One evaluation of the rule as module m's warp sees it (all modules' warps call this, each
+// with its own new reading).  Without the frontmost policy every module advances and reports
+// for itself.  With it, only the frontmost module that is not frozen advances; its warp (the
+// last module's when all are frozen) also reports for everybody: mask[j] = j is frozen,
+// slopes[j] = the slope of this evaluation for the monitored module, the final slope of a
+// frozen one, +inf for one that has not been monitored yet.  `parity` selects which of the
+// two front counters this evaluation reads; it writes the other, so that a module that
+// becomes the front during an evaluation starts with the next one.
+__device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepLoaded &L, int m, int M, int W,
+                                                     int flags, int parity, float reading, double *out_slopes,
+                                                     uint8_t *out_mask, int lane) {
+    if (!(flags & kRuleFrontmost)) {
+        double slope;
+        const bool conv = plasticity_step_apply(st, L, m, W, flags, reading, lane, slope);
+        if (lane == 0) {
+            if (out_slopes) out_slopes[m] = slope;
+            if (out_mask) out_mask[m] = conv ? 1 : 0;
+        }
+        return;
+    }
+    const int front = st.front[parity];
+    const int reporter = front < M ? front : M - 1;
+    if (m != reporter) return;
+    int front_new = front;
+    double slope = INFINITY;
+    if (front < M) {
+        const bool conv = plasticity_step_apply(st, L, m, W, flags, reading, lane, slope);
+        if (conv) front_new = front + 1;
+    }
+    if (lane == 0) st.front[parity ^ 1] = front_new;
+    for (int j = lane; j < M; j += 32) {
+        if (out_mask) out_mask[j] = (j < front_new) ? 1 : 0;
+        if (out_slopes) out_slopes[j] = (j == m && front < M) ? slope : (j < front ? st.last_slope[j] : INFINITY);
+    }
 }
 
 // One new reading per module.  grid = M warps (one 32-thread block each).
-__global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int M, int W, int signed_test,
+__global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int M, int W, int flags, int parity,
                                                              const float *losses, double *out_slopes,
                                                              uint8_t *out_mask) {
     const int m = blockIdx.x, lane = threadIdx.x;
     if (m >= M) return;
-    plasticity_step_module(st, m, W, signed_test, losses[m], out_slopes, out_mask, lane);
+    StepLoaded L = plasticity_step_load(st, m, W, lane);
+    plasticity_rule_step(st, L, m, M, W, flags, parity, losses[m], out_slopes, out_mask, lane);
 }
 
-// Whole histories from a cleared private state (rings in shared memory: 2 * W doubles).
-__global__ void __launch_bounds__(32) plasticity_replay_kernel(const float *T, int M, int W, int signed_test,
+// Whole histories from a cleared private state (windows in shared memory: 2 * W doubles).
+// Without the frontmost policy: one warp per module (grid = M).  With it: one warp in all
+// (grid = 1) walks the modules front to back.  out_slopes[m][i] is NaN where module m was
+// not advanced at evaluation i.
+__global__ void __launch_bounds__(32) plasticity_replay_kernel(const float *T, int M, int W, int flags,
                                                                const float *hist, int H, double *out_slopes,
                                                                uint8_t *out_mask, int32_t *out_freeze_eval) {
-    extern __shared__ double rings[];
-    double *raw = rings, *plist = rings + W;
-    const int m = blockIdx.x, lane = threadIdx.x;
+    extern __shared__ double windows[];
+    double *raw = windows, *plist = windows + W;
+    const int lane = threadIdx.x;
+    const bool frontmost = (flags & kRuleFrontmost) != 0;
+    int m = frontmost ? 0 : (int)blockIdx.x;
     if (m >= M) return;
-    int n_evals = 0, counter = 0, freeze_eval = -1;
-    const double Tm = (double)T[m];
-    for (int i = 0; i < H; ++i) {
-        double slope = NAN;
-        if (counter < W)
-            slope = plasticity_advance(raw, plist, n_evals, counter, freeze_eval, (double)hist[(int64_t)m * H + i],
-                                       W, Tm, signed_test != 0, lane);
-        if (out_slopes && lane == 0) out_slopes[(int64_t)m * H + i] = slope;
+    if (frontmost) {
+        for (int64_t k = lane; k < (int64_t)M * H; k += 32)
+            if (out_slopes) out_slopes[k] = NAN;
+        for (int j = lane; j < M; j += 32) {
+            if (out_mask) out_mask[j] = 0;
+            if (out_freeze_eval) out_freeze_eval[j] = -1;
+        }
+        __syncwarp();
     }
-    if (lane == 0) {
+    int len = 0, n_evals = 0, counter = 0, freeze_eval = -1;
+    double Tauto = NAN, smax = 0.0;
+    for (int i = 0; i < H && m < M; ++i) {
+        double slope = NAN;
+        if (counter < W) {
+            double pbar;
+            len = window_push(raw, plist, len, W, (double)hist[(int64_t)m * H + i], lane, pbar, slope);
+            const bool stale = rule_is_stale(slope, n_evals, flags, (double)T[m], Tauto, smax);
+            counter = stale ? counter + 1 : 0;
+            if (counter >= W) freeze_eval = i;
+            ++n_evals;
+        }
+        if (out_slopes && lane == 0) out_slopes[(int64_t)m * H + i] = slope;
+        if (frontmost && counter >= W) {  // frozen: the next evaluation starts the next module afresh
+            if (lane == 0) {
+                if (out_mask) out_mask[m] = 1;
+                if (out_freeze_eval) out_freeze_eval[m] = freeze_eval;
+            }
+            ++m;
+            len = n_evals = counter = 0;
+            freeze_eval = -1;
+            Tauto = NAN;
+            smax = 0.0;
+            __syncwarp();
+        }
+    }
+    if (!frontmost && lane == 0) {
         if (out_mask) out_mask[m] = (counter >= W) ? 1 : 0;
         if (out_freeze_eval) out_freeze_eval[m] = freeze_eval;
     }
@@ -269,11 +331,77 @@ __global__ void __launch_bounds__(32) plasticity_replay_kernel(const float *T, i
 
 __global__ void plasticity_clear_kernel(SlopeState st, int M) {
     const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m < 2) st.front[m] = 0;
     if (m >= M) return;
     st.n_evals[m] = 0;
     st.counter[m] = 0;
     st.freeze_eval[m] = -1;
     st.last_slope[m] = INFINITY;
+    st.Tauto[m] = NAN;
+    st.smax[m] = 0.0;
+}
+
+// ------------------------------------------------------------------------------------------
+// End of the bootstrapping stage (Sec. 3; the 10 % of Sec. 4.2.2): the training loss is
+// smoothed and fitted like the plasticity; with a full window of W smoothed values, slope s
+// and window mean ybar, the changing rate is |s| (W - 1) / |ybar|, and the stage ends at the
+// first evaluation whose rate is below the tolerance.
+// ------------------------------------------------------------------------------------------
+struct BootState {
+    double *raw;       // [W_cap] raw training losses, oldest first
+    double *plist;     // [W_cap] smoothed ones
+    int32_t *n_evals;  // [1]
+    int32_t *end;      // [1] evaluation at which the stage ended, -1 while it lasts
+};
+
+// One warp: one more training loss.  Returns the changing rate of this evaluation (NaN before
+// the window is full and after the end); `end` is updated.
+__device__ __forceinline__ double bootstrap_advance(double *raw, double *plist, int &n_evals, int &end, double loss,
+                                                    int W, double rate_tol, int lane) {
+    if (end >= 0) return NAN;
+    const int len = n_evals < W ? n_evals : W;
+    double pbar, slope;
+    const int n = window_push(raw, plist, len, W, loss, lane, pbar, slope);
+    const int i = n_evals++;
+    if (n < W) return NAN;
+    double sy = 0.0;
+    for (int k = lane; k < W; k += 32) sy += plist[k];
+    const double ybar = warp_sum_f64(sy) / (double)W;
+    const double rate = fabs(slope) * (double)(W - 1) / fabs(ybar);
+    if (rate < rate_tol) end = i;
+    return rate;
+}
+
+__global__ void __launch_bounds__(32) bootstrap_step_kernel(BootState bs, int W, double rate_tol, const float *loss,
+                                                            double *out_rate, uint8_t *out_done) {
+    const int lane = threadIdx.x;
+    int n_evals = *bs.n_evals, end = *bs.end;
+    __syncwarp();
+    const double rate = bootstrap_advance(bs.raw, bs.plist, n_evals, end, (double)*loss, W, rate_tol, lane);
+    if (lane == 0) {
+        *bs.n_evals = n_evals;
+        *bs.end = end;
+        if (out_rate) *out_rate = rate;
+        if (out_done) *out_done = end >= 0 ? 1 : 0;
+    }
+}
+
+// A whole training-loss history from a cleared private state (2 * W doubles of shared memory).
+__global__ void __launch_bounds__(32) bootstrap_replay_kernel(int W, double rate_tol, const float *hist, int H,
+                                                              double *out_rates, int32_t *out_end) {
+    extern __shared__ double windows[];
+    const int lane = threadIdx.x;
+    int n_evals = 0, end = -1;
+    for (int i = 0; i < H; ++i) {
+        const double rate = bootstrap_advance(windows, windows + W, n_evals, end, (double)hist[i], W, rate_tol, lane);
+        if (out_rates && lane == 0) out_rates[i] = rate;
+    }
+    if (out_end && lane == 0) *out_end = end;
+}
+
+__global__ void bootstrap_clear_kernel(BootState bs) {
+    *bs.n_evals = 0;
+    *bs.end = -1;
 }
 
 }  // namespace egeria

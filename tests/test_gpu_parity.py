@@ -404,6 +404,177 @@ def test_step_with_a_window_too_long_for_registers():
     ctx.close()
 
 
+# ----------------------------------------------------------------------------- policies around Algorithm 1
+
+def _policy_histories(M, H, seed):
+    rng = np.random.default_rng(seed)
+    k = np.arange(H)
+    return np.stack([0.3 * np.exp(-k / rng.uniform(2, 12)) * (1 + 0.2 * np.sin(0.9 * k + m)) + 0.01 * (m + 1)
+                     + 1e-4 * rng.standard_normal(H) for m in range(M)]).astype(np.float32)
+
+
+def _near_T(slopes, T):
+    s = slopes[np.isfinite(slopes)]
+    return bool(np.any(np.abs(np.abs(s) - T) <= 1e-6))
+
+
+@pytest.mark.parametrize("W", [3, 10, 150])
+def test_auto_tolerance_matches_oracle(W):
+    M, H = 5, 420 if W > 100 else 90
+    hist = _policy_histories(M, H, seed=W)
+    ctx = eg.Context([64] * M, 8, W, 1.0, eg.FLAG_AUTO_T, device=DEV)      # the T given is ignored
+    hist_dev = torch.from_numpy(hist).to(DEV)
+    r_slopes, r_mask, r_fe = [t.cpu().numpy() for t in ctx.egeria_plasticity_replay(hist_dev)]
+    step_masks = np.empty((M, H), dtype=np.uint8)
+    step_slopes = np.empty((M, H))
+    for i in range(H):
+        s, mk = ctx.egeria_plasticity_step(hist_dev[:, i].contiguous())
+        step_slopes[:, i], step_masks[:, i] = s.cpu().numpy(), mk.cpu().numpy()
+    for m in range(M):
+        ref = oracle.plasticity_replay_auto(hist[m], W)
+        live = ~np.isnan(ref["slopes"])
+        assert np.array_equal(np.isnan(r_slopes[m]), ~live)
+        fin = live & np.isfinite(ref["slopes"])
+        np.testing.assert_allclose(r_slopes[m][fin], ref["slopes"][fin], rtol=1e-9, atol=1e-15)
+        np.testing.assert_allclose(step_slopes[m][fin], ref["slopes"][fin], rtol=1e-9, atol=1e-15)
+        if not (np.isfinite(ref["T"]) and _near_T(ref["slopes"], ref["T"])):
+            assert int(r_fe[m]) == ref["freeze_eval"]
+            assert bool(r_mask[m]) == ref["converged"]
+            want = np.zeros(H, dtype=np.uint8)
+            if ref["converged"]:
+                want[ref["freeze_eval"]:] = 1
+            assert np.array_equal(step_masks[m], want)
+    ctx.close()
+
+
+@pytest.mark.parametrize("auto,H", [(False, 45), (True, 100)])
+def test_frontmost_policy_matches_oracle(auto, H):
+    M, W = 6, 4
+    hist = _policy_histories(M, H, seed=77 + auto)
+    T = np.linspace(4e-3, 1.2e-2, M).astype(np.float32)
+    flags = eg.FLAG_FRONTMOST | (eg.FLAG_AUTO_T if auto else 0)
+    ctx = eg.Context([64] * M, 8, W, T, flags, device=DEV)
+    ref = oracle.frontmost_replay(hist, W, None if auto else T.astype(np.float64))
+    assert 1 <= ref["frozen"] < M                              # the case is not a trivial one
+    hist_dev = torch.from_numpy(hist).to(DEV)
+    slopes, mask, fe = [t.cpu().numpy() for t in ctx.egeria_plasticity_replay(hist_dev)]
+    assert fe.tolist() == ref["freeze_eval"].tolist()
+    assert mask.tolist() == [1] * ref["frozen"] + [0] * (M - ref["frozen"])
+    for i in range(H):
+        l = ref["monitored"][i]
+        for m in range(M):
+            if m == l:
+                if np.isfinite(ref["slopes"][i]):
+                    assert slopes[m, i] == pytest.approx(ref["slopes"][i], rel=1e-9, abs=1e-15)
+                else:
+                    assert np.isinf(slopes[m, i])
+            else:
+                assert np.isnan(slopes[m, i])
+    # the same through one evaluation at a time: prefix mask, slope of the monitored module
+    for i in range(H):
+        s, mk = ctx.egeria_plasticity_step(hist_dev[:, i].contiguous())
+        s, mk = s.cpu().numpy(), mk.cpu().numpy()
+        frozen_after = int(np.sum((ref["freeze_eval"] >= 0) & (ref["freeze_eval"] <= i)))
+        assert mk.tolist() == [1] * frozen_after + [0] * (M - frozen_after)
+        l = ref["monitored"][i]
+        if np.isfinite(ref["slopes"][i]):
+            assert s[l] == pytest.approx(ref["slopes"][i], rel=1e-9, abs=1e-15)
+        assert np.all(np.isinf(s[l + 1:]))
+    ctx.close()
+
+
+def test_frontmost_policy_inside_the_fused_evaluation():
+    """egeria_plasticity_evaluate with the frontmost policy: same decisions as the losses fed to
+    egeria_plasticity_step of a second context."""
+    ds, b, W = [4096, 2048, 1001, 8192], 40, 2
+    flags = eg.FLAG_FRONTMOST | eg.FLAG_EQUAL_SPLIT
+    fused = eg.Context(ds, b, W, 0.5, flags, device=DEV)       # a generous T: modules freeze quickly
+    split = eg.Context(ds, b, W, 0.5, flags, device=DEV)
+    seen = []
+    for k in range(12):
+        at, ar = [], []
+        for m, d in enumerate(ds):
+            t, r = wl.make_pair(b, d, "relu", 0.3, seed=800 + 10 * k + m, device=DEV)
+            at.append(t)
+            ar.append(r)
+        l1, s1, m1 = fused.egeria_plasticity_evaluate(at, ar)
+        l2 = split.egeria_sp_loss_batch(at, ar)
+        s2, m2 = split.egeria_plasticity_step(l2)
+        assert l1.cpu().numpy().tobytes() == l2.cpu().numpy().tobytes()
+        assert s1.cpu().numpy().tobytes() == s2.cpu().numpy().tobytes()
+        assert m1.cpu().numpy().tobytes() == m2.cpu().numpy().tobytes()
+        seen.append(int(m1.sum()))
+    assert seen == sorted(seen) and seen[-1] == len(ds) and seen[0] == 0   # froze front to back, all of them
+    fused.close()
+    split.close()
+
+
+def test_bootstrap_detector_matches_oracle():
+    rng = np.random.default_rng(11)
+    H, W = 120, 8
+    loss = (2.5 * np.exp(-np.arange(H) / 15.0) + 0.4 + 0.01 * rng.standard_normal(H)).astype(np.float32)
+    ctx = eg.Context([64], 8, W, 1e-3, device=DEV)
+    for tol in (0.1, 0.02):
+        ref = oracle.bootstrap_replay(loss, W, tol)
+        assert 2 * W < ref["end"] < H - 5
+        rates, end = ctx.egeria_bootstrap_replay(torch.from_numpy(loss).to(DEV), tol)
+        rates = rates.cpu().numpy()
+        near = np.nanmin(np.abs(ref["rates"] - tol)) < 1e-9
+        if not near:
+            assert int(end.cpu()[0]) == ref["end"]
+        live = ~np.isnan(ref["rates"])
+        assert np.array_equal(np.isnan(rates), ~live)
+        np.testing.assert_allclose(rates[live], ref["rates"][live], rtol=1e-9)
+        # one reading at a time
+        ctx.egeria_bootstrap_reset()
+        dev = torch.from_numpy(loss).to(DEV)
+        ended = -1
+        for i in range(H):
+            rate, done = ctx.egeria_bootstrap_step(dev[i:i + 1], tol)
+            if live[i]:
+                assert float(rate.cpu()[0]) == pytest.approx(ref["rates"][i], rel=1e-9)
+            if ended < 0 and int(done.cpu()[0]):
+                ended = i
+        if not near:
+            assert ended == ref["end"]
+    ctx.close()
+
+
+def test_state_export_import_resumes_the_same_decisions():
+    M, H, W = 4, 60, 5
+    hist = _policy_histories(M, H, seed=5)
+    dev = torch.from_numpy(hist).to(DEV)
+    flags = eg.FLAG_AUTO_T
+    a = eg.Context([64] * M, 8, W, 1e-3, flags, device=DEV)
+    full = []
+    for i in range(H):
+        s, mk = a.egeria_plasticity_step(dev[:, i].contiguous())
+        full.append((s.cpu().numpy().copy(), mk.cpu().numpy().copy()))
+        if i == 22:
+            a.egeria_bootstrap_step(dev[0, i:i + 1])
+            saved = a.egeria_plasticity_export()
+    assert saved.nbytes == a.egeria_plasticity_state_bytes()
+    b2 = eg.Context([64] * M, 8, W, 1e-3, flags, device=DEV)
+    b2.egeria_plasticity_import(saved)
+    for i in range(23, H):
+        s, mk = b2.egeria_plasticity_step(dev[:, i].contiguous())
+        assert s.cpu().numpy().tobytes() == full[i][0].tobytes()
+        assert mk.cpu().numpy().tobytes() == full[i][1].tobytes()
+    # a context with another window, module count or rule refuses the buffer
+    for other in (eg.Context([64] * M, 8, W + 1, 1e-3, flags, device=DEV),
+                  eg.Context([64] * (M + 1), 8, W, 1e-3, flags, device=DEV),
+                  eg.Context([64] * M, 8, W, 1e-3, 0, device=DEV)):
+        with pytest.raises(eg.EgeriaError) as e:
+            other.egeria_plasticity_import(saved)
+        assert e.value.status == eg.ERR_INVALID_ARG
+        other.close()
+    with pytest.raises(eg.EgeriaError) as e:
+        b2.egeria_plasticity_import(saved[:-8])
+    assert e.value.status == eg.ERR_WORKSPACE
+    a.close()
+    b2.close()
+
+
 def test_alg1_hand_traces_on_gpu():
     from fractions import Fraction
     for line in (GOLDEN / "alg1_traces.txt").read_text().splitlines():
