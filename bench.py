@@ -3,9 +3,9 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-A step is one pass of the whole path over one synthetic mini-batch: egeria_plasticity_evaluate
-(Gram kernel, then the finalisation kernel that also advances the freezing rule).  Prints ONE
-JSON line.
+A step is one pass of the whole path over one synthetic mini-batch: egeria_plasticity_evaluate,
+which is ONE kernel launch (Gram matrices on the tensor cores, then row normalisation,
+difference, Frobenius reduction and the freezing rule by the same kernel).  Prints ONE JSON line.
 With N > 1 (torchrun) every rank evaluates its own replica of the workload on its own
 GPU; there is no data-path collective.
 """
@@ -32,6 +32,11 @@ METRIC = "module-evals/s (SP loss, all modules)"
 UNIT = "module-evals/s"
 PEAKS_FILE = ROOT / "MEASURED_PEAKS.json"
 FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the evaluation kernel, from the ncu
+# captures summarised under profiles/ (gpt2_medium: a 6-module launch scaled x4 by the modules
+# processed).  Valid for the kernel as captured; set to None when the kernel changes.
+NCU_TRAFFIC_BYTES = {"gpt2_medium": None, "resnet50": None}
 
 
 # ----------------------------------------------------------------------------- helpers
@@ -337,9 +342,10 @@ def run_ours(args):
     peak, peak_kind = hbm_peak()
     gram_s = (gram_ms / max(1, gram_calls)) * 1e-3
     achieved = w.input_bytes / gram_s / 1e9 if gram_s > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "gram_tc_kernel", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "gram_tc_kernel (Gram + finalisation + freezing rule)", "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "algorithmic_bytes_per_launch": w.input_bytes,
+                "traffic": NCU_TRAFFIC_BYTES.get(w.name) if not args.modules else None,
+                "algorithmic_bytes_per_launch": w.input_bytes,
                 "avg_launch_ms": gram_s * 1e3, "launches_timed": gram_calls}
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
