@@ -106,6 +106,32 @@ def test_many_modules_mixed_sizes(b):
     compare_with_oracle(at, ar, what=f"mixed b={b}")
 
 
+@pytest.mark.parametrize("b", [5, 33, 70, 130])
+def test_hundreds_of_small_modules(b):
+    """More modules than CTAs: whole modules inside one CTA's range, many units per CTA, the scan
+    over other modules longer than one warp, a few CUDA-core modules in between; evaluated
+    repeatedly (the progress counters alternate between two sets)."""
+    rng = np.random.default_rng(b)
+    M = 200
+    ds = [int(rng.integers(1, 200)) * 8 for _ in range(M)]
+    for m in (3, 77, 150):
+        ds[m] += 3                                           # not a multiple of 8: CUDA-core path
+    at, ar = [], []
+    for m, d in enumerate(ds):
+        t, r = wl.make_pair(b, d, "relu" if m % 3 else "normal", 0.02 + 0.002 * m, seed=5000 + m, device=DEV)
+        at.append(t)
+        ar.append(r)
+    ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+    ctx = eg.Context(ds, b, 4, 1e-3, device=DEV)
+    for rep in range(3):
+        losses, slopes, mask = ctx.egeria_plasticity_evaluate(at, ar)
+        assert_loss_close(losses.cpu().numpy(), ref, f"many modules b={b} rep={rep}")
+    ctx.check_device_status()
+    # three identical readings per module: slope 0 from the second on, not yet frozen (W = 4)
+    assert np.all(slopes.cpu().numpy() == 0.0) and not mask.cpu().numpy().any()
+    ctx.close()
+
+
 # ----------------------------------------------------------------------------- closed forms / invariants on the GPU
 
 def _fixture_cases():
