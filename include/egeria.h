@@ -58,8 +58,9 @@ enum {
     EGERIA_FLAG_KEEP_GRAMS = 4u,
     /* Reserve device staging for egeria_sp_loss_batch_host in the workspace. */
     EGERIA_FLAG_HOST_STAGING = 8u,
-    /* Record a CUDA event before and after the Gram kernel(s) of every
-     * egeria_sp_loss_batch call, for egeria_gram_kernel_time. */
+    /* Record a CUDA event before and after the evaluation kernel(s) of every
+     * egeria_sp_loss_batch / egeria_plasticity_evaluate call, for
+     * egeria_gram_kernel_time. */
     EGERIA_FLAG_TIME_GRAM = 16u,
     /* Always cut the work into equal shares.  Without this flag the first
      * evaluations of a context that keep every SM busy report how fast each
@@ -283,9 +284,12 @@ egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At, const voi
                                     int64_t d, float *out_loss);
 
 /* Measurement hook (needs EGERIA_FLAG_TIME_GRAM): device time, in milliseconds,
- * spent in the Gram kernels of the egeria_sp_loss_batch calls made since the
- * last query (the finalisation kernel is not included), and the number of those
- * calls.  Waits for the last recorded event.  Resets the tally. */
+ * spent in the evaluation kernels of the egeria_sp_loss_batch /
+ * egeria_plasticity_evaluate calls made since the last query (for tensor-core
+ * modules that is the whole evaluation; the separate finalisation kernel of
+ * CUDA-core modules is not included), and the number of those calls; at most
+ * 4096 calls between two queries are timed.  Waits for the last recorded event.
+ * Resets the tally. */
 egeria_status egeria_gram_kernel_time(egeria_ctx *ctx, double *total_ms, int64_t *n_calls);
 
 /* Number of kernels the library has launched through this context so far. */

@@ -21,6 +21,7 @@ constexpr int kMaxCtas = 160;  // sizing bound for the work split (a B200 has 14
 constexpr int kMaxW = 2048;    // replay keeps 2 * W doubles in shared memory
 constexpr int kPlanSlots = 16; // device-side plans kept, keyed by (b, activation pointers)
 constexpr int kCalibLaunches = 3;  // launches whose per-CTA streaming rates set the split weights
+constexpr size_t kMaxTimedCalls = 4096;  // EGERIA_FLAG_TIME_GRAM: calls timed between two queries
 constexpr int kCalibRounds = 3;    // times the weights are re-measured under the split they produced
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -151,7 +152,8 @@ struct egeria_ctx {
     int cur = 0;           // entry the last egeria_sp_loss_batch used
     int plan_b = -1;       // its b
     uint64_t use_clock = 0;
-    std::vector<uint8_t> pack;  // host image of one plan region
+    std::vector<uint8_t> pack;  // host image of one plan region (when there is no pinned one)
+    uint8_t *pinned_plans = nullptr;  // kPlanSlots images of plan_stride bytes: uploads that do not stall the stream
     uint8_t *plan_region(int i) const { return ws + L.plan0 + (size_t)i * L.plan_stride; }
     cudaStream_t last_stream = nullptr;
     int64_t launches = 0;
@@ -316,6 +318,13 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     std::vector<float> Th(M);
     for (int m = 0; m < M; ++m) Th[m] = T ? T[m] : T_all;
     ctx->weights.assign(ctx->n_ctas, 1.0f);
+    {
+        void *hp = nullptr;
+        if (cudaHostAlloc(&hp, L.plan_stride * kPlanSlots, cudaHostAllocDefault) == cudaSuccess)
+            ctx->pinned_plans = static_cast<uint8_t *>(hp);
+        else
+            (void)cudaGetLastError();  // fall back to pageable staging
+    }
     if (!(flags & EGERIA_FLAG_EQUAL_SPLIT)) {
         void *hp = nullptr;
         if (cudaHostAlloc(&hp, sizeof(CtaLog) * kCalibLaunches * kMaxCtas, cudaHostAllocDefault) == cudaSuccess) {
@@ -338,6 +347,7 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     }
     if (e != cudaSuccess) {
         if (ctx->host_log) cudaFreeHost(ctx->host_log);
+        if (ctx->pinned_plans) cudaFreeHost(ctx->pinned_plans);
         delete ctx;
         return EGERIA_ERR_CUDA;
     }
@@ -349,6 +359,7 @@ egeria_status egeria_plasticity_destroy(egeria_ctx *ctx) {
     if (!ctx) return EGERIA_ERR_INVALID_ARG;
     for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
     if (ctx->host_log) cudaFreeHost(ctx->host_log);
+    if (ctx->pinned_plans) cudaFreeHost(ctx->pinned_plans);
     delete ctx;
     return EGERIA_OK;
 }
@@ -448,8 +459,16 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
         L.units + P.units.size() * sizeof(Unit) > L.cta_begin_tc)
         return EGERIA_ERR_WORKSPACE;
 
-    ctx->pack.assign(L.plan_stride, 0);
-    uint8_t *img = ctx->pack.data();
+    uint8_t *img;
+    if (ctx->pinned_plans) {
+        // One pinned image per plan slot: the copy below is truly asynchronous, and an image is not
+        // written again before its slot is replaced, i.e. after at least kPlanSlots - 1 other uploads.
+        img = ctx->pinned_plans + (size_t)lru * L.plan_stride;
+        memset(img, 0, L.plan_stride);
+    } else {
+        ctx->pack.assign(L.plan_stride, 0);
+        img = ctx->pack.data();
+    }
     const int box_rows = pitch_of_mode(P.mode);  // rows of one TMA box: all rows of one side
     CUtensorMap *maps = reinterpret_cast<CUtensorMap *>(img + L.tmaps);
     ModulePtrs *mods = reinterpret_cast<ModulePtrs *>(img + L.modules);
@@ -464,7 +483,7 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
     memcpy(img + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t));
     memcpy(img + L.cta_begin_simt, P.cta_begin_simt.data(), P.cta_begin_simt.size() * sizeof(int32_t));
     memcpy(img + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo));
-    // One copy from pageable memory: the runtime stages it before returning, so `pack` may be reused.
+    // From pageable memory the runtime stages the bytes before returning, so `pack` may be reused.
     EG_CUDA(cudaMemcpyAsync(ctx->plan_region(lru), img, L.plan_stride, cudaMemcpyHostToDevice, stream));
     e.b = b;
     e.weights_version = ctx->weights_version;
@@ -552,7 +571,7 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
     const uint8_t *region = ctx->plan_region(ctx->cur);
     const int64_t slot_floats = slot_floats_of_mode(P.mode);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    if (ctx->flags & EGERIA_FLAG_TIME_GRAM) {
+    if ((ctx->flags & EGERIA_FLAG_TIME_GRAM) && ctx->ev_used < kMaxTimedCalls * 2) {
         if (ctx->ev_used + 2 > ctx->ev_pool.size()) {
             cudaEvent_t a, c;
             EG_CUDA(cudaEventCreate(&a));
