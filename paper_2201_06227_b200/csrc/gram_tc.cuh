@@ -50,9 +50,11 @@ struct TcCfg {
     static constexpr int kBoxRows = (MODE == kStacked32) ? 32 : (MODE == kStacked64 ? 64 : (MODE == kSingle1 ? 128 : 256));
     static constexpr int kSlabRows = kStacked ? 2 * kBoxRows : kBoxRows;   // rows of one 64-column slab
     static constexpr int kSlabBytes = kSlabRows * 128;
-    static constexpr int kKbPerStage = (MODE == kStacked32) ? 2 : 1;       // slabs per pipeline stage
-    static constexpr int kStageBytes = kSlabBytes * kKbPerStage;           // 16 KB (32 KB for b > 128)
-    static constexpr int kStages = (MODE == kSingle2) ? 6 : 12;            // 192 KB of loads in flight
+    // Slabs per pipeline stage.  The 8 KB slabs of kStacked32 go six to a stage: with 16 KB stages
+    // the per-stage hand-shakes (not the loads) set the pace there, 20 % slower on 150 MB of input.
+    static constexpr int kKbPerStage = (MODE == kStacked32) ? 6 : 1;
+    static constexpr int kStageBytes = kSlabBytes * kKbPerStage;           // 48 KB, 16 KB, 16 KB, 32 KB
+    static constexpr int kStages = (MODE == kStacked32) ? 4 : (MODE == kSingle2 ? 6 : 12);  // 192 KB of loads in flight
     // kStacked32 issues M = 128 MMAs over a 64-row slab: the A operand reaches one slab further.
     static constexpr int kPadBytes = (MODE == kStacked32) ? kSlabBytes : 0;
     static constexpr int kAccCols = (MODE == kStacked32) ? 64 : (MODE == kSingle2 ? 384 : 128);
