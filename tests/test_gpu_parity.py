@@ -132,6 +132,37 @@ def test_hundreds_of_small_modules(b):
     ctx.close()
 
 
+@pytest.mark.parametrize("seed", range(4))
+def test_random_shapes_repeat_bit_for_bit(seed):
+    """Random b, module counts and sizes; six evaluations each: every one within tolerance of the
+    oracle, and with the equal split all six bit-identical (the in-kernel finalisation must not
+    depend on which CTA or warp did what)."""
+    rng = np.random.default_rng(900 + seed)
+    for _ in range(10):
+        b = int(rng.choice([2, 7, 16, 31, 32, 33, 48, 64, 65, 100, 128, 129, 192, 256]))
+        M = int(rng.choice([1, 2, 5, 13, 40]))
+        top = 4000 if rng.random() < 0.3 else 300
+        ds = [int(rng.integers(1, top)) * 8 for _ in range(M)]
+        if M > 2 and rng.random() < 0.3:
+            ds[int(rng.integers(M))] += 5                    # one CUDA-core module
+        if b >= 128 and M >= 40:
+            ds = [min(d, 2048) for d in ds]                  # keeps the oracle quick
+        at, ar = [], []
+        for m, d in enumerate(ds):
+            t, r = wl.make_pair(b, d, "relu" if m % 2 else "normal", 0.02 + 0.3 * rng.random(),
+                                seed=int(rng.integers(1 << 30)), device=DEV)
+            at.append(t)
+            ar.append(r)
+        ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+        ctx = eg.Context(ds, b, 4, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
+        outs = [ctx.egeria_plasticity_evaluate(at, ar)[0].cpu().numpy().copy() for _ in range(6)]
+        ctx.check_device_status()
+        ctx.close()
+        for o in outs:
+            assert_loss_close(o, ref, f"random b={b} M={M}")
+            assert o.tobytes() == outs[0].tobytes()
+
+
 # ----------------------------------------------------------------------------- closed forms / invariants on the GPU
 
 def _fixture_cases():
