@@ -168,6 +168,26 @@ egeria_status egeria_plasticity_evaluate(egeria_ctx *ctx, void *cuda_stream, con
                                          const void *const *Ar, int b, const int64_t *d,
                                          float *out_losses, double *out_slopes, uint8_t *out_mask);
 
+/* The two calls above for a SUBSET of the modules: active is a host uint8 [M];
+ * modules with active[m] == 0 are left out -- their pointers are not read (may be
+ * NULL), no work is done for them, their entries of out_losses, out_slopes and
+ * out_mask are not written and their freezing rule does not advance.  The work of
+ * the active modules is spread over the whole GPU, so evaluating one module of
+ * many costs about its share.  This is how the frontmost-active policy is meant
+ * to be used [Sec. 3: "collects the intermediate activation of the frontmost
+ * non-frozen layer"]: read out_mask back now and then and pass only the frontmost
+ * module that is not frozen (under EGERIA_FLAG_FRONTMOST that module reports the
+ * prefix mask and the slopes of all modules; if it is left out, or all modules
+ * are frozen, nothing is reported).  At least one module must be active. */
+egeria_status egeria_sp_loss_subset(egeria_ctx *ctx, void *cuda_stream, const void *const *At,
+                                    const void *const *Ar, int b, const int64_t *d,
+                                    const uint8_t *active, float *out_losses);
+egeria_status egeria_plasticity_evaluate_subset(egeria_ctx *ctx, void *cuda_stream,
+                                                const void *const *At, const void *const *Ar, int b,
+                                                const int64_t *d, const uint8_t *active,
+                                                float *out_losses, double *out_slopes,
+                                                uint8_t *out_mask);
+
 /* The same rule over whole histories, from a cleared state that is private to
  * the call (the context's step state is not touched).
  *   hist             device float [M, H] row-major raw readings

@@ -31,6 +31,7 @@ EXPORTS = [
     "egeria_gram_kernel_time", "egeria_sp_loss_static", "egeria_plasticity_evaluate",
     "egeria_split_weights", "egeria_status_string", "egeria_bootstrap_step", "egeria_bootstrap_replay",
     "egeria_bootstrap_reset", "egeria_plasticity_state_bytes", "egeria_plasticity_export", "egeria_plasticity_import",
+    "egeria_sp_loss_subset", "egeria_plasticity_evaluate_subset",
 ]
 
 
@@ -63,6 +64,10 @@ def lib() -> ctypes.CDLL:
     L.egeria_plasticity_step.argtypes = [vp, vp, vp, vp, vp]
     L.egeria_plasticity_evaluate.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, i64p,
                                              vp, vp, vp]
+    L.egeria_sp_loss_subset.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, i64p,
+                                        ctypes.POINTER(ctypes.c_uint8), vp]
+    L.egeria_plasticity_evaluate_subset.argtypes = [vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int, i64p,
+                                                    ctypes.POINTER(ctypes.c_uint8), vp, vp, vp]
     L.egeria_plasticity_replay.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp]
     L.egeria_plasticity_reset.argtypes = [vp, vp, ctypes.c_int]
     L.egeria_plasticity_window.argtypes = [vp]
@@ -207,11 +212,14 @@ class Context:
             pass
 
     # ------------------------------------------------------------------ calls
-    def _ptr_array(self, tensors: Sequence[torch.Tensor], b: int, on_device: bool):
+    def _ptr_array(self, tensors: Sequence[torch.Tensor], b: int, on_device: bool, active=None):
         if len(tensors) != self.M:
             raise ValueError("one activation per module is required")
         ptrs = (ctypes.c_void_p * self.M)()
         for m, t in enumerate(tensors):
+            if active is not None and not active[m]:
+                ptrs[m] = None
+                continue
             if t.dtype != torch.bfloat16 or t.shape != (b, self.d[m]) or not t.is_contiguous():
                 raise ValueError(f"module {m}: expected contiguous bfloat16 [{b}, {self.d[m]}]")
             if t.is_cuda != on_device:
@@ -230,6 +238,29 @@ class Context:
                                         out_losses.data_ptr())
         _check(st, "egeria_sp_loss_batch")
         return out_losses
+
+    def egeria_sp_loss_subset(self, At, Ar, active, out_losses: torch.Tensor,
+                              stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """SP loss of the modules with active[m] != 0 only; the other entries of out_losses stay."""
+        act = np.ascontiguousarray(active, dtype=np.uint8)
+        b = int(next((t for t, a in zip(At, act) if a), next(t for t in At if t is not None)).shape[0])
+        pa, pr = self._ptr_array(At, b, True, act), self._ptr_array(Ar, b, True, act)
+        st = lib().egeria_sp_loss_subset(self._h, _stream_ptr(stream), pa, pr, b, self._d_arr,
+                                         act.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)), out_losses.data_ptr())
+        _check(st, "egeria_sp_loss_subset")
+        return out_losses
+
+    def egeria_plasticity_evaluate_subset(self, At, Ar, active, losses: torch.Tensor, slopes: torch.Tensor,
+                                          mask: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+        """One evaluation (loss + freezing rule) of the active modules only, into the caller's tensors."""
+        act = np.ascontiguousarray(active, dtype=np.uint8)
+        b = int(next((t for t, a in zip(At, act) if a), next(t for t in At if t is not None)).shape[0])
+        pa, pr = self._ptr_array(At, b, True, act), self._ptr_array(Ar, b, True, act)
+        st = lib().egeria_plasticity_evaluate_subset(self._h, _stream_ptr(stream), pa, pr, b, self._d_arr,
+                                                     act.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)),
+                                                     losses.data_ptr(), slopes.data_ptr(), mask.data_ptr())
+        _check(st, "egeria_plasticity_evaluate_subset")
+        return losses, slopes, mask
 
     def egeria_plasticity_evaluate(self, At: Sequence[torch.Tensor], Ar: Sequence[torch.Tensor],
                                    stream: Optional[torch.cuda.Stream] = None):

@@ -83,7 +83,7 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
     L.last_slope = take((size_t)M * sizeof(double));
     L.Tauto = take((size_t)M * sizeof(double));
     L.smax = take((size_t)M * sizeof(double));
-    L.front = take(2 * sizeof(int32_t));
+    L.front = take(sizeof(unsigned long long));
     L.boot_raw = take((size_t)W * sizeof(double));
     L.boot_plist = take((size_t)W * sizeof(double));
     L.boot_ints = take(2 * sizeof(int32_t));
@@ -158,7 +158,7 @@ struct egeria_ctx {
     cudaStream_t last_stream = nullptr;
     int64_t launches = 0;
     uint32_t tc_launches = 0;  // selects the set of progress counters the next tensor-core launch uses
-    uint32_t rule_evals = 0;   // evaluations of the freezing rule enqueued: its parity selects the front counter
+    uint32_t rule_evals = 0;   // evaluations of the freezing rule enqueued so far (the serial of the last one)
     // Split weights: one per CTA, from the streaming rates the CTAs report (SMs do not all get
     // the same share of HBM bandwidth; the CTA -> SM placement repeats from launch to launch).
     std::vector<float> weights;
@@ -169,6 +169,7 @@ struct egeria_ctx {
     uint32_t calib_serial[kCalibLaunches] = {};
     CtaLog *host_log = nullptr;  // pinned, kCalibLaunches x kMaxCtas
     std::vector<void *> staging_t, staging_r;
+    std::vector<const void *> subset_t, subset_r;  // pointer arrays of a subset call (left-out modules nulled)
     // EGERIA_FLAG_TIME_GRAM: event pairs around the Gram kernel launches since the last query
     std::vector<cudaEvent_t> ev_pool;
     size_t ev_used = 0;
@@ -199,7 +200,7 @@ struct egeria_ctx {
         st.last_slope = at<double>(L.last_slope);
         st.Tauto = at<double>(L.Tauto);
         st.smax = at<double>(L.smax);
-        st.front = at<int32_t>(L.front);
+        st.front = at<unsigned long long>(L.front);
         st.T = at<float>(L.T);
         st.W_cap = W_cap;
         return st;
@@ -447,9 +448,13 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
 
     std::vector<uint8_t> tc_ok(M);
     for (int m = 0; m < M; ++m) {
+        if (!At[m]) {  // not evaluated in this call (subset entry points)
+            tc_ok[m] = 2;
+            continue;
+        }
         const bool aligned = (reinterpret_cast<uintptr_t>(At[m]) % 16 == 0) &&
                              (reinterpret_cast<uintptr_t>(Ar[m]) % 16 == 0) && (ctx->d[m] % 8 == 0);
-        tc_ok[m] = aligned && !(ctx->flags & EGERIA_FLAG_FORCE_SIMT);
+        tc_ok[m] = (aligned && !(ctx->flags & EGERIA_FLAG_FORCE_SIMT)) ? 1 : 0;
     }
     build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), e.plan,
                ctx->weights_version > 0 ? ctx->weights.data() : nullptr);
@@ -474,7 +479,7 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
     ModulePtrs *mods = reinterpret_cast<ModulePtrs *>(img + L.modules);
     for (int m = 0; m < M; ++m) {
         mods[m] = ModulePtrs{At[m], Ar[m], ctx->d[m]};
-        if (!tc_ok[m]) continue;
+        if (tc_ok[m] != 1) continue;
         egeria_status s = encode_map(ctx, &maps[2 * m], At[m], b, ctx->d[m], box_rows);
         if (s == EGERIA_OK) s = encode_map(ctx, &maps[2 * m + 1], Ar[m], b, ctx->d[m], box_rows);
         if (s != EGERIA_OK) return s;
@@ -548,13 +553,29 @@ static egeria_status set_attrs(egeria_ctx *ctx) {
 
 }  // namespace egeria
 
-static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void *const *At, const void *const *Ar,
-                                  int b, const int64_t *d, float *out_losses, bool fuse_step, double *out_slopes,
-                                  uint8_t *out_mask) {
-    if (!ctx || !At || !Ar || !d || !out_losses) return EGERIA_ERR_INVALID_ARG;
+static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void *const *At_in,
+                                  const void *const *Ar_in, int b, const int64_t *d, float *out_losses, bool fuse_step,
+                                  double *out_slopes, uint8_t *out_mask, const uint8_t *active = nullptr) {
+    if (!ctx || !At_in || !Ar_in || !d || !out_losses) return EGERIA_ERR_INVALID_ARG;
     if (b < 2 || b > ctx->b_max) return EGERIA_ERR_INVALID_ARG;
+    const void *const *At = At_in, *const *Ar = Ar_in;
+    if (active) {  // the plan is keyed by the pointers: a module left out has none
+        ctx->subset_t.assign(At_in, At_in + ctx->M);
+        ctx->subset_r.assign(Ar_in, Ar_in + ctx->M);
+        int n_active = 0;
+        for (int m = 0; m < ctx->M; ++m) {
+            if (active[m])
+                ++n_active;
+            else
+                ctx->subset_t[m] = ctx->subset_r[m] = nullptr;
+        }
+        if (n_active == 0) return EGERIA_ERR_INVALID_ARG;
+        At = ctx->subset_t.data();
+        Ar = ctx->subset_r.data();
+    }
     for (int m = 0; m < ctx->M; ++m) {
         if (d[m] != ctx->d[m]) return EGERIA_ERR_INVALID_ARG;
+        if (active && !active[m]) continue;
         if (!At[m] || !Ar[m]) return EGERIA_ERR_INVALID_ARG;
         if ((reinterpret_cast<uintptr_t>(At[m]) | reinterpret_cast<uintptr_t>(Ar[m])) & 1) return EGERIA_ERR_INVALID_ARG;
     }
@@ -595,9 +616,9 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
     fc.fuse_step = fuse_step ? 1 : 0;
     fc.W = ctx->W;
     fc.rule_flags = ctx->rule_flags();
-    fc.rule_parity = (int)(ctx->rule_evals & 1u);
-    fc.M = ctx->M;
     if (fuse_step) ctx->rule_evals++;
+    fc.rule_serial = ctx->rule_evals;
+    fc.M = ctx->M;
     fc.st = ctx->slope_state();
     fc.out_slopes = out_slopes;
     fc.out_mask = out_mask;
@@ -668,6 +689,19 @@ egeria_status egeria_plasticity_evaluate(egeria_ctx *ctx, void *cuda_stream, con
     return sp_loss_impl(ctx, cuda_stream, At, Ar, b, d, out_losses, true, out_slopes, out_mask);
 }
 
+egeria_status egeria_sp_loss_subset(egeria_ctx *ctx, void *cuda_stream, const void *const *At, const void *const *Ar,
+                                    int b, const int64_t *d, const uint8_t *active, float *out_losses) {
+    if (!active) return EGERIA_ERR_INVALID_ARG;
+    return sp_loss_impl(ctx, cuda_stream, At, Ar, b, d, out_losses, false, nullptr, nullptr, active);
+}
+
+egeria_status egeria_plasticity_evaluate_subset(egeria_ctx *ctx, void *cuda_stream, const void *const *At,
+                                                const void *const *Ar, int b, const int64_t *d, const uint8_t *active,
+                                                float *out_losses, double *out_slopes, uint8_t *out_mask) {
+    if (!active) return EGERIA_ERR_INVALID_ARG;
+    return sp_loss_impl(ctx, cuda_stream, At, Ar, b, d, out_losses, true, out_slopes, out_mask, active);
+}
+
 egeria_status egeria_sp_loss_batch_host(egeria_ctx *ctx, void *cuda_stream, const void *const *At_host,
                                         const void *const *Ar_host, int b, const int64_t *d, float *out_losses_host) {
     if (!ctx || !At_host || !Ar_host || !d || !out_losses_host) return EGERIA_ERR_INVALID_ARG;
@@ -695,9 +729,9 @@ egeria_status egeria_plasticity_step(egeria_ctx *ctx, void *cuda_stream, const f
     if (!ctx || !losses) return EGERIA_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     ctx->last_stream = stream;
-    plasticity_step_kernel<<<ctx->M, 32, 0, stream>>>(ctx->slope_state(), ctx->M, ctx->W, ctx->rule_flags(),
-                                                      (int)(ctx->rule_evals & 1u), losses, out_slopes, out_mask);
     ctx->rule_evals++;
+    plasticity_step_kernel<<<ctx->M, 32, 0, stream>>>(ctx->slope_state(), ctx->M, ctx->W, ctx->rule_flags(),
+                                                      ctx->rule_evals, losses, out_slopes, out_mask);
     if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
     ctx->launches++;
     return EGERIA_OK;
@@ -1009,7 +1043,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     fc.fuse_step = 0;
     fc.W = 0;
     fc.rule_flags = 0;
-    fc.rule_parity = 0;
+    fc.rule_serial = 0;
     fc.M = 1;
     fc.st = SlopeState{};
     fc.out_slopes = nullptr;

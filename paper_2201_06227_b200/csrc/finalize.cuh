@@ -34,7 +34,7 @@ struct FinCommon {
     int32_t fuse_step;
     int32_t W;
     int32_t rule_flags;     // RuleFlags
-    int32_t rule_parity;    // which front counter this evaluation reads (frontmost policy)
+    uint32_t rule_serial;   // number of this evaluation of the rule, from 1 (frontmost policy)
     int32_t M;
     SlopeState st;
     double *out_slopes;     // [M] or nullptr
@@ -235,7 +235,7 @@ __device__ __forceinline__ void finalize_module_total(const FinCommon &p, int m,
     const float loss = (float)(s / ((double)b * (double)b));
     if (lane == 0) p.out_losses[m] = loss;
     if (p.fuse_step)
-        plasticity_rule_step(p.st, L, m, p.M, p.W, p.rule_flags, p.rule_parity, loss, p.out_slopes, p.out_mask, lane);
+        plasticity_rule_step(p.st, L, m, p.M, p.W, p.rule_flags, p.rule_serial, loss, p.out_slopes, p.out_mask, lane);
 }
 
 struct FinParams {
@@ -247,7 +247,8 @@ struct FinParams {
 template <int NC>
 __global__ void __launch_bounds__(kFinThreads) finalize_kernel(const FinParams p) {
     const int m = blockIdx.x;
-    if (p.c.sides[2 * m].tensor_core) return;  // finished inside the tensor-core kernel
+    const SideInfo s0 = p.c.sides[2 * m];
+    if (s0.tensor_core || s0.module_units == 0) return;  // finished inside the tensor-core kernel / not evaluated
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = p.c.b;
     const int i = blockIdx.y * kFinRowsPerCta + warp;

@@ -531,7 +531,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 int best_left = 0, best_m = -1;
                 for (int mm = lane; mm < p.M; mm += 32) {
                     const SideInfo si = p.fin.sides[2 * mm];
-                    if (!si.tensor_core) continue;
+                    if (!si.tensor_core || si.module_units == 0) continue;
                     const int done = detail::ld_acquire(&p.ctr[mm].units_done);
                     const int cur = detail::ld_acquire(&p.ctr[mm].row_cursor);
                     const int left = (done >= si.module_units) ? b - cur : 0;

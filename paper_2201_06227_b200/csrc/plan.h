@@ -184,8 +184,9 @@ inline void split_tiles(const std::vector<Tile> &tiles, int n_ctas, int slot0, s
 }
 }  // namespace detail
 
-// tc_ok[m] != 0: module m may use the TMA + tcgen05 kernel.  weights: see split_tiles (applies to
-// the tensor-core split only).
+// tc_ok[m]: 1 = module m takes the TMA + tcgen05 kernel, 0 = the CUDA-core kernel, 2 = module m
+// is not evaluated in this plan (no units, never finished).  weights: see split_tiles (applies
+// to the tensor-core split only).
 inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t *tc_ok, Plan &plan,
                        const float *weights = nullptr) {
     plan.mode = mode_of_b(b);
@@ -194,6 +195,7 @@ inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t
     plan.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, {0, 0}});
     std::vector<detail::Tile> tc, simt;
     for (int m = 0; m < M; ++m) {
+        if (tc_ok[m] == 2) continue;
         std::vector<detail::Tile> &dst = tc_ok[m] ? tc : simt;
         if (mode_is_stacked(plan.mode)) {
             dst.push_back({m, 2, kblocks_of(d[m])});
@@ -222,7 +224,7 @@ inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t
     for (int m = 0; m < M; ++m) {
         SideInfo &t = plan.sides[2 * (size_t)m], &r = plan.sides[2 * (size_t)m + 1];
         const int32_t units = mode_is_stacked(plan.mode) ? t.n_slots : t.n_slots + r.n_slots;
-        t.tensor_core = r.tensor_core = tc_ok[m] ? 1 : 0;
+        t.tensor_core = r.tensor_core = (tc_ok[m] == 1) ? 1 : 0;
         t.module_units = r.module_units = units;
     }
 }

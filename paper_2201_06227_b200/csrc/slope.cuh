@@ -26,7 +26,8 @@ struct SlopeState {     // per-module arrays (device)
     double *last_slope; // [M]
     double *Tauto;      // [M] automatic tolerance (NaN until the third reading)
     double *smax;       // [M] largest |slope| of the initial readings
-    int32_t *front;     // [2] number of frozen modules (frontmost policy): read [parity], write [parity ^ 1]
+    unsigned long long *front;  // [1] frontmost policy: (serial of the evaluation that last moved the front) << 32
+                                //     | number of frozen modules; one 8-byte word, read and written whole
     const float *T;     // [M] tolerance given at creation
     int32_t W_cap;      // window pitch
 };
@@ -234,11 +235,11 @@ __device__ __forceinline__ bool plasticity_step_apply(const SlopeState &st, Step
 // for itself.  With it, only the frontmost module that is not frozen advances; its warp (the
 // last module's when all are frozen) also reports for everybody: mask[j] = j is frozen,
 // slopes[j] = the slope of this evaluation for the monitored module, the final slope of a
-// frozen one, +inf for one that has not been monitored yet.  `parity` selects which of the
-// two front counters this evaluation reads; it writes the other, so that a module that
-// becomes the front during an evaluation starts with the next one.
+// frozen one, +inf for one that has not been monitored yet.  `serial` numbers the evaluations
+// (from 1): a front that moved during evaluation `serial` is left alone for the rest of it,
+// so the module that becomes the front starts with the next evaluation.
 __device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepLoaded &L, int m, int M, int W,
-                                                     int flags, int parity, float reading, double *out_slopes,
+                                                     int flags, uint32_t serial, float reading, double *out_slopes,
                                                      uint8_t *out_mask, int lane) {
     if (!(flags & kRuleFrontmost)) {
         double slope;
@@ -249,7 +250,9 @@ __device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepL
         }
         return;
     }
-    const int front = st.front[parity];
+    const unsigned long long word = *reinterpret_cast<volatile unsigned long long *>(st.front);
+    if ((uint32_t)(word >> 32) == serial) return;  // the front moved in this evaluation: it has been dealt with
+    const int front = (int)(uint32_t)word;
     const int reporter = front < M ? front : M - 1;
     if (m != reporter) return;
     int front_new = front;
@@ -258,7 +261,9 @@ __device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepL
         const bool conv = plasticity_step_apply(st, L, m, W, flags, reading, lane, slope);
         if (conv) front_new = front + 1;
     }
-    if (lane == 0) st.front[parity ^ 1] = front_new;
+    if (lane == 0 && front_new != front)
+        *reinterpret_cast<volatile unsigned long long *>(st.front) =
+            ((unsigned long long)serial << 32) | (unsigned long long)(uint32_t)front_new;
     for (int j = lane; j < M; j += 32) {
         if (out_mask) out_mask[j] = (j < front_new) ? 1 : 0;
         if (out_slopes) out_slopes[j] = (j == m && front < M) ? slope : (j < front ? st.last_slope[j] : INFINITY);
@@ -266,13 +271,13 @@ __device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepL
 }
 
 // One new reading per module.  grid = M warps (one 32-thread block each).
-__global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int M, int W, int flags, int parity,
+__global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int M, int W, int flags, uint32_t serial,
                                                              const float *losses, double *out_slopes,
                                                              uint8_t *out_mask) {
     const int m = blockIdx.x, lane = threadIdx.x;
     if (m >= M) return;
     StepLoaded L = plasticity_step_load(st, m, W, lane);
-    plasticity_rule_step(st, L, m, M, W, flags, parity, losses[m], out_slopes, out_mask, lane);
+    plasticity_rule_step(st, L, m, M, W, flags, serial, losses[m], out_slopes, out_mask, lane);
 }
 
 // Whole histories from a cleared private state (windows in shared memory: 2 * W doubles).
@@ -331,7 +336,7 @@ __global__ void __launch_bounds__(32) plasticity_replay_kernel(const float *T, i
 
 __global__ void plasticity_clear_kernel(SlopeState st, int M) {
     const int m = blockIdx.x * blockDim.x + threadIdx.x;
-    if (m < 2) st.front[m] = 0;
+    if (m == 0) *st.front = 0ull;
     if (m >= M) return;
     st.n_evals[m] = 0;
     st.counter[m] = 0;

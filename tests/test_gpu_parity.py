@@ -566,6 +566,70 @@ def test_frontmost_policy_inside_the_fused_evaluation():
     split.close()
 
 
+def test_subset_evaluation_touches_only_the_active_modules():
+    ds, b = [4096, 1001, 30000, 520, 8192, 64], 72
+    at, ar = [], []
+    for m, d in enumerate(ds):
+        t, r = wl.make_pair(b, d, "relu", 0.05 + 0.05 * m, seed=600 + m, device=DEV)
+        at.append(t)
+        ar.append(r)
+    ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+    ctx = eg.Context(ds, b, 3, 1e-3, device=DEV)
+    for active in ([1, 0, 0, 0, 0, 0], [0, 1, 0, 0, 0, 0], [0, 0, 1, 0, 1, 0], [1, 1, 1, 1, 1, 1], [0, 0, 0, 1, 0, 1]):
+        out = torch.full((len(ds),), -7.0, dtype=torch.float32, device=DEV)
+        left_out = [None if not a else t for t, a in zip(at, active)]       # pointers of the others are not read
+        ctx.egeria_sp_loss_subset(left_out, [None if not a else r for r, a in zip(ar, active)], active, out)
+        got = out.cpu().numpy()
+        act = np.array(active, dtype=bool)
+        assert_loss_close(got[act], ref[act], f"subset {active}")
+        assert np.all(got[~act] == -7.0)
+    ctx.check_device_status()
+    with pytest.raises(eg.EgeriaError) as e:
+        ctx.egeria_sp_loss_subset(at, ar, [0] * len(ds), out)
+    assert e.value.status == eg.ERR_INVALID_ARG
+    # the rule advances for the active modules only
+    losses = torch.zeros(len(ds), dtype=torch.float32, device=DEV)
+    slopes = torch.full((len(ds),), -1.0, dtype=torch.float64, device=DEV)
+    mask = torch.full((len(ds),), 9, dtype=torch.uint8, device=DEV)
+    for _ in range(2):
+        ctx.egeria_plasticity_evaluate_subset(at, ar, [0, 0, 1, 0, 0, 0], losses, slopes, mask)
+    s, mk = slopes.cpu().numpy(), mask.cpu().numpy()
+    assert s[2] == 0.0 and mk[2] == 0                       # two equal readings: slope 0, not frozen yet (W = 3)
+    assert np.all(s[[0, 1, 3, 4, 5]] == -1.0) and np.all(mk[[0, 1, 3, 4, 5]] == 9)
+    ctx.close()
+
+
+def test_frontmost_policy_evaluating_only_the_front_module():
+    """The intended use of the frontmost policy: read the mask back, evaluate only the first module
+    that is not frozen.  Same decisions as evaluating everything."""
+    ds, b, W = [4096, 2048, 1001, 8192, 520], 40, 2
+    flags = eg.FLAG_FRONTMOST
+    full = eg.Context(ds, b, W, 0.5, flags, device=DEV)
+    front_only = eg.Context(ds, b, W, 0.5, flags, device=DEV)
+    M = len(ds)
+    losses = torch.zeros(M, dtype=torch.float32, device=DEV)
+    slopes = torch.zeros(M, dtype=torch.float64, device=DEV)
+    mask = torch.zeros(M, dtype=torch.uint8, device=DEV)
+    front, seen = 0, []
+    for k in range(16):
+        at, ar = [], []
+        for m, d in enumerate(ds):
+            t, r = wl.make_pair(b, d, "relu", 0.3, seed=800 + 10 * k + m, device=DEV)
+            at.append(t)
+            ar.append(r)
+        l1, s1, m1 = full.egeria_plasticity_evaluate(at, ar)
+        if front < M:
+            active = [1 if m == front else 0 for m in range(M)]
+            front_only.egeria_plasticity_evaluate_subset(at, ar, active, losses, slopes, mask)
+            assert_loss_close(losses.cpu().numpy()[front:front + 1], l1.cpu().numpy().astype(np.float64)[front:front + 1])
+        assert mask.cpu().numpy().tolist() == m1.cpu().numpy().tolist()
+        front = int(mask.cpu().numpy().sum())
+        seen.append(front)
+    assert seen[-1] == M and seen[0] == 0
+    full.close()
+    front_only.close()
+
+
 def test_bootstrap_detector_matches_oracle():
     rng = np.random.default_rng(11)
     H, W = 120, 8
