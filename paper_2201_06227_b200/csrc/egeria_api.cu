@@ -162,6 +162,7 @@ struct egeria_ctx {
     // Split weights: one per CTA, from the streaming rates the CTAs report (SMs do not all get
     // the same share of HBM bandwidth; the CTA -> SM placement repeats from launch to launch).
     std::vector<float> weights;
+    std::vector<double> rate_sum;  // blocks per nanosecond of every CTA, summed over the later rounds
     int weights_version = 0;
     bool calibrated = false;   // no more measuring
     int calib_round = 0;
@@ -408,6 +409,12 @@ static void poll_calibration(egeria_ctx *ctx) {
             }
             rate[c] += (double)blocks / (double)ns;
         }
+    }
+    // From the second round on the rates were measured under shares close to the final ones: keep
+    // adding them up, so that the last word is an average over six launches, not three.
+    if (ctx->calib_round >= 1) {
+        if (ctx->rate_sum.size() != (size_t)n) ctx->rate_sum.assign(n, 0.0);
+        for (int c = 0; c < n; ++c) rate[c] = (ctx->rate_sum[c] += rate[c]);
     }
     double mean = 0.0;
     for (int c = 0; c < n; ++c) mean += rate[c];
