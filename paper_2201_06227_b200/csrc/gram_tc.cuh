@@ -55,8 +55,7 @@ struct TcCfg {
     static constexpr int kKbPerStage = (MODE == kStacked32) ? 6 : 1;
     static constexpr int kStageBytes = kSlabBytes * kKbPerStage;           // 48 KB, 16 KB, 16 KB, 32 KB
     static constexpr int kStages = (MODE == kStacked32) ? 4 : (MODE == kSingle2 ? 6 : 12);  // 192 KB of loads in flight
-    // kStacked32 issues M = 128 MMAs over a 64-row slab: the A operand reaches one slab further.
-    static constexpr int kPadBytes = (MODE == kStacked32) ? kSlabBytes : 0;
+    static constexpr int kPadBytes = 0;
     static constexpr int kAccCols = (MODE == kStacked32) ? 64 : (MODE == kSingle2 ? 384 : 128);
     static constexpr int kAccStages = (MODE == kSingle2) ? 1 : 2;
     static constexpr int kTmemCols = (MODE == kStacked32) ? 128 : (MODE == kSingle2 ? 512 : 256);
@@ -113,7 +112,9 @@ struct Chunk {
 
 // Chunk k of the accumulator of one unit, for the warp of TMEM lane quarter q.  False if there
 // is no such chunk (warp-uniform).  Layouts per mode:
-//   kStacked32: rows 0..31 x cols 0..31 = G_T, rows 32..63 x cols 32..63 = G_R
+//   kStacked32: one M = 64 accumulator: rows 0..31 x cols 0..31 = G_T, rows 32..63 x cols 32..63 = G_R
+//               (an M = 64 accumulator keeps row r in TMEM lane (r % 16) + 32 * (r / 16): the lower
+//               16 lanes of every lane quarter)
 //   kStacked64: rows 0..63 x cols 0..63 = G_T, rows 64..127 x cols 64..127 = G_R
 //   kSingle1:   rows 0..127 x cols 0..127 = G
 //   kSingle2:   cols 0..255 = rows 0..127 of G (all 256 columns); cols 256..383 = G11
@@ -121,10 +122,12 @@ template <int MODE>
 __device__ __forceinline__ bool chunk_of(int k, int q, int lane, int b, float *slot, Chunk &ch) {
     ch.mirror_c0 = -1;
     if (MODE == kStacked32) {
-        if (k != 0 || q >= 2) return false;
-        ch.col = q * 32;
-        ch.dst = slot + q * 32 * 32 + lane * 32;
-        ch.valid = lane < b;
+        // quarter q holds accumulator rows 16 q .. 16 q + 15: quarters 0, 1 = G_T, 2, 3 = G_R
+        const int side = q >> 1, r = 16 * (q & 1) + lane;
+        if (k != 0 || 16 * (q & 1) >= b) return false;
+        ch.col = side * 32;
+        ch.dst = slot + side * 32 * 32 + r * 32;
+        ch.valid = lane < 16 && r < b;
         return true;
     } else if (MODE == kStacked64) {
         const int side = q >> 1, r = (q & 1) * 32 + lane, c0 = 32 * k;
@@ -356,7 +359,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc64 = ptx::make_idesc_bf16_f32(128, 64);
+            constexpr uint32_t idesc64x64 = ptx::make_idesc_bf16_f32(64, 64);
             constexpr uint32_t idesc128 = ptx::make_idesc_bf16_f32(128, 128);
             constexpr uint32_t idesc256 = ptx::make_idesc_bf16_f32(128, 256);
             const uint64_t t_entry = ptx::globaltimer_ns();
@@ -394,9 +397,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                                 // G11 = rows 128..255 against themselves
                                 ptx::mma_bf16_ss(d_tmem + 256, hi, hi, idesc128, accum);
                             } else if (MODE == kStacked32) {
-                                // 128 operand rows, of which only 0..63 (this slab) matter
-                                ptx::mma_bf16_ss(d_tmem, lo, lo, idesc64, accum);
+                                // the whole 64-row slab against itself
+                                ptx::mma_bf16_ss(d_tmem, lo, lo, idesc64x64, accum);
                             } else {
+                                // kStacked64 too: two M = 64 MMAs without the cross terms draw less power but
+                                // take longer (the issue rate of small MMAs, not their size, sets the pace)
                                 ptx::mma_bf16_ss(d_tmem, lo, lo, idesc128, accum);
                             }
                         }
