@@ -232,29 +232,47 @@ def test_bert_base_workload_full():
 
 
 def _sampled_check(name, full_modules, row_modules, rows):
-    """Full-size workload in the benchmark's launch configuration; the oracle checks the
-    whole loss of a few modules and sampled rows of the normalised Grams of others."""
+    """Full-size workload in the benchmark's launch configuration -- the call bench.py times
+    (egeria_plasticity_evaluate), first with the equal split and again once the adaptive split
+    has settled; the oracle checks the whole loss of a few modules and sampled rows of the
+    normalised Grams of others."""
     w = wl.WORKLOADS[name]
     at, ar = wl.make_activations(w, DEV)
-    losses, grams = run_gpu(at, ar, keep=True, W=w.W, T=w.T)
-    assert np.isfinite(losses).all() and np.all(losses >= 0) and np.all(losses <= 4.0 / w.b)
-    for m in full_modules:
-        ref, gt, gr = oracle.sp_loss(wl.bf16_bits(at[m]), wl.bf16_bits(ar[m]), return_grams=True)
-        np.testing.assert_allclose(grams[m][0], gt, rtol=0, atol=ENTRY_ATOL)
-        np.testing.assert_allclose(grams[m][1], gr, rtol=0, atol=ENTRY_ATOL)
-        assert_loss_close(losses[m:m + 1], [ref], f"{name} module {m}")
+    full_ref = {m: oracle.sp_loss(wl.bf16_bits(at[m]), wl.bf16_bits(ar[m]), return_grams=True) for m in full_modules}
+    row_ref = {}
     for m in row_modules:
         for side, acts in enumerate((at, ar)):
             bits = wl.bf16_bits(acts[m])
             for i in rows:
                 g = oracle.gram_row(bits, i)
-                gn = g / max(np.linalg.norm(g), oracle.EPS)
-                np.testing.assert_allclose(grams[m][side][i], gn, rtol=0, atol=ENTRY_ATOL)
-    # properties that hold at any size: unit rows, symmetric-positive diagonal
-    for m in range(w.M):
-        for side in (0, 1):
-            np.testing.assert_allclose(np.linalg.norm(grams[m][side].astype(np.float64), axis=1), 1.0, atol=1e-5)
-            assert np.all(np.diag(grams[m][side]) > 0)
+                row_ref[(m, side, i)] = g / max(np.linalg.norm(g), oracle.EPS)
+    ctx = eg.Context(list(w.d), w.b, w.W, float(np.float32(w.T)), eg.FLAG_KEEP_GRAMS, device=DEV)
+
+    def check(what):
+        losses = ctx.egeria_plasticity_evaluate(at, ar)[0].cpu().numpy()
+        grams = [tuple(g.cpu().numpy() for g in ctx.egeria_debug_dump_gram(m, w.b)) for m in range(w.M)]
+        ctx.check_device_status()
+        assert np.isfinite(losses).all() and np.all(losses >= 0) and np.all(losses <= 4.0 / w.b)
+        for m, (ref, gt, gr) in full_ref.items():
+            np.testing.assert_allclose(grams[m][0], gt, rtol=0, atol=ENTRY_ATOL)
+            np.testing.assert_allclose(grams[m][1], gr, rtol=0, atol=ENTRY_ATOL)
+            assert_loss_close(losses[m:m + 1], [ref], f"{name} module {m} ({what})")
+        for (m, side, i), gn in row_ref.items():
+            np.testing.assert_allclose(grams[m][side][i], gn, rtol=0, atol=ENTRY_ATOL)
+        # properties that hold at any size: unit rows, symmetric-positive diagonal
+        for m in range(w.M):
+            for side in (0, 1):
+                np.testing.assert_allclose(np.linalg.norm(grams[m][side].astype(np.float64), axis=1), 1.0, atol=1e-5)
+                assert np.all(np.diag(grams[m][side]) > 0)
+        return losses
+
+    first = check("equal split")
+    for _ in range(12):
+        ctx.egeria_plasticity_evaluate(at, ar)[0].cpu()       # .cpu() waits: the launch logs land
+    assert ctx.egeria_split_weights()[0] > 0                  # the shares now follow the measured rates
+    settled = check("adaptive split")
+    assert_loss_close(settled, first.astype(np.float64), f"{name} adaptive vs equal split")
+    ctx.close()
 
 
 def test_resnet50_workload_sampled():
