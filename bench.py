@@ -36,7 +36,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the evaluation kernel, from the ncu
 # captures summarised under profiles/ (gpt2_medium: a 6-module launch scaled x4 by the modules
 # processed).  Valid for the kernel as captured; set to None when the kernel changes.
-NCU_TRAFFIC_BYTES = {"gpt2_medium": 6478744000, "resnet50": 1418083000}   # kernels <3> and <1>: unchanged since
+NCU_TRAFFIC_BYTES = {"gpt2_medium": 6476067000, "resnet50": 1419185000}
 
 
 # ----------------------------------------------------------------------------- helpers
