@@ -55,13 +55,12 @@ struct TcCfg {
     static constexpr int kKbPerStage = (MODE == kStacked32) ? 6 : 1;
     static constexpr int kStageBytes = kSlabBytes * kKbPerStage;           // 48 KB, 16 KB, 16 KB, 32 KB
     static constexpr int kStages = (MODE == kStacked32) ? 4 : (MODE == kSingle2 ? 6 : 12);  // 192 KB of loads in flight
-    static constexpr int kPadBytes = 0;
     static constexpr int kAccCols = (MODE == kStacked32) ? 64 : (MODE == kSingle2 ? 384 : 128);
     static constexpr int kAccStages = (MODE == kSingle2) ? 1 : 2;
     static constexpr int kTmemCols = (MODE == kStacked32) ? 128 : (MODE == kSingle2 ? 512 : 256);
     static constexpr int kNC = (MODE == kStacked32) ? 1 : (MODE == kStacked64 ? 2 : (MODE == kSingle1 ? 4 : 8));
     static constexpr int kSmemBytes =
-        kStages * kStageBytes + kPadBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
+        kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
 };
 
 struct TcParams {
@@ -250,7 +249,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     // 1024-byte alignment: the 128-byte swizzle pattern is a function of address bits 4..9.
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_aligned = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_aligned + Cfg::kStages * Cfg::kStageBytes + Cfg::kPadBytes);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_aligned + Cfg::kStages * Cfg::kStageBytes);
     // bars: full[kStages], empty[kStages], acc_full[kAccStages], acc_empty[kAccStages]
     const uint32_t full0 = ptx::smem_u32(bars);
     const uint32_t empty0 = full0 + 8 * Cfg::kStages;

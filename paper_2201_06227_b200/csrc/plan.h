@@ -17,8 +17,7 @@ constexpr int kKBlock = 64;
 
 // How the b rows of A_T / A_R are laid into MMA tiles.
 //   kStacked32 : b <= 32.  One tile per module: A_T in rows 0..31 and A_R in rows 32..63 of a
-//                64-row slab, one 128x64 MMA (the upper 64 accumulator rows are unused); the
-//                two diagonal 32x32 blocks are G_T and G_R.
+//                64-row slab, one 64x64 MMA; the two diagonal 32x32 blocks are G_T and G_R.
 //   kStacked64 : b <= 64.  Same with 64 rows per side: 128-row slab, one 128x128 MMA.
 //   kSingle1   : b <= 128. One tile per (module, side): 128-row slab, one 128x128 MMA.
 //   kSingle2   : b <= 256. One tile per (module, side): 256-row slab, the upper triangle of
