@@ -28,6 +28,32 @@ def test_library_exports_every_declared_symbol():
     assert sorted(eg.EXPORTS) == names
 
 
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 on its own, and a C program that
+    only uses the host-side calls must link against the library."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    src = tmp_path / "use_header.c"
+    src.write_text(
+        '#include "egeria.h"\n'
+        '#include <stdio.h>\n'
+        'int main(void) {\n'
+        '    int64_t d[2] = {4096, 8192};\n'
+        '    size_t n = egeria_workspace_bytes(2, d, 64, 10, EGERIA_FLAG_KEEP_GRAMS | EGERIA_FLAG_FRONTMOST);\n'
+        '    printf("%zu %s\\n", n, egeria_status_string(EGERIA_ERR_TIMEOUT));\n'
+        '    return n > 0 ? 0 : 1;\n'
+        '}\n')
+    exe = tmp_path / "use_header"
+    lib_dir = Path(eg._LIB_PATH).parent
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", str(HEADER.parent), str(src), "-o", str(exe),
+                    "-L", str(lib_dir), "-legeria", f"-Wl,-rpath,{lib_dir}"], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split(" ", 1)
+    assert int(out[0]) == eg.egeria_workspace_bytes(2, [4096, 8192], 64, 10, eg.FLAG_KEEP_GRAMS | eg.FLAG_FRONTMOST)
+    assert out[1].strip() == eg.status_string(eg.ERR_TIMEOUT)
+
+
 def test_status_strings():
     for s in range(7):
         assert eg.status_string(s) not in ("", "unknown status")
