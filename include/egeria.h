@@ -24,11 +24,11 @@
  *     no CPU fallback: without an sm_100 device the compute calls fail with
  *     EGERIA_ERR_UNSUPPORTED_DEVICE or EGERIA_ERR_CUDA.
  *   - One context per stream; a context is not thread-safe.
- *   - A call passes the kernel state that belongs to that call (which of two sets of
+ *   - A call on a context passes the kernel state that belongs to that call (which of two sets of
  *     progress counters to use, the serial number of the rule evaluation), and may
  *     enqueue small copies (a new work plan, the launch log of the adaptive split):
- *     enqueue every evaluation through the library; replaying one from a captured
- *     CUDA graph would reuse that state and give wrong results.
+ *     enqueue every evaluation of a context through the library; replaying one from a
+ *     captured CUDA graph would reuse that state and give wrong results.
  */
 #ifndef EGERIA_H_
 #define EGERIA_H_
