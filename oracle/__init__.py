@@ -7,7 +7,8 @@ the smoke check and the benchmark's CPU-baseline leg -- never by the product.
 
 Paper passages followed: Sec. 4.2.1 / Eq. 1 (SP loss = plasticity), Sec. 4.2.2 /
 Eq. 2 (moving average), Sec. 4.2.2 + Algorithm 1 (window linear fit, stale
-counter, freezing decision).
+counter, freezing decision, frontmost-active module, learning-rate-based
+unfreezing), Sec. 3 (end of the bootstrapping stage).
 """
 from __future__ import annotations
 
@@ -76,6 +77,11 @@ def lib() -> ctypes.CDLL:
         L.egeria_oracle_frontmost_replay.restype = ctypes.c_int
         L.egeria_oracle_bootstrap_replay.argtypes = [ctypes.POINTER(ctypes.c_float), i64, i64, ctypes.c_double, f64p]
         L.egeria_oracle_bootstrap_replay.restype = ctypes.c_int64
+        u8p = ctypes.POINTER(ctypes.c_uint8)
+        L.egeria_oracle_unfreeze_replay.argtypes = [
+            ctypes.POINTER(ctypes.c_float), f64p, i64, i64, i64, f64p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            f64p, u8p, i32p, i32p]
+        L.egeria_oracle_unfreeze_replay.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -231,3 +237,28 @@ def bootstrap_replay(loss_hist, W: int, rate_tol: float = 0.1):
     if end < -1:
         raise RuntimeError("oracle bootstrap_replay: bad sizes")
     return dict(end=int(end), rates=rates[:H])
+
+
+def unfreeze_replay(hist, lr, W: int, T=None, frontmost: bool = False, signed_test: bool = False):
+    """Algorithm 1 with its learning-rate-based unfreezing (Sec. 4.2.2 "Unfreezing") over [M, H]
+    raw readings and the learning rate lr[H] at each evaluation: once the learning rate is a
+    tenth (or less) of what it was at the first freeze, all modules restart and W is halved
+    (never below 2).  T: per-module tolerances, or None for the automatic one.
+    Returns dict(slopes[M, H], frozen[H, M], window[H], restarted[H], restarts)."""
+    h = np.ascontiguousarray(hist, dtype=np.float32)
+    M, H = h.shape
+    lr = np.ascontiguousarray(np.broadcast_to(lr, (H,)), dtype=np.float64)
+    auto = T is None
+    Tarr = np.zeros(M, dtype=np.float64) if auto else np.ascontiguousarray(np.broadcast_to(T, (M,)), dtype=np.float64)
+    fz = np.zeros((max(H, 1), M), dtype=np.uint8)
+    win = np.empty(max(H, 1), dtype=np.int32)
+    rs = np.zeros(max(H, 1), dtype=np.int32)
+    sl_c = np.empty(M * max(H, 1), dtype=np.float64)
+    rc = lib().egeria_oracle_unfreeze_replay(_p(h, ctypes.c_float), _p(lr, ctypes.c_double), M, H, int(W),
+                                             _p(Tarr, ctypes.c_double), int(bool(signed_test)), int(auto),
+                                             int(bool(frontmost)), _p(sl_c, ctypes.c_double),
+                                             _p(fz, ctypes.c_uint8), _p(win, ctypes.c_int32), _p(rs, ctypes.c_int32))
+    if rc < 0:
+        raise RuntimeError(f"oracle unfreeze_replay failed ({rc})")
+    sl = sl_c[:M * H].reshape(M, H)
+    return dict(slopes=sl, frozen=fz[:H], window=win[:H], restarted=rs[:H], restarts=int(rc))

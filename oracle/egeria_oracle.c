@@ -19,7 +19,11 @@
  *   - the least-squares straight-line fit of the last min(len, W) smoothed
  *     values against the evaluation index, and its slope [Sec. 4.2.2,
  *     Algorithm 1 "windowLinearFit"];
- *   - the stale counter and the convergence decision [Algorithm 1].
+ *   - the stale counter and the convergence decision [Algorithm 1];
+ *   - the policies stated around Algorithm 1: per-module automatic tolerance,
+ *     frontmost-active module, end of the bootstrapping stage [Sec. 3,
+ *     Sec. 4.2.2], and unfreezing on learning-rate annealing with the halved
+ *     window [Sec. 4.2.2 "Unfreezing"; Algorithm 1, second half].
  *
  * Everything is written out as the definition: no symmetry shortcut, no
  * tiling, no split sums.  Sums run in ascending index order in float64.
@@ -28,8 +32,9 @@
  *
  * Pins (see tests): closed forms for b = 2 and for one-hot / identical-row
  * inputs, exact rational arithmetic on tiny inputs, a BLAS route, invariants
- * and a negative control, closed-form and pair-wise brute-force slopes, and
- * hand-replayed Algorithm 1 traces.  Nothing numerical is printed in the paper
+ * and a negative control, closed-form and pair-wise brute-force slopes,
+ * hand-replayed Algorithm 1 traces, and for the policies hand-worked traces
+ * plus their reduction to chained runs of the plain rule.  Nothing numerical is printed in the paper
  * for this path, so no value here is pinned to a number of the paper's own.
  */
 #include <math.h>
@@ -299,9 +304,9 @@ int egeria_oracle_plasticity_replay_auto(const float *hist, int64_t H, int64_t W
     return conv;
 }
 
-/* The frontmost-active policy [Sec. 4.2.2: "monitors the frontmost active layer module l to
- * avoid a fragmented frozen model"; Algorithm 1: freeze, then l <- l + 1].  Modules are ordered
- * front to back.  Only module l = (number of frozen modules) is monitored: evaluation i feeds
+/* The frontmost-active policy [Sec. 4.2.2: only the frontmost module that is still active is
+ * monitored, so that the frozen modules always form a prefix; Algorithm 1: freeze, then
+ * l <- l + 1].  Modules are ordered front to back.  Only module l = (number of frozen modules) is monitored: evaluation i feeds
  * it hist[l][i]; when its counter reaches W it is frozen at that evaluation and the next
  * evaluation starts module l + 1 from a cleared state.  hist is [M][H] row-major.
  * Outputs: freeze_eval[M] (-1 = not frozen within the history), monitored[H] (module fed at
@@ -337,7 +342,7 @@ int egeria_oracle_frontmost_replay(const float *hist, int64_t M, int64_t H, int6
 }
 
 /* End of the bootstrapping stage [Sec. 3 "Bootstrapping stage": the changing rate of the
- * training loss is monitored "in line with the later plasticity monitoring"; Sec. 4.2.2: the
+ * training loss is watched with the same machinery as the plasticity later on; Sec. 4.2.2: the
  * changing rate that ends the stage is 10%].  The training-loss readings are smoothed [Eq. 2]
  * and fitted like the plasticity; with a full window of W smoothed values, slope s and window
  * mean ybar, the changing rate is |s| (W - 1) / |ybar|: the relative change of the fitted line
@@ -367,4 +372,98 @@ int64_t egeria_oracle_bootstrap_replay(const float *loss, int64_t H, int64_t W, 
     }
     free(P); free(pl);
     return end;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Unfreezing on learning-rate annealing [Sec. 4.2.2 "Unfreezing"; Algorithm 1, the branch that
+ * follows the freeze step: unfreezeAllLayers, l <- l_0].
+ *
+ * The rule as the paper states it: once the learning rate has fallen by a factor of ten or
+ * more since the frontmost layers were frozen, every frozen module is trained again, the
+ * monitored module goes back to the first one, and the counter / history-buffer length W is
+ * halved for the refreezing.
+ *
+ * Readings taken where the text leaves room:
+ *   - "since the frontmost layers' freeze": the learning rate in force at the first freeze
+ *     after the start or after the last restart is remembered (lr_ref);
+ *   - the test runs at the end of every evaluation, after the freeze step, as in Algorithm 1:
+ *     restart iff lr_i <= lr_ref / 10 * (1 + 1e-6).  The slack of one part in a million lets a
+ *     step decay by exactly 10x count ("decreased by 90%") even when the schedule was computed
+ *     in single precision.  A learning rate that is not positive carries no information: it
+ *     neither sets lr_ref nor triggers a restart;
+ *   - a restart clears every module's raw history, pList and staleCounter (with the automatic
+ *     tolerance also the derived T: the initial readings are those after the restart), forgets
+ *     lr_ref (nothing is frozen any more) and sets W <- max(2, floor(W / 2)) (a line needs two
+ *     points; W = 1 stays 1).  The reading of the evaluation that triggered the restart has
+ *     been consumed by the old state; the next evaluation is the first of the new one.
+ *
+ * hist is [M][H] row-major raw readings, lr is [H] (the learning rate at each evaluation),
+ * T is [M] (ignored with auto_T).  frontmost != 0 monitors only the frontmost module that is
+ * not frozen (as egeria_oracle_frontmost_replay), else every module runs Algorithm 1 on its own.
+ * Outputs (any may be NULL):
+ *   slopes[M][H]   slope of module m at evaluation i, NaN where the module was not advanced
+ *   frozen[H][M]   1 where module m is frozen after evaluation i (after the unfreezing test)
+ *   window[H]      W in force during evaluation i
+ *   restarted[H]   1 if the unfreezing fired at the end of evaluation i
+ * Returns the number of restarts, negative on error. */
+static int64_t halve_window(int64_t W) {
+    if (W < 2) return W;
+    int64_t h = W / 2;
+    return h < 2 ? 2 : h;
+}
+
+int egeria_oracle_unfreeze_replay(const float *hist, const double *lr, int64_t M, int64_t H, int64_t W0,
+                                  const double *T, int signed_test, int auto_T, int frontmost,
+                                  double *slopes, uint8_t *frozen, int32_t *window, int32_t *restarted) {
+    if (M < 1 || H < 0 || W0 < 1 || !hist || !lr) return -2;
+    module_state *st = (module_state *)calloc((size_t)M, sizeof(module_state));
+    uint8_t *is_frozen = (uint8_t *)calloc((size_t)M, 1);
+    if (!st || !is_frozen) { free(st); free(is_frozen); return -1; }
+    int rc = 0;
+    for (int64_t m = 0; m < M; ++m) {
+        st[m].P = (double *)malloc(sizeof(double) * (size_t)(H > 0 ? H : 1));
+        st[m].pl = (double *)malloc(sizeof(double) * (size_t)(H > 0 ? H : 1));
+        if (!st[m].P || !st[m].pl) rc = -1;
+    }
+    if (rc == 0) {
+        int64_t W = W0, l = 0;
+        double lr_ref = NAN;
+        for (int64_t m = 0; m < M; ++m) {
+            st[m].len = 0; st[m].counter = 0; st[m].smax = 0.0;
+            st[m].T = auto_T ? NAN : T[m];
+        }
+        for (int64_t i = 0; i < H; ++i) {
+            if (window) window[i] = (int32_t)W;
+            if (slopes) for (int64_t m = 0; m < M; ++m) slopes[m * H + i] = NAN;
+            int froze_now = 0;
+            /* checkPlasticity for the monitored module(s) */
+            for (int64_t m = 0; m < M; ++m) {
+                if (is_frozen[m]) continue;
+                if (frontmost && m != l) continue;
+                double s = module_advance(&st[m], (double)hist[m * H + i], W, signed_test, auto_T);
+                if (slopes) slopes[m * H + i] = s;
+                if (st[m].counter >= W) { is_frozen[m] = 1; froze_now = 1; }
+            }
+            if (frontmost && l < M && is_frozen[l]) ++l;   /* freezeLayer(l); l <- l + 1 */
+            if (froze_now && isnan(lr_ref) && lr[i] > 0.0) lr_ref = lr[i];
+            /* learning-rate-based unfreezing */
+            int fire = (!isnan(lr_ref) && lr[i] > 0.0 && lr[i] <= lr_ref / 10.0 * (1.0 + 1e-6));
+            if (fire) {
+                for (int64_t m = 0; m < M; ++m) {          /* unfreezeAllLayers() */
+                    is_frozen[m] = 0;
+                    st[m].len = 0; st[m].counter = 0; st[m].smax = 0.0;
+                    st[m].T = auto_T ? NAN : T[m];
+                }
+                l = 0;                                      /* l <- l_0 */
+                W = halve_window(W);
+                lr_ref = NAN;
+                ++rc;
+            }
+            if (restarted) restarted[i] = fire;
+            if (frozen) for (int64_t m = 0; m < M; ++m) frozen[i * M + m] = is_frozen[m];
+        }
+    }
+    for (int64_t m = 0; m < M; ++m) { free(st[m].P); free(st[m].pl); }
+    free(st); free(is_frozen);
+    return rc;
 }

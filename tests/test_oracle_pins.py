@@ -467,3 +467,151 @@ def test_bootstrap_closed_forms():
     np.testing.assert_allclose(r1["rates"][4:r1["end"] + 1], r2["rates"][4:r1["end"] + 1], rtol=1e-12)
     # a looser tolerance can only end the stage earlier
     assert oracle.bootstrap_replay(base, 5, 0.3)["end"] <= r1["end"]
+
+
+# ----------------------------------------------------------------------------- unfreezing on learning-rate annealing
+
+def _unfreeze_lines():
+    for line in (GOLDEN / "unfreeze_traces.txt").read_text().splitlines():
+        if line.startswith("#") or not line.strip():
+            continue
+        yield [x.strip() for x in line.split("|")]
+
+
+@pytest.mark.parametrize("f", list(_unfreeze_lines()))
+def test_unfreeze_hand_traces(f):
+    frontmost, W = bool(int(f[1])), int(f[2])
+    T = [float(v) for v in f[3].split()]
+    hist = np.array([[float(v) for v in row.split()] for row in f[4].split(";")], dtype=np.float32)
+    lr = np.array([float(v) for v in f[5].split()])
+    got = oracle.unfreeze_replay(hist, lr, W, T, frontmost=frontmost)
+    assert got["window"].tolist() == [int(v) for v in f[6].split()]
+    assert ["".join(str(int(v)) for v in row) for row in got["frozen"]] == f[7].split()
+    fired = [int(v) for v in f[8].split()]
+    assert np.nonzero(got["restarted"])[0].tolist() == fired and got["restarts"] == len(fired)
+    want = _frac_list(f[9])
+    assert np.array_equal(np.isnan(got["slopes"][0]), np.isnan(want))
+    fin = np.isfinite(want)
+    np.testing.assert_allclose(got["slopes"][0][fin], want[fin], rtol=1e-6, atol=1e-7)
+    assert np.all(np.isinf(got["slopes"][0][~np.isnan(want) & ~fin]))
+
+
+def _unfreeze_case(seed, M=4, H=160):
+    rng = np.random.default_rng(seed)
+    k = np.arange(H)
+    hist = np.stack([0.3 * np.exp(-(k % 55) / rng.uniform(2, 8)) + 0.01 * (m + 1) + 1e-4 * rng.standard_normal(H)
+                     for m in range(M)]).astype(np.float32)
+    T = rng.uniform(3e-3, 2e-2, size=M)
+    lr = 0.1 * np.power(0.1, k // 55).astype(np.float64)        # step decay by 10x at 55 and 110
+    return hist, T, lr
+
+
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("frontmost", [False, True])
+def test_unfreeze_is_plain_runs_chained(seed, frontmost):
+    """Between two restarts the run is the plain rule (already pinned) started afresh on the
+    remaining readings with the window in force; the restart is where the learning rate first
+    reaches a tenth of its value at the segment's first freeze; the window halves each time."""
+    hist, T, lr = _unfreeze_case(seed)
+    M, H = hist.shape
+    W0 = int(np.random.default_rng(seed).integers(4, 9))
+    got = oracle.unfreeze_replay(hist, lr, W0, T, frontmost=frontmost)
+    start, W, n_restarts = 0, W0, 0
+    while start < H:
+        seg = hist[:, start:]
+        if frontmost:
+            ref = oracle.frontmost_replay(seg, W, T)
+            fe = ref["freeze_eval"]
+        else:
+            runs = [oracle.plasticity_replay(seg[m], W, float(T[m])) for m in range(M)]
+            fe = np.array([r["freeze_eval"] for r in runs])
+        first = min([e for e in fe if e >= 0], default=None)
+        restart_at = None                                       # evaluation of this segment that ends it
+        if first is not None:
+            later = [i for i in range(first, H - start) if lr[start + i] <= lr[start + first] / 10 * (1 + 1e-6)]
+            restart_at = later[0] if later else None
+        end = H - start if restart_at is None else restart_at + 1
+        assert np.all(got["window"][start:start + end] == W)
+        assert got["restarted"][start:start + end].tolist() == [int(i == restart_at) for i in range(end)]
+        for i in range(end):
+            want = np.zeros(M, dtype=np.uint8) if i == restart_at else ((fe >= 0) & (fe <= i)).astype(np.uint8)
+            assert got["frozen"][start + i].tolist() == want.tolist(), (start, i)
+        if frontmost:
+            for i in range(end):
+                for m in range(M):
+                    s = got["slopes"][m, start + i]
+                    if m == ref["monitored"][i]:
+                        assert s == ref["slopes"][i]
+                    else:
+                        assert np.isnan(s)
+        else:
+            for m in range(M):
+                np.testing.assert_array_equal(got["slopes"][m, start:start + end], runs[m]["slopes"][:end])
+        if restart_at is not None:
+            n_restarts += 1
+            W = max(2, W // 2)
+        start += end
+    assert got["restarts"] == n_restarts and n_restarts >= 1
+
+
+def test_unfreeze_needs_a_freeze_and_a_tenfold_drop():
+    hist, T, lr = _unfreeze_case(3)
+    M, H = hist.shape
+    plain = [oracle.plasticity_replay(hist[m], 5, float(T[m])) for m in range(M)]
+    # a constant learning rate: nothing ever restarts, the run is the plain rule
+    got = oracle.unfreeze_replay(hist, np.full(H, 0.1), 5, T)
+    assert got["restarts"] == 0 and np.all(got["window"] == 5)
+    for m in range(M):
+        np.testing.assert_array_equal(got["slopes"][m], plain[m]["slopes"])
+    # a drop by less than ten (x0.2) does not restart either
+    got = oracle.unfreeze_replay(hist, np.where(np.arange(H) < 60, 0.1, 0.02), 5, T)
+    assert got["restarts"] == 0
+    # a tenfold drop BEFORE anything froze is not "since the frontmost freeze": the reference
+    # rate is the one at the first freeze, which is already the low one
+    first = min(p["freeze_eval"] for p in plain if p["freeze_eval"] >= 0)
+    got = oracle.unfreeze_replay(hist, np.where(np.arange(H) < first, 0.1, 0.01), 5, T)
+    assert got["restarts"] == 0
+    # tolerances that never let anything freeze: no reference rate, no restart
+    got = oracle.unfreeze_replay(hist, lr, 5, np.full(M, 1e-12))
+    assert got["restarts"] == 0 and not got["frozen"].any()
+    # the reference rate is that of the FIRST freeze, not of a later one: module 0 (constant)
+    # freezes at 2 under 0.1, module 1 (constant from 4 on) at 6 under 0.05; 0.01 is a tenth of the
+    # former only
+    two = np.array([[1] * 12, [0, 1, 2, 3, 3, 3, 3, 3, 3, 3, 3, 3]], dtype=np.float32)
+    rate = np.array([0.1] * 4 + [0.05] * 4 + [0.01] * 4)
+    got = oracle.unfreeze_replay(two, rate, 2, [0.1, 0.1])
+    assert got["frozen"][:8].tolist() == [[0, 0]] * 2 + [[1, 0]] * 4 + [[1, 1]] * 2
+    assert np.nonzero(got["restarted"])[0].tolist() == [8]
+    # a rate that is not positive carries no information
+    got = oracle.unfreeze_replay(hist, np.where(np.arange(H) < 60, 0.1, 0.0), 5, T)
+    assert got["restarts"] == 0
+
+
+def test_unfreeze_halves_the_window_with_a_floor_of_two():
+    # a constant module freezes W evaluations after each (re)start; the rate falls tenfold every 30
+    H = 150
+    lr = 0.5 * np.power(0.1, np.arange(H) // 30)
+    for W0, want in ((10, [10, 5, 2, 2, 2]), (7, [7, 3, 2, 2, 2]), (3, [3, 2, 2, 2, 2]), (2, [2, 2, 2, 2, 2])):
+        got = oracle.unfreeze_replay(np.ones((1, H), dtype=np.float32), lr, W0, [1e-3])
+        assert [int(got["window"][30 * k + 15]) for k in range(5)] == want
+        assert np.nonzero(got["restarted"])[0].tolist() == [30, 60, 90, 120]
+        # frozen W evaluations after the restart (the first evaluation of a run has no line)
+        for k in range(5):
+            s0 = 0 if k == 0 else 30 * k + 1
+            assert got["frozen"][s0 + want[k] - 1, 0] == 0 and got["frozen"][s0 + want[k], 0] == 1
+
+
+def test_unfreeze_rederives_the_automatic_tolerance():
+    # after a restart the initial three readings are those of the new run
+    k = np.arange(40)
+    run = (np.exp(-k / 4.0) + 0.05).astype(np.float32)
+    hist = np.concatenate([run, 3 * run])[None, :]
+    lr = np.where(np.arange(80) < 40, 0.1, 0.01)
+    got = oracle.unfreeze_replay(hist, lr, 4, None)
+    a = oracle.plasticity_replay_auto(run, 4)
+    b = oracle.plasticity_replay_auto(3 * run[1:], 2)
+    assert a["converged"] and b["converged"]
+    assert np.nonzero(got["restarted"])[0].tolist() == [40]
+    assert got["frozen"][:, 0].tolist() == ([0] * a["freeze_eval"] + [1] * (40 - a["freeze_eval"]) + [0]
+                                            + [0] * b["freeze_eval"] + [1] * (39 - b["freeze_eval"]))
+    np.testing.assert_array_equal(got["slopes"][0, 41:], b["slopes"])
