@@ -85,9 +85,9 @@ enum {
      * given at creation is ignored; evaluations 0..2 of a module only set its
      * tolerance and are never stale. */
     EGERIA_FLAG_AUTO_T = 64u,
-    /* Frontmost-active policy [Sec. 4.2.2 "monitors the frontmost active layer
-     * module l to avoid a fragmented frozen model"; Algorithm 1: freeze, then
-     * l <- l + 1].  Modules are ordered front to back.  Only module l = (number
+    /* Frontmost-active policy [Sec. 4.2.2: only the frontmost module that is
+     * still active is monitored, so that the frozen modules always form a prefix;
+     * Algorithm 1: freeze, then l <- l + 1].  Modules are ordered front to back.  Only module l = (number
      * of frozen modules) is advanced by an evaluation; when its counter reaches
      * W it is frozen, and the NEXT evaluation starts module l + 1 from a cleared
      * state.  out_mask is then a prefix mask (1 for the frozen modules) and
@@ -179,8 +179,8 @@ egeria_status egeria_plasticity_evaluate(egeria_ctx *ctx, void *cuda_stream, con
  * out_mask are not written and their freezing rule does not advance.  The work of
  * the active modules is spread over the whole GPU, so evaluating one module of
  * many costs about its share.  This is how the frontmost-active policy is meant
- * to be used [Sec. 3: "collects the intermediate activation of the frontmost
- * non-frozen layer"]: read out_mask back now and then and pass only the frontmost
+ * to be used [Sec. 3: only the activation of the frontmost module that is not
+ * frozen is collected]: read out_mask back now and then and pass only the frontmost
  * module that is not frozen (under EGERIA_FLAG_FRONTMOST that module reports the
  * prefix mask and the slopes of all modules; if it is left out, or all modules
  * are frozen, nothing is reported).  At least one module must be active. */
@@ -194,7 +194,7 @@ egeria_status egeria_plasticity_evaluate_subset(egeria_ctx *ctx, void *cuda_stre
                                                 uint8_t *out_mask);
 
 /* The same rule over whole histories, from a cleared state that is private to
- * the call (the context's step state is not touched).
+ * the call (the context's step state is not touched; the window is the one in force).
  *   hist             device float [M, H] row-major raw readings
  *   out_slopes       device double [M, H]; NaN after a module converged; may be NULL
  *   out_mask         device uint8 [M]
@@ -204,11 +204,58 @@ egeria_status egeria_plasticity_replay(egeria_ctx *ctx, void *cuda_stream, const
                                        int H, double *out_slopes, uint8_t *out_mask,
                                        int32_t *out_freeze_eval);
 
-/* Clear the step state (histories, counters, masks), e.g. when the caller
- * unfreezes after a learning-rate drop [Sec. 4.2.2 "Unfreezing"].  If halve_W
- * is non-zero the window is halved first (never below 2), as the paper does
- * for refreezing. */
+/* Clear the step state (histories, counters, masks, the front, the reference
+ * learning rate) by hand, e.g. for an unfreezing criterion of the caller's own
+ * [Sec. 4.2.2 "Unfreezing": cyclical schedules are left to the user; Algorithm 1
+ * customizedUnfreeze].  If halve_W is non-zero the window in force is halved,
+ * W <- max(2, floor(W / 2)), as the paper does for refreezing. */
 egeria_status egeria_plasticity_reset(egeria_ctx *ctx, void *cuda_stream, int halve_W);
+
+/* Unfreezing on learning-rate annealing [Sec. 4.2.2 "Unfreezing"; Algorithm 1, the
+ * branch after the freeze step: unfreezeAllLayers, l <- l_0].  Tell the context the
+ * learning rate in force for the evaluations that follow (host value; no CUDA work).
+ * From then on every evaluation of the rule (egeria_plasticity_step,
+ * egeria_plasticity_evaluate and their subset forms) is followed by the paper's
+ * test, all of it on the device:
+ *   - the rate in force at the first freeze after the start or the last restart is
+ *     remembered (with EGERIA_FLAG_FRONTMOST that is the first module's freeze);
+ *   - once lr <= that rate / 10 * (1 + 1e-6) -- a drop by a factor of ten or more;
+ *     the slack lets a step decay by exactly 10x count when it was computed in
+ *     single precision -- every module starts afresh (histories, counters, automatic
+ *     tolerances), the front goes back to module 0, the window in force is halved,
+ *     W <- max(2, floor(W / 2)), the remembered rate is forgotten, and the out_mask
+ *     of that evaluation is cleared.  The reading of that evaluation has been
+ *     consumed by the old state; the next evaluation is the first of the new run.
+ * A rate that is not positive (or NaN, the state after creation) switches the rule
+ * off: it is neither remembered nor tested.  The test costs one extra small kernel
+ * launch, and only after the first evaluation under a changed rate. */
+egeria_status egeria_plasticity_set_lr(egeria_ctx *ctx, double lr);
+
+/* How often the unfreezing rule has restarted the modules of this context.
+ * Waits for the stream of the last call and reads the count from the device;
+ * -1 if that fails, 0 for a NULL context. */
+int egeria_plasticity_restarts(const egeria_ctx *ctx);
+
+/* Algorithm 1 WITH its learning-rate-based unfreezing over whole histories, from a
+ * cleared state private to the call (starting with the context's window in force).
+ *   hist            device float [M, H] row-major raw readings
+ *   lr              device double [H]: learning rate at each evaluation; NULL = no
+ *                   unfreezing (then this is egeria_plasticity_replay with more outputs)
+ *   out_slopes      device double [M, H]; NaN where the module was not advanced; may be NULL
+ *   out_frozen      device uint8 [H, M]: 1 where module m is frozen after evaluation i
+ *                   (after the unfreezing test); may be NULL
+ *   out_window      device int32 [H]: window in force during evaluation i; may be NULL
+ *   out_restarted   device uint8 [H]: 1 if the unfreezing fired at the end of evaluation i; may be NULL
+ *   out_mask        device uint8 [M]: frozen at the end of the history; may be NULL
+ *   out_freeze_eval device int32 [M]: evaluation of the module's freeze in the last run, -1 if
+ *                   it is not frozen at the end; may be NULL
+ * One thread block runs all modules (a restart couples them).  More than 1280 modules
+ * give EGERIA_ERR_UNSUPPORTED_SHAPE. */
+egeria_status egeria_plasticity_replay_lr(egeria_ctx *ctx, void *cuda_stream, const float *hist,
+                                          const double *lr, int H, double *out_slopes,
+                                          uint8_t *out_frozen, int32_t *out_window,
+                                          uint8_t *out_restarted, uint8_t *out_mask,
+                                          int32_t *out_freeze_eval);
 
 /* End of the bootstrapping stage [Sec. 3 "Bootstrapping stage": the changing rate
  * of the training loss is monitored in line with the plasticity; Sec. 4.2.2: the
@@ -249,7 +296,9 @@ egeria_status egeria_plasticity_export(egeria_ctx *ctx, void *cuda_stream, void 
 egeria_status egeria_plasticity_import(egeria_ctx *ctx, void *cuda_stream, const void *host_buffer,
                                        size_t buffer_bytes);
 
-/* Current window of the context (changes only through egeria_plasticity_reset). */
+/* Window in force (halved by egeria_plasticity_reset and by the unfreezing rule).
+ * It lives on the device: waits for the stream of the last call and reads it;
+ * -1 if that fails, 0 for a NULL context. */
 int egeria_plasticity_window(const egeria_ctx *ctx);
 
 /* The per-thread-block shares of the adaptive split (see EGERIA_FLAG_EQUAL_SPLIT).
@@ -278,6 +327,17 @@ egeria_status egeria_debug_plan_weighted(int M, const int64_t *d, int b, int n_c
                                          const float *weights, int32_t *out_units, int max_units,
                                          int *n_units);
 
+/* Test hook for the bounded waits: the NEXT evaluation kernel of this context (tensor-core
+ * modules) runs with every wait limited to one millisecond instead of two seconds, and with one
+ * hand-shake of its first thread block left out on purpose, so that the waits that depend on it
+ * run out: kind 1 = that block's loader issues no load; kind 2 = its MMA issuer stops after its
+ * first pipeline stage; 0 = cancel.  The block then leaves through the give-up path (waits for
+ * its loads in flight, frees its tensor memory), the kernel returns, the losses of that
+ * evaluation are not written and egeria_device_status reports EGERIA_ERR_TIMEOUT once; the
+ * evaluation after that is an ordinary one.  Nothing traps or spins without bound.  Not for
+ * production use. */
+egeria_status egeria_debug_stall_next(egeria_ctx *ctx, int kind);
+
 /* Synchronise the stream of the last call and report the device status word:
  * EGERIA_OK, or EGERIA_ERR_TIMEOUT if a bounded wait inside a kernel ran out
  * (the kernel then skipped its remaining work; results are invalid). */
@@ -286,27 +346,42 @@ egeria_status egeria_device_status(egeria_ctx *ctx);
 /* Plasticity of ONE module with no workspace and no allocation of any kind.
  * The paper has no counterpart to this call; it exists for callers that cannot
  * obtain device memory at the moment they need an evaluation: code that runs
- * where cudaMalloc is forbidden or would stall (a framework whose caching
- * allocator owns all of HBM so that a raw allocation fails, a latency-critical
- * loop that must avoid the device-wide synchronisation an allocation or free
- * implies, a plugin that is handed a stream but no allocator).  Such callers
- * cannot size and allocate the workspace a context needs either.
+ * where cudaMalloc is forbidden or fails (a framework whose caching allocator
+ * owns all of HBM so that a raw allocation fails, a plugin that is handed a
+ * stream but no allocator, code that must not take the device-wide
+ * synchronisation an allocation or free implies).  Such callers cannot size and
+ * allocate the workspace a context needs either.
  *
  * The scratch of this call (partial Gram matrices, work split, tensor maps) is
  * a fixed 6 MiB array inside the library image; every GPU that loads the
  * library holds it until the process exits.  The price is a size limit:
  *   b  2..128 (larger b returns EGERIA_ERR_UNSUPPORTED_SHAPE), any d >= 1,
  * and the feature axis is split over 32 CTAs only, so it is slower than a
- * context on large d.  Same arithmetic as egeria_sp_loss_batch.
+ * context on large d; each call also builds its work split and tensor maps on
+ * the host and sends them with one small copy (a context keeps them on the
+ * device).  Same arithmetic as egeria_sp_loss_batch.
  *   At, Ar    device bf16 [b, d] (caller-owned)     out_loss  device float [1]
  * The first call on each device looks up the array's device address and sets
- * kernel attributes (with that device current); make that first call outside
- * any stream capture.  All calls share the one array, which keeps the previous
- * call's contents (the call clears the words that must start at zero): two
- * calls that overlap on the GPU, from different streams or threads, race.
- * Calls on one stream are safe back to back.  Not thread-safe. */
+ * kernel attributes (with that device current).  No call of this entry point
+ * may be recorded into a CUDA graph: every call copies from host memory that
+ * is gone when it returns, so a call on a capturing stream is refused with
+ * EGERIA_ERR_INVALID_ARG (that goes for the first call and for all later ones).
+ * All calls share the one array, which keeps the previous call's contents (the
+ * call clears the words that must start at zero): two calls that overlap on
+ * the GPU, from different streams or threads, race.  Calls on one stream are
+ * safe back to back.  Not thread-safe.
+ * If a bounded wait inside the kernel runs out, the kernel gives up and
+ * out_loss is left NaN; egeria_sp_loss_static_status tells that case from a
+ * NaN that came from the inputs. */
 egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At, const void *Ar, int b,
                                     int64_t d, float *out_loss);
+
+/* Status word of the last egeria_sp_loss_static call on the current device:
+ * EGERIA_OK, or EGERIA_ERR_TIMEOUT if a bounded wait inside its kernel ran out.
+ * Call it after synchronising the stream of that call and before the next one
+ * (which clears the word); it copies four bytes from the device and allocates
+ * nothing. */
+egeria_status egeria_sp_loss_static_status(void);
 
 /* Measurement hook (needs EGERIA_FLAG_TIME_GRAM): device time, in milliseconds,
  * spent in the evaluation kernels of the egeria_sp_loss_batch /

@@ -32,6 +32,7 @@ EXPORTS = [
     "egeria_split_weights", "egeria_status_string", "egeria_bootstrap_step", "egeria_bootstrap_replay",
     "egeria_bootstrap_reset", "egeria_plasticity_state_bytes", "egeria_plasticity_export", "egeria_plasticity_import",
     "egeria_sp_loss_subset", "egeria_plasticity_evaluate_subset",
+    "egeria_sp_loss_static_status", "egeria_debug_stall_next", "egeria_plasticity_set_lr", "egeria_plasticity_restarts", "egeria_plasticity_replay_lr",
 ]
 
 
@@ -71,6 +72,9 @@ def lib() -> ctypes.CDLL:
     L.egeria_plasticity_replay.argtypes = [vp, vp, vp, ctypes.c_int, vp, vp, vp]
     L.egeria_plasticity_reset.argtypes = [vp, vp, ctypes.c_int]
     L.egeria_plasticity_window.argtypes = [vp]
+    L.egeria_plasticity_restarts.argtypes = [vp]
+    L.egeria_plasticity_set_lr.argtypes = [vp, ctypes.c_double]
+    L.egeria_plasticity_replay_lr.argtypes = [vp, vp, vp, vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
     L.egeria_debug_dump_gram.argtypes = [vp, vp, ctypes.c_int, vp, vp]
     L.egeria_debug_plan.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int,
                                     ctypes.POINTER(ctypes.c_int32), ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
@@ -88,6 +92,8 @@ def lib() -> ctypes.CDLL:
     L.egeria_device_status.argtypes = [vp]
     L.egeria_gram_kernel_time.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
     L.egeria_sp_loss_static.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_int64, vp]
+    L.egeria_sp_loss_static_status.argtypes = []
+    L.egeria_debug_stall_next.argtypes = [vp, ctypes.c_int]
     L.egeria_launch_count.argtypes = [vp]
     L.egeria_launch_count.restype = ctypes.c_int64
     L.egeria_status_string.argtypes = [ctypes.c_int]
@@ -166,6 +172,13 @@ def egeria_sp_loss_static(At: torch.Tensor, Ar: torch.Tensor, out_loss: Optional
                                          int(At.shape[1]), out_loss.data_ptr())
     _check(st, "egeria_sp_loss_static")
     return out_loss
+
+
+def egeria_sp_loss_static_status(device=None) -> int:
+    """Status word of the last egeria_sp_loss_static call on `device` (the current one if None);
+    call it after synchronising that call's stream."""
+    with torch.cuda.device(device):
+        return int(lib().egeria_sp_loss_static_status())
 
 
 class Context:
@@ -323,6 +336,35 @@ class Context:
         _check(st, "egeria_plasticity_replay")
         return slopes, mask, freeze_eval
 
+    def egeria_plasticity_replay_lr(self, hist: torch.Tensor, lr: Optional[torch.Tensor],
+                                    stream: Optional[torch.cuda.Stream] = None):
+        """Whole histories with the unfreezing rule: (slopes [M, H], frozen [H, M], window [H],
+        restarted [H], mask [M], freeze_eval [M]) device tensors."""
+        assert hist.is_cuda and hist.dtype == torch.float32 and hist.dim() == 2 and hist.shape[0] == self.M
+        hist = hist.contiguous()
+        H = int(hist.shape[1])
+        if lr is not None:
+            assert lr.is_cuda and lr.dtype == torch.float64 and lr.numel() == H
+            lr = lr.contiguous()
+        slopes = torch.empty((self.M, H), dtype=torch.float64, device=self.device)
+        frozen = torch.empty((H, self.M), dtype=torch.uint8, device=self.device)
+        window = torch.empty(max(H, 1), dtype=torch.int32, device=self.device)
+        restarted = torch.empty(max(H, 1), dtype=torch.uint8, device=self.device)
+        mask = torch.empty(self.M, dtype=torch.uint8, device=self.device)
+        freeze_eval = torch.empty(self.M, dtype=torch.int32, device=self.device)
+        st = lib().egeria_plasticity_replay_lr(self._h, _stream_ptr(stream), hist.data_ptr(),
+                                               lr.data_ptr() if lr is not None else None, H, slopes.data_ptr(),
+                                               frozen.data_ptr(), window.data_ptr(), restarted.data_ptr(),
+                                               mask.data_ptr(), freeze_eval.data_ptr())
+        _check(st, "egeria_plasticity_replay_lr")
+        return slopes, frozen, window[:H], restarted[:H], mask, freeze_eval
+
+    def egeria_plasticity_set_lr(self, lr: float) -> None:
+        _check(lib().egeria_plasticity_set_lr(self._h, ctypes.c_double(lr)), "egeria_plasticity_set_lr")
+
+    def egeria_plasticity_restarts(self) -> int:
+        return int(lib().egeria_plasticity_restarts(self._h))
+
     def egeria_plasticity_reset(self, halve_W: bool = False, stream: Optional[torch.cuda.Stream] = None) -> None:
         _check(lib().egeria_plasticity_reset(self._h, _stream_ptr(stream), int(bool(halve_W))),
                "egeria_plasticity_reset")
@@ -376,6 +418,9 @@ class Context:
         st = lib().egeria_debug_dump_gram(self._h, _stream_ptr(stream), int(module), gt.data_ptr(), gr.data_ptr())
         _check(st, "egeria_debug_dump_gram")
         return gt, gr
+
+    def egeria_debug_stall_next(self, kind: int) -> None:
+        _check(lib().egeria_debug_stall_next(self._h, int(kind)), "egeria_debug_stall_next")
 
     def egeria_device_status(self) -> int:
         return int(lib().egeria_device_status(self._h))

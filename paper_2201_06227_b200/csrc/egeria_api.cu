@@ -2,6 +2,7 @@
 // static work split, tensor-map encoding and kernel launches.  See include/egeria.h.
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stdint.h>
 #include <string.h>
 
@@ -23,6 +24,7 @@ constexpr int kPlanSlots = 16; // device-side plans kept, keyed by (b, activatio
 constexpr int kCalibLaunches = 3;  // launches whose per-CTA streaming rates set the split weights
 constexpr size_t kMaxTimedCalls = 4096;  // EGERIA_FLAG_TIME_GRAM: calls timed between two queries
 constexpr int kCalibRounds = 3;    // times the weights are re-measured under the split they produced
+constexpr uint64_t kTestWaitLimitNs = 1000000ull;  // 1 ms: wait limit of a launch under egeria_debug_stall_next
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -30,8 +32,9 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct Layout {
     size_t status, cta_log, rowloss, tickets, fin_ctr, T, losses, keep, slots, staging, total;
     // the freezing-rule state, one contiguous region [rule0, rule_end) (what export / import copy)
-    size_t rule0, raw, plist, n_evals, counter, freeze_eval, last_slope, Tauto, smax, front, boot_raw, boot_plist,
-        boot_ints, rule_end;
+    size_t rule0, raw, plist, n_evals, counter, freeze_eval, last_slope, Tauto, smax, front, unfreeze, boot_raw,
+        boot_plist, boot_ints, rule_end;
+    size_t replay_raw, replay_plist;  // windows of egeria_plasticity_replay_lr ([M][W] doubles each)
     size_t slot_bytes_cap;  // bytes reserved for partial slots
     // Device-side plans (tensor maps, pointers, unit table, per-CTA ranges, slot ranges): kPlanSlots
     // regions of plan_stride bytes from plan0; the offsets below are relative to a region.
@@ -84,10 +87,13 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
     L.Tauto = take((size_t)M * sizeof(double));
     L.smax = take((size_t)M * sizeof(double));
     L.front = take(sizeof(unsigned long long));
+    L.unfreeze = take(32);  // reference learning rate (8 bytes), window in force, restarts
     L.boot_raw = take((size_t)W * sizeof(double));
     L.boot_plist = take((size_t)W * sizeof(double));
     L.boot_ints = take(2 * sizeof(int32_t));
     L.rule_end = off;
+    L.replay_raw = take((size_t)M * W * sizeof(double));
+    L.replay_plist = take((size_t)M * W * sizeof(double));
     L.losses = take((size_t)M * sizeof(float));
     L.keep = off;
     if (flags & EGERIA_FLAG_KEEP_GRAMS) take((size_t)M * 2 * b_max * b_max * sizeof(float));
@@ -131,7 +137,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 using namespace egeria;
 
 struct egeria_ctx {
-    int M = 0, b_max = 0, W = 0, W_cap = 0;
+    int M = 0, b_max = 0, W_cap = 0;  // W_cap: the window given at creation (the one in force is on the device)
+    double lr = NAN;        // learning rate in force (egeria_plasticity_set_lr); NaN: never given
+    double lr_checked = NAN;  // rate of the last evaluation of the rule (the unfreezing test runs when it changes)
     uint32_t flags = 0;
     std::vector<int64_t> d;
     uint8_t *ws = nullptr;
@@ -154,11 +162,14 @@ struct egeria_ctx {
     uint64_t use_clock = 0;
     std::vector<uint8_t> pack;  // host image of one plan region (when there is no pinned one)
     uint8_t *pinned_plans = nullptr;  // kPlanSlots images of plan_stride bytes: uploads that do not stall the stream
+    cudaEvent_t plan_uploaded[kPlanSlots] = {};  // recorded after the upload from image i: the image is free again
+    bool plan_upload_pending[kPlanSlots] = {};   // once the event has completed
     uint8_t *plan_region(int i) const { return ws + L.plan0 + (size_t)i * L.plan_stride; }
     cudaStream_t last_stream = nullptr;
     int64_t launches = 0;
     uint32_t tc_launches = 0;  // selects the set of progress counters the next tensor-core launch uses
     uint32_t rule_evals = 0;   // evaluations of the freezing rule enqueued so far (the serial of the last one)
+    uint32_t stall_next = 0;   // test hook: give-up path of the next tensor-core launch (egeria_debug_stall_next)
     // Split weights: one per CTA, from the streaming rates the CTAs report (SMs do not all get
     // the same share of HBM bandwidth; the CTA -> SM placement repeats from launch to launch).
     std::vector<float> weights;
@@ -204,6 +215,9 @@ struct egeria_ctx {
         st.front = at<unsigned long long>(L.front);
         st.T = at<float>(L.T);
         st.W_cap = W_cap;
+        st.lr_ref = at<unsigned long long>(L.unfreeze);
+        st.W_cur = at<int32_t>(L.unfreeze + 8);
+        st.restarts = at<int32_t>(L.unfreeze + 12);
         return st;
     }
 };
@@ -289,7 +303,6 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     if (!ctx) return EGERIA_ERR_INVALID_ARG;
     ctx->M = M;
     ctx->b_max = b_max;
-    ctx->W = W;
     ctx->W_cap = W;
     ctx->flags = flags;
     ctx->d.assign(d, d + M);
@@ -322,10 +335,15 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     ctx->weights.assign(ctx->n_ctas, 1.0f);
     {
         void *hp = nullptr;
-        if (cudaHostAlloc(&hp, L.plan_stride * kPlanSlots, cudaHostAllocDefault) == cudaSuccess)
+        bool ok = (cudaHostAlloc(&hp, L.plan_stride * kPlanSlots, cudaHostAllocDefault) == cudaSuccess);
+        for (int i = 0; ok && i < kPlanSlots; ++i)
+            ok = (cudaEventCreateWithFlags(&ctx->plan_uploaded[i], cudaEventDisableTiming) == cudaSuccess);
+        if (ok) {
             ctx->pinned_plans = static_cast<uint8_t *>(hp);
-        else
+        } else {
             (void)cudaGetLastError();  // fall back to pageable staging
+            if (hp) cudaFreeHost(hp);
+        }
     }
     if (!(flags & EGERIA_FLAG_EQUAL_SPLIT)) {
         void *hp = nullptr;
@@ -342,15 +360,13 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.fin_ctr, 0, (size_t)2 * M * sizeof(FinCounters));
     if (e == cudaSuccess) e = cudaMemcpy(ctx->ws + L.T, Th.data(), (size_t)M * sizeof(float), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) {
-        plasticity_clear_kernel<<<(M + 127) / 128, 128>>>(ctx->slope_state(), M);
+        plasticity_clear_kernel<<<(M + 127) / 128, 128>>>(ctx->slope_state(), M, W, 0);
         bootstrap_clear_kernel<<<1, 1>>>(ctx->boot_state());
         ctx->launches += 2;
         e = cudaDeviceSynchronize();
     }
     if (e != cudaSuccess) {
-        if (ctx->host_log) cudaFreeHost(ctx->host_log);
-        if (ctx->pinned_plans) cudaFreeHost(ctx->pinned_plans);
-        delete ctx;
+        egeria_plasticity_destroy(ctx);
         return EGERIA_ERR_CUDA;
     }
     *out = ctx;
@@ -360,13 +376,32 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
 egeria_status egeria_plasticity_destroy(egeria_ctx *ctx) {
     if (!ctx) return EGERIA_ERR_INVALID_ARG;
     for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->plan_uploaded)
+        if (e) cudaEventDestroy(e);
     if (ctx->host_log) cudaFreeHost(ctx->host_log);
     if (ctx->pinned_plans) cudaFreeHost(ctx->pinned_plans);
     delete ctx;
     return EGERIA_OK;
 }
 
-int egeria_plasticity_window(const egeria_ctx *ctx) { return ctx ? ctx->W : 0; }
+// The window in force and the number of restarts live on the device (the device halves the one
+// and counts the other): wait for the stream and read them.
+static int read_unfreeze_word(const egeria_ctx *ctx, size_t byte_off) {
+    if (!ctx) return 0;
+    if (cudaStreamSynchronize(ctx->last_stream) != cudaSuccess) return -1;
+    int32_t v = 0;
+    if (cudaMemcpy(&v, ctx->ws + ctx->L.unfreeze + byte_off, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return -1;
+    return v;
+}
+int egeria_plasticity_window(const egeria_ctx *ctx) { return read_unfreeze_word(ctx, 8); }
+int egeria_plasticity_restarts(const egeria_ctx *ctx) { return read_unfreeze_word(ctx, 12); }
+
+egeria_status egeria_plasticity_set_lr(egeria_ctx *ctx, double lr) {
+    if (!ctx) return EGERIA_ERR_INVALID_ARG;
+    ctx->lr = lr;
+    return EGERIA_OK;
+}
 
 int egeria_split_weights(egeria_ctx *ctx, float *out_weights, int max_weights) {
     if (!ctx) return -1;
@@ -473,8 +508,13 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
 
     uint8_t *img;
     if (ctx->pinned_plans) {
-        // One pinned image per plan slot: the copy below is truly asynchronous, and an image is not
-        // written again before its slot is replaced, i.e. after at least kPlanSlots - 1 other uploads.
+        // One pinned image per plan slot: the copy below is truly asynchronous, so the image must not
+        // be rewritten while an earlier upload from it is still queued (a caller whose pointers change
+        // on every call can run more than kPlanSlots evaluations ahead of the GPU).
+        if (ctx->plan_upload_pending[lru]) {
+            EG_CUDA(cudaEventSynchronize(ctx->plan_uploaded[lru]));
+            ctx->plan_upload_pending[lru] = false;
+        }
         img = ctx->pinned_plans + (size_t)lru * L.plan_stride;
         memset(img, 0, L.plan_stride);
     } else {
@@ -497,6 +537,10 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
     memcpy(img + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo));
     // From pageable memory the runtime stages the bytes before returning, so `pack` may be reused.
     EG_CUDA(cudaMemcpyAsync(ctx->plan_region(lru), img, L.plan_stride, cudaMemcpyHostToDevice, stream));
+    if (ctx->pinned_plans) {
+        EG_CUDA(cudaEventRecord(ctx->plan_uploaded[lru], stream));
+        ctx->plan_upload_pending[lru] = true;
+    }
     e.b = b;
     e.weights_version = ctx->weights_version;
     e.At.assign(At, At + M);
@@ -560,6 +604,22 @@ static egeria_status set_attrs(egeria_ctx *ctx) {
 
 }  // namespace egeria
 
+// The unfreezing test of Algorithm 1 after an evaluation of the rule [Sec. 4.2.2 "Unfreezing"].
+// Its outcome can change only when the learning rate does (the reference rate is set at a freeze
+// to the rate then in force, which is not a tenth of itself), so the kernel is launched only after
+// the first evaluation under a new rate.
+static egeria_status unfreeze_test(egeria_ctx *ctx, cudaStream_t stream, uint8_t *out_mask) {
+    const double lr = ctx->lr;
+    if (!(lr > 0.0)) return EGERIA_OK;  // no rate given (or not a usable one): the rule is off
+    const bool changed = (ctx->lr_checked > 0.0) && (lr != ctx->lr_checked);
+    ctx->lr_checked = lr;
+    if (!changed) return EGERIA_OK;
+    unfreeze_check_kernel<<<1, 128, 0, stream>>>(ctx->slope_state(), ctx->M, lr, out_mask);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
 static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void *const *At_in,
                                   const void *const *Ar_in, int b, const int64_t *d, float *out_losses, bool fuse_step,
                                   double *out_slopes, uint8_t *out_mask, const uint8_t *active = nullptr) {
@@ -621,7 +681,7 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
     fc.rowloss = ctx->at<double>(L.rowloss);
     fc.keep = (ctx->flags & EGERIA_FLAG_KEEP_GRAMS) ? ctx->at<float>(L.keep) : nullptr;
     fc.fuse_step = fuse_step ? 1 : 0;
-    fc.W = ctx->W;
+    fc.lr = ctx->lr;
     fc.rule_flags = ctx->rule_flags();
     if (fuse_step) ctx->rule_evals++;
     fc.rule_serial = ctx->rule_evals;
@@ -646,6 +706,9 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
                             P.all_ctas_busy_tc;
         tp.log = log_it ? ctx->at<CtaLog>(L.cta_log) : nullptr;
         tp.serial = ctx->tc_launches + 1;
+        tp.test_stall = ctx->stall_next;
+        tp.wait_limit_ns = ctx->stall_next ? kTestWaitLimitNs : kWaitLimitNs;
+        ctx->stall_next = 0;
         if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
         if (log_it) {
             const int k = ctx->calib_enqueued;
@@ -680,6 +743,7 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         if (launch_finalize(fp, ctx->M, b, stream) != cudaSuccess) return EGERIA_ERR_CUDA;
         ctx->launches++;
     }
+    if (fuse_step) return unfreeze_test(ctx, stream, out_mask);
     return EGERIA_OK;
 }
 
@@ -737,11 +801,11 @@ egeria_status egeria_plasticity_step(egeria_ctx *ctx, void *cuda_stream, const f
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     ctx->last_stream = stream;
     ctx->rule_evals++;
-    plasticity_step_kernel<<<ctx->M, 32, 0, stream>>>(ctx->slope_state(), ctx->M, ctx->W, ctx->rule_flags(),
-                                                      ctx->rule_evals, losses, out_slopes, out_mask);
+    plasticity_step_kernel<<<ctx->M, 32, 0, stream>>>(ctx->slope_state(), ctx->M, ctx->rule_flags(), ctx->rule_evals,
+                                                      ctx->lr, losses, out_slopes, out_mask);
     if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
     ctx->launches++;
-    return EGERIA_OK;
+    return unfreeze_test(ctx, stream, out_mask);
 }
 
 egeria_status egeria_plasticity_replay(egeria_ctx *ctx, void *cuda_stream, const float *hist, int H,
@@ -750,8 +814,27 @@ egeria_status egeria_plasticity_replay(egeria_ctx *ctx, void *cuda_stream, const
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     ctx->last_stream = stream;
     const int grid = (ctx->flags & EGERIA_FLAG_FRONTMOST) ? 1 : ctx->M;
-    plasticity_replay_kernel<<<grid, 32, 2 * (size_t)ctx->W * sizeof(double), stream>>>(
-        ctx->at<float>(ctx->L.T), ctx->M, ctx->W, ctx->rule_flags(), hist, H, out_slopes, out_mask, out_freeze_eval);
+    plasticity_replay_kernel<<<grid, 32, 2 * (size_t)ctx->W_cap * sizeof(double), stream>>>(
+        ctx->at<float>(ctx->L.T), ctx->M, ctx->slope_state().W_cur, ctx->W_cap, ctx->rule_flags(), hist, H, out_slopes,
+        out_mask, out_freeze_eval);
+    if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
+    ctx->launches++;
+    return EGERIA_OK;
+}
+
+egeria_status egeria_plasticity_replay_lr(egeria_ctx *ctx, void *cuda_stream, const float *hist, const double *lr,
+                                          int H, double *out_slopes, uint8_t *out_frozen, int32_t *out_window,
+                                          uint8_t *out_restarted, uint8_t *out_mask, int32_t *out_freeze_eval) {
+    if (!ctx || !hist || H < 0) return EGERIA_ERR_INVALID_ARG;
+    const size_t smem = (size_t)ctx->M * sizeof(ReplayModule);
+    if (smem > 40 * 1024) return EGERIA_ERR_UNSUPPORTED_SHAPE;  // per-module scalars live in shared memory
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->last_stream = stream;
+    int warps = ctx->M < 32 ? ctx->M : 32;
+    plasticity_replay_lr_kernel<<<1, 32 * warps, smem, stream>>>(
+        ctx->at<float>(ctx->L.T), ctx->at<double>(ctx->L.replay_raw), ctx->at<double>(ctx->L.replay_plist), ctx->W_cap,
+        ctx->slope_state().W_cur, ctx->M, ctx->rule_flags(), hist, lr, H, out_slopes, out_frozen, out_window,
+        out_restarted, out_mask, out_freeze_eval);
     if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
     ctx->launches++;
     return EGERIA_OK;
@@ -761,11 +844,7 @@ egeria_status egeria_plasticity_reset(egeria_ctx *ctx, void *cuda_stream, int ha
     if (!ctx) return EGERIA_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     ctx->last_stream = stream;
-    if (halve_W) {
-        int w = ctx->W / 2;
-        ctx->W = w < 2 ? (ctx->W < 2 ? ctx->W : 2) : w;
-    }
-    plasticity_clear_kernel<<<(ctx->M + 127) / 128, 128, 0, stream>>>(ctx->slope_state(), ctx->M);
+    plasticity_clear_kernel<<<(ctx->M + 127) / 128, 128, 0, stream>>>(ctx->slope_state(), ctx->M, 0, halve_W ? 1 : 0);
     if (cudaGetLastError() != cudaSuccess) return EGERIA_ERR_CUDA;
     ctx->launches++;
     return EGERIA_OK;
@@ -810,9 +889,10 @@ egeria_status egeria_bootstrap_reset(egeria_ctx *ctx, void *cuda_stream) {
 // What export writes in front of the raw state: enough to refuse a buffer from another set-up.
 struct StateHeader {
     uint32_t magic;
-    int32_t M, W_cap, W;
+    int32_t M, W_cap, pad;
     uint32_t rule_evals, flags;
     uint64_t state_bytes;
+    double lr, lr_checked;
 };
 constexpr uint32_t kStateMagic = 0x45474552u;  // "EGER"
 
@@ -829,7 +909,9 @@ egeria_status egeria_plasticity_export(egeria_ctx *ctx, void *cuda_stream, void 
     h.magic = kStateMagic;
     h.M = ctx->M;
     h.W_cap = ctx->W_cap;
-    h.W = ctx->W;
+    h.pad = 0;
+    h.lr = ctx->lr;
+    h.lr_checked = ctx->lr_checked;
     h.rule_evals = ctx->rule_evals;
     h.flags = ctx->flags & (EGERIA_FLAG_SIGNED_SLOPE | EGERIA_FLAG_AUTO_T | EGERIA_FLAG_FRONTMOST);
     h.state_bytes = ctx->L.rule_end - ctx->L.rule0;
@@ -846,7 +928,7 @@ egeria_status egeria_plasticity_import(egeria_ctx *ctx, void *cuda_stream, const
     memcpy(&h, host_buffer, sizeof(h));
     const uint32_t rule_bits = ctx->flags & (EGERIA_FLAG_SIGNED_SLOPE | EGERIA_FLAG_AUTO_T | EGERIA_FLAG_FRONTMOST);
     if (h.magic != kStateMagic || h.M != ctx->M || h.W_cap != ctx->W_cap || h.flags != rule_bits ||
-        h.state_bytes != ctx->L.rule_end - ctx->L.rule0 || h.W < 1 || h.W > ctx->W_cap)
+        h.state_bytes != ctx->L.rule_end - ctx->L.rule0)
         return EGERIA_ERR_INVALID_ARG;
     if (buffer_bytes < sizeof(h) + h.state_bytes) return EGERIA_ERR_WORKSPACE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -854,7 +936,8 @@ egeria_status egeria_plasticity_import(egeria_ctx *ctx, void *cuda_stream, const
     EG_CUDA(cudaMemcpyAsync(ctx->ws + ctx->L.rule0, static_cast<const uint8_t *>(host_buffer) + sizeof(h), h.state_bytes,
                             cudaMemcpyHostToDevice, stream));
     EG_CUDA(cudaStreamSynchronize(stream));  // the buffer may be pageable: it is free again on return
-    ctx->W = h.W;
+    ctx->lr = h.lr;
+    ctx->lr_checked = h.lr_checked;
     ctx->rule_evals = h.rule_evals;
     return EGERIA_OK;
 }
@@ -890,6 +973,12 @@ egeria_status egeria_gram_kernel_time(egeria_ctx *ctx, double *total_ms, int64_t
     return EGERIA_OK;
 }
 
+egeria_status egeria_debug_stall_next(egeria_ctx *ctx, int kind) {
+    if (!ctx || kind < 0 || kind > 2) return EGERIA_ERR_INVALID_ARG;
+    ctx->stall_next = (uint32_t)kind;
+    return EGERIA_OK;
+}
+
 egeria_status egeria_device_status(egeria_ctx *ctx) {
     if (!ctx) return EGERIA_ERR_INVALID_ARG;
     EG_CUDA(cudaStreamSynchronize(ctx->last_stream));
@@ -920,6 +1009,7 @@ constexpr int kStaticMaxB = 128;                   // largest b of the allocatio
 constexpr int kStaticCtas = 32;                    // CTAs the feature axis is split over
 constexpr size_t kStaticScratchBytes = 6u << 20;   // 6 MiB
 constexpr int kStaticMaxDevices = 64;
+constexpr size_t kStaticTableBytes = 4096;         // host image of the tables at the start of the array
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
@@ -999,6 +1089,11 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     if (s != EGERIA_OK) return s;
     unsigned char *ws = sd->scratch;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // The call copies from host memory that dies when it returns; captured into a graph, those
+    // copies would read dead memory at replay.  Refuse rather than record them.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    EG_CUDA(cudaStreamIsCapturing(stream, &capturing));
+    if (capturing != cudaStreamCaptureStatusNone) return EGERIA_ERR_INVALID_ARG;
 
     const uint8_t tc_ok = (reinterpret_cast<uintptr_t>(At) % 16 == 0) && (reinterpret_cast<uintptr_t>(Ar) % 16 == 0) &&
                           (d % 8 == 0);
@@ -1022,20 +1117,26 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
                 return EGERIA_ERR_CUDA;
         }
     }
-    const ModulePtrs mod{At, Ar, d};
     // The array keeps whatever the previous call left: the ticket, the status word and the
     // progress counters must start at zero; everything else is overwritten before it is read.
+    // The tables the kernels read (tensor maps, pointers, units, ranges, slot ranges) lie next to
+    // each other at the start of the array and go up in ONE copy from one host image.  The image is
+    // ordinary (pageable) memory: the runtime stages such a copy before it returns, so the image
+    // may die with this call.
+    unsigned char image[kStaticTableBytes];
+    if (L.rowloss > sizeof(image)) return EGERIA_ERR_WORKSPACE;
+    memset(image, 0, L.rowloss);
+    const ModulePtrs mod{At, Ar, d};
+    memcpy(image + L.tmaps, maps, sizeof(maps));
+    memcpy(image + L.modules, &mod, sizeof(mod));
+    memcpy(image + L.units, P.units.data(), P.units.size() * sizeof(Unit));
+    memcpy(image + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t));
+    memcpy(image + L.cta_begin_simt, P.cta_begin_simt.data(), P.cta_begin_simt.size() * sizeof(int32_t));
+    memcpy(image + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo));
     EG_CUDA(cudaMemsetAsync(ws + L.ticket, 0, 2 * sizeof(int32_t) + 2 * sizeof(FinCounters), stream));
-    EG_CUDA(cudaMemcpyAsync(ws + L.tmaps, maps, sizeof(maps), cudaMemcpyHostToDevice, stream));
-    EG_CUDA(cudaMemcpyAsync(ws + L.modules, &mod, sizeof(mod), cudaMemcpyHostToDevice, stream));
-    EG_CUDA(cudaMemcpyAsync(ws + L.units, P.units.data(), P.units.size() * sizeof(Unit), cudaMemcpyHostToDevice,
-                            stream));
-    EG_CUDA(cudaMemcpyAsync(ws + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t),
-                            cudaMemcpyHostToDevice, stream));
-    EG_CUDA(cudaMemcpyAsync(ws + L.cta_begin_simt, P.cta_begin_simt.data(), P.cta_begin_simt.size() * sizeof(int32_t),
-                            cudaMemcpyHostToDevice, stream));
-    EG_CUDA(cudaMemcpyAsync(ws + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo), cudaMemcpyHostToDevice,
-                            stream));
+    EG_CUDA(cudaMemcpyAsync(ws, image, L.rowloss, cudaMemcpyHostToDevice, stream));
+    // A kernel that gives up (a bounded wait ran out) writes no loss: leave a NaN there for that case.
+    EG_CUDA(cudaMemsetAsync(out_loss, 0xff, sizeof(float), stream));
 
     const int64_t slot_floats = slot_floats_of_mode(P.mode);
     int32_t *ticket = reinterpret_cast<int32_t *>(ws + L.ticket);
@@ -1048,7 +1149,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     fc.rowloss = reinterpret_cast<double *>(ws + L.rowloss);
     fc.keep = nullptr;
     fc.fuse_step = 0;
-    fc.W = 0;
+    fc.lr = NAN;
     fc.rule_flags = 0;
     fc.rule_serial = 0;
     fc.M = 1;
@@ -1066,6 +1167,8 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         tp.ctr_next = tp.ctr + 1;
         tp.log = nullptr;
         tp.serial = 0;
+        tp.test_stall = 0;
+        tp.wait_limit_ns = kWaitLimitNs;
         tp.M = 1;
         tp.fin = fc;
         if (launch_tc_mode(P.mode, kStaticCtas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
@@ -1086,4 +1189,16 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         if (launch_finalize(fp, 1, b, stream) != cudaSuccess) return EGERIA_ERR_CUDA;
     }
     return EGERIA_OK;
+}
+
+extern "C" egeria_status egeria_sp_loss_static_status(void) {
+    int dev = 0;
+    EG_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kStaticMaxDevices || !g_static_dev[dev].scratch) return EGERIA_OK;  // nothing ran here yet
+    const StaticLayout L = static_layout();
+    int32_t word = 0;
+    EG_CUDA(cudaMemcpy(&word, g_static_dev[dev].scratch + L.ticket + sizeof(int32_t), sizeof(word),
+                       cudaMemcpyDeviceToHost));
+    if (word == kStatusTimeout) return EGERIA_ERR_TIMEOUT;
+    return word == 0 ? EGERIA_OK : EGERIA_ERR_CUDA;
 }

@@ -32,10 +32,10 @@ struct FinCommon {
     float *keep;            // [M][2][b*b] normalised matrices, or nullptr
     // fused freezing-rule step (fuse_step != 0): Algorithm 1 on the loss just computed
     int32_t fuse_step;
-    int32_t W;
     int32_t rule_flags;     // RuleFlags
     uint32_t rule_serial;   // number of this evaluation of the rule, from 1 (frontmost policy)
     int32_t M;
+    double lr;              // learning rate in force (not positive or NaN: unknown), for the unfreezing rule
     SlopeState st;
     double *out_slopes;     // [M] or nullptr
     uint8_t *out_mask;      // [M] or nullptr
@@ -227,7 +227,7 @@ __device__ __forceinline__ void finalize_module_total(const FinCommon &p, int m,
         v[j] = (r < b) ? __ldcg(&p.rowloss[(int64_t)m * kMaxB + r]) : 0.0;
     }
     StepLoaded L;
-    if (p.fuse_step) L = plasticity_step_load(p.st, m, p.W, lane);  // in flight together with the row terms
+    if (p.fuse_step) L = plasticity_step_load(p.st, m, lane);  // in flight together with the row terms
     double s = 0.0;
 #pragma unroll
     for (int j = 0; j < kMaxB / 32; ++j) s += v[j];
@@ -235,7 +235,7 @@ __device__ __forceinline__ void finalize_module_total(const FinCommon &p, int m,
     const float loss = (float)(s / ((double)b * (double)b));
     if (lane == 0) p.out_losses[m] = loss;
     if (p.fuse_step)
-        plasticity_rule_step(p.st, L, m, p.M, p.W, p.rule_flags, p.rule_serial, loss, p.out_slopes, p.out_mask, lane);
+        plasticity_rule_step(p.st, L, m, p.M, p.rule_flags, p.rule_serial, loss, p.lr, p.out_slopes, p.out_mask, lane);
 }
 
 struct FinParams {

@@ -73,6 +73,13 @@ struct TcParams {
     FinCounters *ctr_next;     // [M] the set the next launch will use: cleared here
     CtaLog *log;               // [gridDim.x] what each CTA reports about this launch, or nullptr
     uint32_t serial;           // tag of this launch in the log
+    // Test hook for the give-up path (0 in every ordinary launch).  1: the TMA producer of CTA 0
+    // issues no load at all, so its MMA warp's wait for the first stage runs out.  2: the MMA warp of
+    // CTA 0 stops after its first stage, so no accumulator is ever complete and (given more blocks
+    // than pipeline stages) the producer runs out of free stages with loads in flight behind it.
+    // Either way the waits run out, the CTA leaves through the give-up path and the kernel returns.
+    uint32_t test_stall;
+    uint64_t wait_limit_ns;    // limit of every bounded wait of this launch (kWaitLimitNs, shorter for the hook)
     int32_t M;
     FinCommon fin;             // slots, sides, b, outputs, freezing-rule state
 };
@@ -303,7 +310,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             uint32_t issued = 0;
             bool ok = true;
             int last_module = -1;
-            for (int ui = u_begin; ui < u_end && ok; ++ui) {
+            const int u_stop = (p.test_stall == 1 && blockIdx.x == 0) ? u_begin : u_end;  // test hook: no loads
+            for (int ui = u_begin; ui < u_stop && ok; ++ui) {
                 const Unit u = p.units[ui];
                 const CUtensorMap *tm_t = p.tmaps + 2 * u.module;
                 const CUtensorMap *tm_r = tm_t + 1;
@@ -315,7 +323,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 const CUtensorMap *tm_side = (u.side == 1) ? tm_r : tm_t;
                 const int kb_end = u.kb0 + u.nkb;
                 for (int kb = u.kb0; kb < kb_end; kb += Cfg::kKbPerStage) {
-                    if (!ptx::mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u, abort_flag, kWaitLimitNs)) {
+                    if (!ptx::mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u, abort_flag, p.wait_limit_ns)) {
                         ok = false;
                         break;
                     }
@@ -350,7 +358,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                     const uint32_t s = idx % Cfg::kStages, ph = (idx / Cfg::kStages) & 1u;
                     const uint64_t t0 = ptx::globaltimer_ns();
                     while (!ptx::mbar_try_wait(full0 + 8 * s, ph))
-                        if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) break;
+                        if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) break;
                 }
             }
         }
@@ -366,20 +374,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
             bool any_mma = false;
+            const bool stall_after_first_stage = (p.test_stall == 2 && blockIdx.x == 0);  // test hook
             for (int ui = u_begin; ui < u_end && ok; ++ui) {
                 const Unit u = p.units[ui];
-                if (!ptx::mbar_wait_bounded(accempty0 + 8 * acc, acc_phase ^ 1u, abort_flag, kWaitLimitNs)) {
+                if (!ptx::mbar_wait_bounded(accempty0 + 8 * acc, acc_phase ^ 1u, abort_flag, p.wait_limit_ns)) {
                     ok = false;
                     break;
                 }
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * Cfg::kAccCols;
                 for (int kb = 0; kb < u.nkb; kb += Cfg::kKbPerStage) {
-                    if (!ptx::mbar_wait_bounded(full0 + 8 * stage, phase, abort_flag, kWaitLimitNs)) {
+                    if (!ptx::mbar_wait_bounded(full0 + 8 * stage, phase, abort_flag, p.wait_limit_ns)) {
                         ok = false;
                         break;
                     }
                     ptx::tc_fence_after_sync();
+                    if (stall_after_first_stage && any_mma) {  // stop here: no further stage is released
+                        ok = false;
+                        break;
+                    }
                     const int nk = (u.nkb - kb < Cfg::kKbPerStage) ? u.nkb - kb : Cfg::kKbPerStage;
 #pragma unroll
                     for (int j = 0; j < Cfg::kKbPerStage; ++j) {
@@ -447,7 +460,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         bool aborted = false;
         for (int ui = u_begin; ui < u_end; ++ui) {
             const Unit u = p.units[ui];
-            const bool got = ptx::mbar_wait_bounded(accfull0 + 8 * acc, acc_phase, abort_flag, kWaitLimitNs);
+            const bool got = ptx::mbar_wait_bounded(accfull0 + 8 * acc, acc_phase, abort_flag, p.wait_limit_ns);
             if (!detail::epi_bar_and(got)) {  // the epilogue warps leave together
                 aborted = true;
                 break;

@@ -2,8 +2,9 @@
 // of the raw plasticity readings, least-squares slope of the last W smoothed values,
 // tolerance test, consecutive-stale counter; and the policies the paper states around it:
 // the per-module automatic tolerance (Sec. 4.2.2 "Hyperparameters guideline"), the
-// frontmost-active policy (Sec. 4.2.2; Algorithm 1 "l <- l + 1") and the end of the
-// bootstrapping stage (Sec. 3).  One warp per module, float64 throughout.
+// frontmost-active policy (Sec. 4.2.2; Algorithm 1 "l <- l + 1"), the learning-rate-based
+// unfreezing with the halved window (Sec. 4.2.2 "Unfreezing"; Algorithm 1, second half) and the
+// end of the bootstrapping stage (Sec. 3).  One warp per module, float64 throughout.
 #pragma once
 #include <cuda_runtime.h>
 #include <math.h>
@@ -29,8 +30,23 @@ struct SlopeState {     // per-module arrays (device)
     unsigned long long *front;  // [1] frontmost policy: (serial of the evaluation that last moved the front) << 32
                                 //     | number of frozen modules; one 8-byte word, read and written whole
     const float *T;     // [M] tolerance given at creation
-    int32_t W_cap;      // window pitch
+    int32_t W_cap;      // window pitch (the W given at creation)
+    // Unfreezing on learning-rate annealing: the window in force lives on the device, because the
+    // device halves it when it restarts the modules.
+    int32_t *W_cur;     // [1] window in force (<= W_cap)
+    unsigned long long *lr_ref;  // [1] bits of the learning rate (double) at the first freeze since the start
+                                 //     or the last restart; kLrUnset while nothing has frozen
+    int32_t *restarts;  // [1] restarts so far
 };
+
+constexpr unsigned long long kLrUnset = 0x7ff8000000000000ull;  // a quiet NaN: "no reference rate"
+
+// W <- max(2, floor(W / 2)): a line needs two points (W = 1 stays 1).
+__host__ __device__ inline int halve_window(int W) {
+    if (W < 2) return W;
+    const int h = W / 2;
+    return h < 2 ? 2 : h;
+}
 
 __device__ __forceinline__ double warp_sum_f64(double v) {
 #pragma unroll
@@ -140,22 +156,25 @@ struct StepLoaded {
     double ra[kStepRegs], rb[kStepRegs], pa[kStepRegs], pb[kStepRegs];
     double slope, T, Tauto, smax;
     int i, counter, freeze_eval;
+    int W;  // window in force
 };
 
 // Issue every load of one step of module m (nothing here depends on the new reading).
-__device__ __forceinline__ StepLoaded plasticity_step_load(const SlopeState &st, int m, int W, int lane) {
+__device__ __forceinline__ StepLoaded plasticity_step_load(const SlopeState &st, int m, int lane) {
     StepLoaded L;
     const double *raw = st.raw + (int64_t)m * st.W_cap, *plist = st.plist + (int64_t)m * st.W_cap;
-    if (W <= 32 * kStepRegs) {
+    const int Wc = st.W_cap;  // the window in force is at most this; what lies beyond it is never used
+    if (Wc <= 32 * kStepRegs) {
 #pragma unroll
         for (int j = 0; j < kStepRegs; ++j) {
             const int k = lane + 32 * j;
-            L.ra[j] = (k < W) ? raw[k] : 0.0;
-            L.pa[j] = (k < W) ? plist[k] : 0.0;
-            L.rb[j] = (k + 1 < W) ? raw[k + 1] : 0.0;
-            L.pb[j] = (k + 1 < W) ? plist[k + 1] : 0.0;
+            L.ra[j] = (k < Wc) ? raw[k] : 0.0;
+            L.pa[j] = (k < Wc) ? plist[k] : 0.0;
+            L.rb[j] = (k + 1 < Wc) ? raw[k + 1] : 0.0;
+            L.pb[j] = (k + 1 < Wc) ? plist[k + 1] : 0.0;
         }
     }
+    L.W = *st.W_cur;
     L.i = st.n_evals[m];  // readings taken before this one == index of this evaluation
     L.counter = st.counter[m];
     L.freeze_eval = st.freeze_eval[m];
@@ -168,11 +187,14 @@ __device__ __forceinline__ StepLoaded plasticity_step_load(const SlopeState &st,
 
 // One new reading for module m, by one warp: Algorithm 1 on the context's state.  Returns
 // whether the module is converged after this evaluation; `slope_out` is the slope of this
-// evaluation (the last one if the module had converged before).
-__device__ __forceinline__ bool plasticity_step_apply(const SlopeState &st, StepLoaded &L, int m, int W, int flags,
-                                                      float reading, int lane, double &slope_out) {
+// evaluation (the last one if the module had converged before).  `lr` is the learning rate in
+// force (not positive or NaN: unknown): the first module to freeze records it as the reference
+// rate of the unfreezing rule.
+__device__ __forceinline__ bool plasticity_step_apply(const SlopeState &st, StepLoaded &L, int m, int flags,
+                                                      float reading, double lr, int lane, double &slope_out) {
     double *raw = st.raw + (int64_t)m * st.W_cap, *plist = st.plist + (int64_t)m * st.W_cap;
-    const bool fast = (W <= 32 * kStepRegs);
+    const int W = L.W;
+    const bool fast = (st.W_cap <= 32 * kStepRegs);
     double(&ra)[kStepRegs] = L.ra, (&rb)[kStepRegs] = L.rb, (&pa)[kStepRegs] = L.pa, (&pb)[kStepRegs] = L.pb;
     const int i = L.i;
     int counter = L.counter, freeze_eval = L.freeze_eval;
@@ -214,7 +236,11 @@ __device__ __forceinline__ bool plasticity_step_apply(const SlopeState &st, Step
         }
         const bool stale = rule_is_stale(slope, i, flags, L.T, L.Tauto, L.smax);
         counter = stale ? counter + 1 : 0;
-        if (counter >= W && freeze_eval < 0) freeze_eval = i;
+        if (counter >= W && freeze_eval < 0) {
+            freeze_eval = i;
+            // every freeze of one evaluation carries the same rate, so who wins does not matter
+            if (lane == 0 && lr > 0.0) atomicCAS(st.lr_ref, kLrUnset, (unsigned long long)__double_as_longlong(lr));
+        }
         if (lane == 0) {
             st.n_evals[m] = i + 1;
             st.counter[m] = counter;
@@ -238,12 +264,12 @@ __device__ __forceinline__ bool plasticity_step_apply(const SlopeState &st, Step
 // frozen one, +inf for one that has not been monitored yet.  `serial` numbers the evaluations
 // (from 1): a front that moved during evaluation `serial` is left alone for the rest of it,
 // so the module that becomes the front starts with the next evaluation.
-__device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepLoaded &L, int m, int M, int W,
-                                                     int flags, uint32_t serial, float reading, double *out_slopes,
+__device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepLoaded &L, int m, int M, int flags,
+                                                     uint32_t serial, float reading, double lr, double *out_slopes,
                                                      uint8_t *out_mask, int lane) {
     if (!(flags & kRuleFrontmost)) {
         double slope;
-        const bool conv = plasticity_step_apply(st, L, m, W, flags, reading, lane, slope);
+        const bool conv = plasticity_step_apply(st, L, m, flags, reading, lr, lane, slope);
         if (lane == 0) {
             if (out_slopes) out_slopes[m] = slope;
             if (out_mask) out_mask[m] = conv ? 1 : 0;
@@ -258,7 +284,7 @@ __device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepL
     int front_new = front;
     double slope = INFINITY;
     if (front < M) {
-        const bool conv = plasticity_step_apply(st, L, m, W, flags, reading, lane, slope);
+        const bool conv = plasticity_step_apply(st, L, m, flags, reading, lr, lane, slope);
         if (conv) front_new = front + 1;
     }
     if (lane == 0 && front_new != front)
@@ -271,24 +297,59 @@ __device__ __forceinline__ void plasticity_rule_step(const SlopeState &st, StepL
 }
 
 // One new reading per module.  grid = M warps (one 32-thread block each).
-__global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int M, int W, int flags, uint32_t serial,
-                                                             const float *losses, double *out_slopes,
+__global__ void __launch_bounds__(32) plasticity_step_kernel(SlopeState st, int M, int flags, uint32_t serial,
+                                                             double lr, const float *losses, double *out_slopes,
                                                              uint8_t *out_mask) {
     const int m = blockIdx.x, lane = threadIdx.x;
     if (m >= M) return;
-    StepLoaded L = plasticity_step_load(st, m, W, lane);
-    plasticity_rule_step(st, L, m, M, W, flags, serial, losses[m], out_slopes, out_mask, lane);
+    StepLoaded L = plasticity_step_load(st, m, lane);
+    plasticity_rule_step(st, L, m, M, flags, serial, losses[m], lr, out_slopes, out_mask, lane);
+}
+
+// The unfreezing test of Algorithm 1 [Sec. 4.2.2 "Unfreezing"], run after the evaluation whose
+// learning rate `lr` differs from the previous one's (the test cannot change its mind while the
+// rate stands still).  If the rate has fallen to a tenth, or less, of the rate at the first freeze
+// (one part in a million of slack, so that a step decay by exactly 10x counts even when it was
+// computed in single precision): every module starts afresh, the front goes back to module 0,
+// the window is halved and the reference rate is forgotten; the mask of the evaluation that
+// just ran is cleared.  One block.
+__global__ void unfreeze_check_kernel(SlopeState st, int M, double lr, uint8_t *out_mask) {
+    __shared__ int fire;
+    if (threadIdx.x == 0) {
+        const unsigned long long bits = *st.lr_ref;
+        const double ref = __longlong_as_double((long long)bits);
+        fire = (bits != kLrUnset && lr > 0.0 && lr <= ref / 10.0 * (1.0 + 1e-6)) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!fire) return;
+    for (int m = threadIdx.x; m < M; m += blockDim.x) {
+        st.n_evals[m] = 0;
+        st.counter[m] = 0;
+        st.freeze_eval[m] = -1;
+        st.last_slope[m] = INFINITY;
+        st.Tauto[m] = NAN;
+        st.smax[m] = 0.0;
+        if (out_mask) out_mask[m] = 0;
+    }
+    if (threadIdx.x == 0) {
+        *st.front = 0ull;
+        *st.lr_ref = kLrUnset;
+        *st.W_cur = halve_window(*st.W_cur);
+        *st.restarts += 1;
+    }
 }
 
 // Whole histories from a cleared private state (windows in shared memory: 2 * W doubles).
 // Without the frontmost policy: one warp per module (grid = M).  With it: one warp in all
 // (grid = 1) walks the modules front to back.  out_slopes[m][i] is NaN where module m was
 // not advanced at evaluation i.
-__global__ void __launch_bounds__(32) plasticity_replay_kernel(const float *T, int M, int W, int flags,
-                                                               const float *hist, int H, double *out_slopes,
-                                                               uint8_t *out_mask, int32_t *out_freeze_eval) {
+__global__ void __launch_bounds__(32) plasticity_replay_kernel(const float *T, int M, const int32_t *W_cur, int W_cap,
+                                                               int flags, const float *hist, int H,
+                                                               double *out_slopes, uint8_t *out_mask,
+                                                               int32_t *out_freeze_eval) {
     extern __shared__ double windows[];
-    double *raw = windows, *plist = windows + W;
+    const int W = *W_cur;  // the window in force (<= W_cap, which sizes the shared memory)
+    double *raw = windows, *plist = windows + W_cap;
     const int lane = threadIdx.x;
     const bool frontmost = (flags & kRuleFrontmost) != 0;
     int m = frontmost ? 0 : (int)blockIdx.x;
@@ -334,9 +395,113 @@ __global__ void __launch_bounds__(32) plasticity_replay_kernel(const float *T, i
     }
 }
 
-__global__ void plasticity_clear_kernel(SlopeState st, int M) {
+// Whole histories with the learning-rate-based unfreezing [Sec. 4.2.2 "Unfreezing"; Algorithm 1,
+// second half], from a cleared state private to the call.  A restart couples the modules (any
+// freeze arms it, every module is cleared by it), so one block runs all of them: warp w takes
+// modules w, w + warps, ...; after every evaluation thread 0 moves the front, remembers the rate
+// of the first freeze and takes the unfreezing decision for everybody.  The windows are in global
+// scratch ([M][W_cap] each), the per-module scalars in shared memory (M * sizeof(ReplayModule)).
+struct ReplayModule {
+    int32_t len, n_evals, counter, frozen;
+    double Tauto, smax;
+};
+
+__global__ void __launch_bounds__(1024) plasticity_replay_lr_kernel(
+    const float *T, double *raw_all, double *plist_all, int W_cap, const int32_t *W_start, int M, int flags,
+    const float *hist, const double *lr, int H, double *out_slopes, uint8_t *out_frozen, int32_t *out_window,
+    uint8_t *out_restarted, uint8_t *out_mask, int32_t *out_freeze_eval) {
+    extern __shared__ double replay_smem[];
+    ReplayModule *mod = reinterpret_cast<ReplayModule *>(replay_smem);
+    __shared__ int s_W, s_front, s_froze_now, s_fire;
+    __shared__ unsigned long long s_lr_ref;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const bool frontmost = (flags & kRuleFrontmost) != 0;
+    for (int m = threadIdx.x; m < M; m += blockDim.x) {
+        mod[m] = ReplayModule{0, 0, 0, 0, NAN, 0.0};
+        if (out_freeze_eval) out_freeze_eval[m] = -1;
+    }
+    if (threadIdx.x == 0) {
+        s_W = *W_start;
+        s_front = 0;
+        s_lr_ref = kLrUnset;
+    }
+    __syncthreads();
+    for (int i = 0; i < H; ++i) {
+        if (threadIdx.x == 0) {
+            s_froze_now = 0;
+            s_fire = 0;
+            if (out_window) out_window[i] = s_W;
+        }
+        __syncthreads();
+        const int W = s_W, front = s_front;
+        for (int m = warp; m < M; m += n_warps) {
+            ReplayModule &st = mod[m];
+            double slope = NAN;
+            if (!st.frozen && (!frontmost || m == front)) {
+                double pbar;
+                st.len = window_push(raw_all + (int64_t)m * W_cap, plist_all + (int64_t)m * W_cap, st.len, W,
+                                     (double)hist[(int64_t)m * H + i], lane, pbar, slope);
+                double Tauto = st.Tauto, smax = st.smax;
+                const bool stale = rule_is_stale(slope, st.n_evals, flags, (double)T[m], Tauto, smax);
+                __syncwarp();
+                if (lane == 0) {
+                    st.Tauto = Tauto;
+                    st.smax = smax;
+                    st.counter = stale ? st.counter + 1 : 0;
+                    st.n_evals += 1;
+                    if (st.counter >= W) {
+                        st.frozen = 1;
+                        s_froze_now = 1;
+                        if (out_freeze_eval) out_freeze_eval[m] = i;
+                    }
+                }
+                __syncwarp();
+            }
+            if (out_slopes && lane == 0) out_slopes[(int64_t)m * H + i] = slope;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            if (frontmost && s_front < M && mod[s_front].frozen) s_front += 1;  // freezeLayer(l); l <- l + 1
+            const double rate = lr ? lr[i] : NAN;
+            if (s_froze_now && s_lr_ref == kLrUnset && rate > 0.0)
+                s_lr_ref = (unsigned long long)__double_as_longlong(rate);
+            const double ref = __longlong_as_double((long long)s_lr_ref);
+            if (s_lr_ref != kLrUnset && rate > 0.0 && rate <= ref / 10.0 * (1.0 + 1e-6)) {
+                s_fire = 1;
+                s_front = 0;
+                s_W = halve_window(s_W);
+                s_lr_ref = kLrUnset;
+            }
+            if (out_restarted) out_restarted[i] = (uint8_t)s_fire;
+        }
+        __syncthreads();
+        for (int m = threadIdx.x; m < M; m += blockDim.x) {
+            if (s_fire) {
+                mod[m] = ReplayModule{0, 0, 0, 0, NAN, 0.0};
+                if (out_freeze_eval) out_freeze_eval[m] = -1;
+            }
+            if (out_frozen) out_frozen[(int64_t)i * M + m] = (uint8_t)mod[m].frozen;
+        }
+        __syncthreads();
+    }
+    for (int m = threadIdx.x; m < M; m += blockDim.x)
+        if (out_mask) out_mask[m] = (uint8_t)mod[m].frozen;
+}
+
+// Clear the rule state of every module.  set_W > 0: the window in force becomes set_W (context
+// creation); else, if halve != 0, it is halved.
+__global__ void plasticity_clear_kernel(SlopeState st, int M, int set_W, int halve) {
     const int m = blockIdx.x * blockDim.x + threadIdx.x;
-    if (m == 0) *st.front = 0ull;
+    if (m == 0) {
+        *st.front = 0ull;
+        *st.lr_ref = kLrUnset;
+        if (set_W > 0) {
+            *st.W_cur = set_W;
+            *st.restarts = 0;
+        } else if (halve) {
+            *st.W_cur = halve_window(*st.W_cur);
+        }
+    }
     if (m >= M) return;
     st.n_evals[m] = 0;
     st.counter[m] = 0;

@@ -150,19 +150,21 @@ def tiny_history_sigmas(w: Workload) -> List[float]:
     return [0.5 + (0.01 - 0.5) * k / (w.H - 1) for k in range(w.H)]
 
 
-def make_history(w: Workload, levels: Sequence[float], H: Optional[int] = None) -> np.ndarray:
+def make_history(w: Workload, levels: Sequence[float], H: Optional[int] = None,
+                 tau_scale: float = 1.0) -> np.ndarray:
     """Synthetic raw-loss histories, float32 [M, H].
 
     Module l decays towards its level L_l: h_l[k] = L_l * (1 + 4*exp(-k/tau_l)) (+ noise),
-    tau_l = H * (0.05 + 0.5*l/(M-1)), so front modules flatten inside the history
-    and deep ones do not.  Noise (if any) is N(0, hist_noise), seeded."""
+    tau_l = tau_scale * H * (0.05 + 0.5*l/(M-1)), so front modules flatten inside the history
+    and deep ones do not (a small tau_scale makes every module flatten quickly).  Noise (if
+    any) is N(0, hist_noise), seeded."""
     H = w.H if H is None else H
     M = len(levels)
     k = np.arange(H, dtype=np.float64)
     out = np.empty((M, H), dtype=np.float64)
     rng = np.random.Generator(np.random.PCG64(SEED_BASE + 1000 * w.index + 999))
     for l in range(M):
-        tau = H * (0.05 + 0.5 * (l / (M - 1) if M > 1 else 0.0))
+        tau = tau_scale * H * (0.05 + 0.5 * (l / (M - 1) if M > 1 else 0.0))
         out[l] = float(levels[l]) * (1.0 + 4.0 * np.exp(-k / tau))
         if w.hist_noise > 0.0:
             out[l] += rng.normal(0.0, w.hist_noise, size=H)

@@ -234,11 +234,13 @@ def test_bert_base_workload_full():
 def _sampled_check(name, full_modules, row_modules, rows):
     """Full-size workload in the benchmark's launch configuration -- the call bench.py times
     (egeria_plasticity_evaluate), first with the equal split and again once the adaptive split
-    has settled; the oracle checks the whole loss of a few modules and sampled rows of the
-    normalised Grams of others."""
+    has settled.  The oracle gives the loss of EVERY module; every entry of the normalised Grams
+    of a few modules and sampled rows of others are compared as well."""
     w = wl.WORKLOADS[name]
     at, ar = wl.make_activations(w, DEV)
     full_ref = {m: oracle.sp_loss(wl.bf16_bits(at[m]), wl.bf16_bits(ar[m]), return_grams=True) for m in full_modules}
+    loss_ref = np.array([full_ref[m][0] if m in full_ref else oracle.sp_loss(wl.bf16_bits(at[m]), wl.bf16_bits(ar[m]))
+                         for m in range(w.M)])
     row_ref = {}
     for m in row_modules:
         for side, acts in enumerate((at, ar)):
@@ -252,11 +254,10 @@ def _sampled_check(name, full_modules, row_modules, rows):
         losses = ctx.egeria_plasticity_evaluate(at, ar)[0].cpu().numpy()
         grams = [tuple(g.cpu().numpy() for g in ctx.egeria_debug_dump_gram(m, w.b)) for m in range(w.M)]
         ctx.check_device_status()
-        assert np.isfinite(losses).all() and np.all(losses >= 0) and np.all(losses <= 4.0 / w.b)
+        assert_loss_close(losses, loss_ref, f"{name}, all {w.M} modules ({what})")
         for m, (ref, gt, gr) in full_ref.items():
             np.testing.assert_allclose(grams[m][0], gt, rtol=0, atol=ENTRY_ATOL)
             np.testing.assert_allclose(grams[m][1], gr, rtol=0, atol=ENTRY_ATOL)
-            assert_loss_close(losses[m:m + 1], [ref], f"{name} module {m} ({what})")
         for (m, side, i), gn in row_ref.items():
             np.testing.assert_allclose(grams[m][side][i], gn, rtol=0, atol=ENTRY_ATOL)
         # properties that hold at any size: unit rows, symmetric-positive diagonal
@@ -319,6 +320,114 @@ def test_call_error_paths():
     ctx.close()
 
 
+def test_raw_abi_argument_errors_leave_the_context_usable():
+    """Requirements checked on the host and reported as status codes, through the raw C ABI (the
+    binding would not let these through): a d[] that differs from creation, a NULL module
+    pointer, an odd pointer, a NULL output, NULL arrays -- each EGERIA_ERR_INVALID_ARG, nothing
+    launched, and the same context evaluates correctly afterwards."""
+    import ctypes
+    L = eg.lib()
+    ds, b = [4096, 520], 24
+    at, ar = [], []
+    for m, d in enumerate(ds):
+        t, r = wl.make_pair(b, d, "normal", 0.2, seed=70 + m, device=DEV)
+        at.append(t)
+        ar.append(r)
+    ctx = eg.Context(ds, b, 5, 1e-3, device=DEV)
+    out = torch.full((2,), -3.0, dtype=torch.float32, device=DEV)
+    sp = int(torch.cuda.current_stream().cuda_stream)
+    good_t, good_r = ctx._ptr_array(at, b, True), ctx._ptr_array(ar, b, True)
+    d_ok = (ctypes.c_int64 * 2)(*ds)
+    launched = ctx.egeria_launch_count()
+
+    def call(pt, pr, d_arr, out_ptr, bb=b):
+        return L.egeria_sp_loss_batch(ctx._h, sp, pt, pr, bb, d_arr, out_ptr)
+
+    def ptrs(a, c):
+        arr = (ctypes.c_void_p * 2)()
+        arr[0], arr[1] = a, c
+        return arr
+
+    assert call(good_t, good_r, (ctypes.c_int64 * 2)(4096, 528), out.data_ptr()) == eg.ERR_INVALID_ARG   # d[] mismatch
+    assert call(ptrs(at[0].data_ptr(), None), good_r, d_ok, out.data_ptr()) == eg.ERR_INVALID_ARG        # NULL module
+    assert call(good_t, ptrs(ar[0].data_ptr(), ar[1].data_ptr() + 1), d_ok, out.data_ptr()) == eg.ERR_INVALID_ARG  # odd
+    assert call(good_t, good_r, d_ok, None) == eg.ERR_INVALID_ARG                                        # no output
+    assert call(None, good_r, d_ok, out.data_ptr()) == eg.ERR_INVALID_ARG
+    assert call(good_t, good_r, None, out.data_ptr()) == eg.ERR_INVALID_ARG
+    assert call(good_t, good_r, d_ok, out.data_ptr(), bb=1) == eg.ERR_INVALID_ARG                        # b < 2
+    assert L.egeria_sp_loss_batch(None, sp, good_t, good_r, b, d_ok, out.data_ptr()) == eg.ERR_INVALID_ARG
+    assert L.egeria_plasticity_step(ctx._h, sp, None, None, None) == eg.ERR_INVALID_ARG
+    assert L.egeria_plasticity_set_lr(None, ctypes.c_double(0.1)) == eg.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert ctx.egeria_launch_count() == launched and np.all(out.cpu().numpy() == -3.0)   # nothing ran
+    assert call(good_t, good_r, d_ok, out.data_ptr()) == eg.OK
+    ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+    assert_loss_close(out.cpu().numpy(), ref)
+    ctx.check_device_status()
+    ctx.close()
+
+
+def test_many_pointer_sets_enqueued_ahead_of_the_gpu():
+    """A caller whose activation buffers are new on every call misses the plan cache every time.
+    With the GPU held busy, far more than the 16 cached plans are enqueued before any of them has
+    run: every evaluation must still see its own tensor maps and work split."""
+    ds, b, n = [2048, 520, 4096], 40, 48
+    sets, refs = [], []
+    for k in range(n):
+        at, ar = [], []
+        for m, d in enumerate(ds):
+            t, r = wl.make_pair(b, d, "relu", 0.05 + 0.01 * k, seed=3000 + 10 * k + m, device=DEV)
+            at.append(t)
+            ar.append(r)
+        sets.append((at, ar))
+    for k in (0, 17, 33, n - 1):
+        refs.append((k, oracle.sp_loss_batch([wl.bf16_bits(t) for t in sets[k][0]],
+                                             [wl.bf16_bits(r) for r in sets[k][1]])))
+    ctx = eg.Context(ds, b, 5, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
+    one = eg.Context(ds, b, 5, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
+    want = [one.egeria_sp_loss_batch(at, ar).cpu().numpy().copy() for at, ar in sets]   # one at a time
+    outs = [torch.empty(len(ds), dtype=torch.float32, device=DEV) for _ in range(n)]
+    big = torch.randn(8192, 8192, device=DEV)
+    torch.cuda.synchronize()
+    for _ in range(40):                       # some tens of milliseconds of work ahead of the evaluations
+        big = torch.mm(big, big).clamp_(-1, 1)
+    for k, (at, ar) in enumerate(sets):
+        ctx.egeria_sp_loss_batch(at, ar, outs[k])
+    torch.cuda.synchronize()
+    ctx.check_device_status()
+    for k in range(n):
+        assert outs[k].cpu().numpy().tobytes() == want[k].tobytes(), f"evaluation {k}"
+    for k, ref in refs:
+        assert_loss_close(outs[k].cpu().numpy(), ref, f"evaluation {k}")
+    ctx.close()
+    one.close()
+
+
+@pytest.mark.parametrize("kind", [1, 2])
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_recovers(kind):
+    """The give-up path of the evaluation kernel, in the form that returns: one hand-shake of the
+    first thread block is left out for ONE launch whose waits are limited to a millisecond.  The
+    kernel returns, the status word says EGERIA_ERR_TIMEOUT (once), and the next evaluation on
+    the same context matches the oracle."""
+    b, d = 64, 64 * 148 * 40                       # 40 blocks per thread block: more than the 12 pipeline stages
+    at, ar = wl.make_pair(b, d, "relu", 0.2, seed=4242, device=DEV)
+    ref = oracle.sp_loss(wl.bf16_bits(at), wl.bf16_bits(ar))
+    ctx = eg.Context([d], b, 5, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
+    good = ctx.egeria_sp_loss_batch([at], [ar]).cpu().numpy().copy()
+    assert_loss_close(good, [ref])
+    out = torch.full((1,), -5.0, dtype=torch.float32, device=DEV)
+    ctx.egeria_debug_stall_next(kind)
+    ctx.egeria_sp_loss_batch([at], [ar], out)
+    assert ctx.egeria_device_status() == eg.ERR_TIMEOUT
+    assert float(out.cpu()[0]) == -5.0             # no loss was written by the launch that gave up
+    assert ctx.egeria_device_status() == eg.OK     # reported once; the counters start afresh
+    for _ in range(3):                             # both sets of progress counters come round
+        again = ctx.egeria_sp_loss_batch([at], [ar]).cpu().numpy()
+        assert again.tobytes() == good.tobytes()
+    ctx.check_device_status()
+    ctx.close()
+
+
 def test_changing_b_and_pointers_between_calls():
     ctx = eg.Context([4096, 264], 128, 5, 1e-3, device=DEV)
     for b in (128, 8, 70, 8):
@@ -336,37 +445,73 @@ def test_changing_b_and_pointers_between_calls():
 
 # ----------------------------------------------------------------------------- freezing rule
 
+def first_freeze(stale, W):
+    """Evaluation at which W consecutive stale evaluations are first complete, -1 if never."""
+    run = 0
+    for i, st in enumerate(stale):
+        run = run + 1 if st else 0
+        if run >= W:
+            return i
+    return -1
+
+
 def masks_agree(gpu_mask, gpu_fe, hist, W, T, signed=False):
+    """Freeze decisions of a whole-history replay against the oracle's.  The stated criterion
+    exempts a decision where the oracle's |slope| is within 1e-6 of T; it is applied per
+    evaluation: an evaluation that close to T may be counted either way.  Where every such
+    choice gives the same freeze evaluation, the GPU must give exactly the oracle's; elsewhere it
+    must lie between the earliest and the latest possible one.  Returns (modules compared
+    exactly, of which converged, modules the oracle converged)."""
+    exact = exact_conv = n_conv = 0
     for m in range(hist.shape[0]):
         ref = oracle.plasticity_replay(hist[m], W, T, signed_test=signed)
-        s = ref["slopes"][np.isfinite(ref["slopes"])]
-        near = np.any(np.abs((s if signed else np.abs(s)) - T) <= 1e-6) if len(s) else False
-        if near:
-            continue
-        assert bool(gpu_mask[m]) == ref["converged"], f"module {m}"
-        assert int(gpu_fe[m]) == ref["freeze_eval"], f"module {m}"
+        n_conv += ref["converged"]
+        # the slopes of all evaluations, also past the oracle's freeze (T = 0: nothing is ever stale)
+        s = oracle.plasticity_replay(hist[m], W, 0.0, signed_test=False)["slopes"]
+        v = s if signed else np.abs(s)
+        usable = np.isfinite(v)
+        near = usable & (np.abs(v - T) <= 1e-6)
+        sure = usable & (v < T) & ~near
+        lo, hi = first_freeze(sure | near, W), first_freeze(sure, W)
+        fe, conv = int(gpu_fe[m]), bool(gpu_mask[m])
+        assert conv == (fe >= 0)
+        if lo == hi:
+            assert ref["freeze_eval"] == lo                      # the oracle's own decision
+            assert fe == lo and conv == ref["converged"], f"module {m}: gpu {fe}, oracle {lo}"
+            exact += 1
+            exact_conv += ref["converged"]
+        else:
+            assert lo >= 0 and (fe >= lo if hi < 0 else lo <= fe <= hi), f"module {m}: gpu {fe} outside [{lo}, {hi}]"
+    return exact, exact_conv, n_conv
 
 
-@pytest.mark.parametrize("name,level", [("resnet56", None), ("resnet56", 1e-2), ("resnet50", 2e-2),
-                                        ("bert_base", 5e-3), ("gpt2_medium", 3e-2)])
-def test_replay_matches_oracle(name, level):
+@pytest.mark.parametrize("name,level,tau_scale", [("resnet56", None, 1.0), ("resnet56", 1e-2, 1.0),
+                                                  ("resnet50", 2e-2, 1.0), ("bert_base", 5e-3, 1.0),
+                                                  ("gpt2_medium", 3e-2, 1.0), ("gpt2_medium", 3e-2, 0.04),
+                                                  ("resnet50", 2e-2, 0.2)])
+def test_replay_matches_oracle(name, level, tau_scale):
+    """The workload's window and tolerance on synthetic histories.  tau_scale < 1 makes the slope
+    cross T quickly (by more than 1e-6 per evaluation), so that the freeze evaluation of most
+    modules does not hinge on an evaluation within 1e-6 of T and is compared exactly."""
     w = wl.WORKLOADS[name]
     levels = [1e-6 * (1 + l) for l in range(w.M)] if level is None else [level * (1 + 0.1 * l) for l in range(w.M)]
-    hist = wl.make_history(w, levels)
+    hist = wl.make_history(w, levels, tau_scale=tau_scale)
     T32 = np.float32(w.T)
     ctx = eg.Context([64] * w.M, 8, w.W, float(T32), device=DEV)
     slopes, mask, fe = ctx.egeria_plasticity_replay(torch.from_numpy(hist).to(DEV))
     slopes, mask, fe = slopes.cpu().numpy(), mask.cpu().numpy(), fe.cpu().numpy()
-    n_conv = 0
     for m in range(w.M):
         ref = oracle.plasticity_replay(hist[m], w.W, float(T32))
         live = ~np.isnan(ref["slopes"])
         assert np.array_equal(np.isnan(slopes[m]), ~live) or not ref["converged"]
         np.testing.assert_allclose(slopes[m][live], ref["slopes"][live], rtol=1e-9, atol=1e-15)
-        n_conv += ref["converged"]
-    masks_agree(mask, fe, hist, w.W, float(T32))
+    exact, exact_conv, n_conv = masks_agree(mask, fe, hist, w.W, float(T32))
+    print(f"{name} tau_scale={tau_scale}: freeze decisions compared exactly for {exact}/{w.M} modules, "
+          f"{exact_conv}/{n_conv} of the converged ones")
     if level is not None and name != "bert_base":
-        assert 0 < n_conv < w.M, "the synthetic history should give a non-trivial mask"
+        assert 0 < n_conv, "the synthetic history should freeze some modules"
+    if tau_scale < 1.0:
+        assert n_conv >= w.M // 2 and 3 * exact_conv >= n_conv, "the mask comparison must not be empty"
     ctx.close()
 
 
@@ -394,11 +539,31 @@ def test_step_matches_replay_and_oracle(signed):
                 assert bool(step_mask[m, i]) == ref["converged"]
             if not ref["converged"]:
                 assert step_slopes[m, i] == pytest.approx(ref["slopes"][i], rel=1e-9, abs=1e-15)
-    # reset clears the state; halving the window follows the unfreezing rule
+    # a reset by hand with the window halved: what follows is the plain rule with W / 2, started
+    # afresh on the readings that follow
     ctx.egeria_plasticity_reset(halve_W=True)
     assert ctx.egeria_plasticity_window() == 2
-    s, mk = ctx.egeria_plasticity_step(hist_dev[:, 0].contiguous())
-    assert np.all(np.isinf(s.cpu().numpy())) and not mk.cpu().numpy().any()
+    tail = hist[:, ::-1].copy()                                 # rising readings this time
+    tail_dev = torch.from_numpy(tail).to(DEV)
+    for i in range(H):
+        s, mk = ctx.egeria_plasticity_step(tail_dev[:, i].contiguous())
+        step_slopes[:, i], step_mask[:, i] = s.cpu().numpy(), mk.cpu().numpy()
+    compared = 0
+    for m in range(M):
+        ref = oracle.plasticity_replay(tail[m], 2, float(T), signed_test=signed)
+        live = ~np.isnan(ref["slopes"])
+        fin = live & np.isfinite(ref["slopes"])
+        np.testing.assert_allclose(step_slopes[m][fin], ref["slopes"][fin], rtol=1e-9, atol=1e-15)
+        assert np.all(np.isinf(step_slopes[m][live & ~fin]))
+        sl = ref["slopes"][fin]
+        if np.any(np.abs((sl if signed else np.abs(sl)) - T) <= 1e-6):
+            continue
+        want = np.zeros(H, dtype=np.uint8)
+        if ref["converged"]:
+            want[ref["freeze_eval"]:] = 1
+        assert np.array_equal(step_mask[m], want)
+        compared += 1
+    assert compared >= M // 2
     ctx.close()
 
 
@@ -646,6 +811,167 @@ def test_frontmost_policy_evaluating_only_the_front_module():
     assert seen[-1] == M and seen[0] == 0
     full.close()
     front_only.close()
+
+
+# ----------------------------------------------------------------------------- unfreezing on learning-rate annealing
+
+def _unfreeze_case(seed, M, H, period):
+    """Histories that decay within each learning-rate period, and a step decay by 10x per period."""
+    rng = np.random.default_rng(seed)
+    k = np.arange(H)
+    hist = np.stack([0.3 * np.exp(-(k % period) / rng.uniform(2, 8)) + 0.01 * (m + 1) + 1e-4 * rng.standard_normal(H)
+                     for m in range(M)]).astype(np.float32)
+    T = rng.uniform(3e-3, 2e-2, size=M).astype(np.float32)
+    lr = 0.1 * np.power(0.1, k // period).astype(np.float64)
+    return hist, T, lr
+
+
+def _clear_of_T(ref, T, auto=False):
+    """No finite oracle slope within 1e-6 of its tolerance: every decision may be compared."""
+    if auto:
+        return True        # checked by the caller through the masks' agreement with the slopes
+    for m in range(ref["slopes"].shape[0]):
+        s = ref["slopes"][m]
+        s = s[np.isfinite(s)]
+        if np.any(np.abs(np.abs(s) - float(T[m])) <= 1e-6):
+            return False
+    return True
+
+
+@pytest.mark.parametrize("frontmost", [False, True])
+@pytest.mark.parametrize("auto", [False, True])
+def test_unfreeze_one_evaluation_at_a_time_matches_oracle(frontmost, auto):
+    """egeria_plasticity_set_lr + egeria_plasticity_step across two tenfold drops of the learning
+    rate: slopes, masks, the window in force and the restarts against oracle.unfreeze_replay."""
+    M, H, W, period = 4, 165, 6, 55
+    hist, T, lr = _unfreeze_case(21 + auto, M, H, period)
+    ref = oracle.unfreeze_replay(hist, lr, W, None if auto else T.astype(np.float64), frontmost=frontmost)
+    assert ref["restarts"] == 2 and _clear_of_T(ref, T, auto)
+    flags = (eg.FLAG_FRONTMOST if frontmost else 0) | (eg.FLAG_AUTO_T if auto else 0)
+    ctx = eg.Context([64] * M, 8, W, T, flags, device=DEV)
+    dev = torch.from_numpy(hist).to(DEV)
+    for i in range(H):
+        ctx.egeria_plasticity_set_lr(float(lr[i]))
+        s, mk = ctx.egeria_plasticity_step(dev[:, i].contiguous())
+        s, mk = s.cpu().numpy(), mk.cpu().numpy()
+        assert mk.tolist() == ref["frozen"][i].tolist(), f"evaluation {i}"
+        adv = ~np.isnan(ref["slopes"][:, i])
+        fin = adv & np.isfinite(ref["slopes"][:, i])
+        np.testing.assert_allclose(s[fin], ref["slopes"][fin, i], rtol=1e-9, atol=1e-15)
+        assert np.all(np.isinf(s[adv & ~fin]))
+        if i in (0, period - 1, period, period + 1, 2 * period + 3):
+            assert ctx.egeria_plasticity_window() == ref["window"][i + 1]   # what the NEXT evaluation will use
+    assert ctx.egeria_plasticity_restarts() == ref["restarts"]
+    ctx.close()
+
+
+@pytest.mark.parametrize("M,H,W,period,frontmost", [(4, 165, 6, 55, False), (4, 165, 6, 55, True),
+                                                    (24, 1000, 50, 334, False), (24, 1000, 50, 334, True),
+                                                    (70, 300, 9, 100, False)])
+def test_unfreeze_whole_histories_match_oracle(M, H, W, period, frontmost):
+    """egeria_plasticity_replay_lr: one launch over the whole history, against oracle.unfreeze_replay."""
+    hist, T, lr = _unfreeze_case(100 + M + W, M, H, period)
+    if W >= 50:                                                   # long windows: slower decays, so that modules still freeze
+        k = np.arange(H)
+        rng = np.random.default_rng(7)
+        hist = np.stack([0.3 * np.exp(-(k % period) / rng.uniform(5, 30)) + 0.01 * (m + 1)
+                         + 1e-5 * rng.standard_normal(H) for m in range(M)]).astype(np.float32)
+    ref = oracle.unfreeze_replay(hist, lr, W, T.astype(np.float64), frontmost=frontmost)
+    assert ref["restarts"] >= 1 and ref["frozen"].any()
+    ctx = eg.Context([64] * M, 8, W, T, eg.FLAG_FRONTMOST if frontmost else 0, device=DEV)
+    out = ctx.egeria_plasticity_replay_lr(torch.from_numpy(hist).to(DEV), torch.from_numpy(lr).to(DEV))
+    slopes, frozen, window, restarted, mask, fe = [t.cpu().numpy() for t in out]
+    assert window.tolist() == ref["window"].tolist()
+    assert restarted.tolist() == ref["restarted"].tolist()
+    assert np.array_equal(np.isnan(slopes), np.isnan(ref["slopes"]))
+    fin = np.isfinite(ref["slopes"])
+    np.testing.assert_allclose(slopes[fin], ref["slopes"][fin], rtol=1e-9, atol=1e-15)
+    # decisions: compared wherever no slope of the module's current run came within 1e-6 of T
+    near = np.zeros((H, M), dtype=bool)
+    for m in range(M):
+        close = np.isfinite(ref["slopes"][m]) & (np.abs(np.abs(ref["slopes"][m]) - float(T[m])) <= 1e-6)
+        run_start = 0
+        for i in range(H):
+            near[i, m] = close[run_start:i + 1].any()
+            if ref["restarted"][i]:
+                run_start = i + 1
+    if frontmost:
+        near = np.repeat(near.any(axis=1)[:, None], M, axis=1)
+    assert (~near).mean() > 0.8
+    assert np.array_equal(frozen[~near], ref["frozen"][~near])
+    assert mask.tolist() == frozen[-1].tolist()
+    # without a learning rate the call is the plain replay
+    s2, fz2, w2, r2, mk2, fe2 = [t.cpu().numpy() for t in
+                                 ctx.egeria_plasticity_replay_lr(torch.from_numpy(hist).to(DEV), None)]
+    s1, mk1, fe1 = [t.cpu().numpy() for t in ctx.egeria_plasticity_replay(torch.from_numpy(hist).to(DEV))]
+    assert not r2.any() and np.all(w2 == W)
+    assert np.array_equal(np.isnan(s1), np.isnan(s2)) and np.array_equal(s1[~np.isnan(s1)], s2[~np.isnan(s2)])
+    assert mk1.tolist() == mk2.tolist() and fe1.tolist() == fe2.tolist()
+    ctx.close()
+
+
+def test_unfreeze_hand_traces_on_gpu():
+    for line in (GOLDEN / "unfreeze_traces.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        f = [x.strip() for x in line.split("|")]
+        frontmost, W = bool(int(f[1])), int(f[2])
+        T = np.array([float(v) for v in f[3].split()], dtype=np.float32)
+        hist = np.array([[float(v) for v in row.split()] for row in f[4].split(";")], dtype=np.float32)
+        lr = np.array([float(v) for v in f[5].split()])
+        M, H = hist.shape
+        ctx = eg.Context([64] * M, 8, W, T, eg.FLAG_FRONTMOST if frontmost else 0, device=DEV)
+        out = ctx.egeria_plasticity_replay_lr(torch.from_numpy(hist).to(DEV), torch.from_numpy(lr).to(DEV))
+        slopes, frozen, window, restarted = [t.cpu().numpy() for t in out[:4]]
+        assert window.tolist() == [int(v) for v in f[6].split()]
+        assert ["".join(str(int(v)) for v in row) for row in frozen] == f[7].split()
+        assert np.nonzero(restarted)[0].tolist() == [int(v) for v in f[8].split()]
+        # and one evaluation at a time
+        dev = torch.from_numpy(hist).to(DEV)
+        for i in range(H):
+            ctx.egeria_plasticity_set_lr(float(lr[i]))
+            _, mk = ctx.egeria_plasticity_step(dev[:, i].contiguous())
+            assert "".join(str(int(v)) for v in mk.cpu().numpy()) == f[7].split()[i], (f[0], i)
+        assert ctx.egeria_plasticity_restarts() == len(f[8].split())
+        ctx.close()
+
+
+def test_unfreeze_inside_the_fused_evaluation():
+    """egeria_plasticity_evaluate under a learning rate that drops tenfold: same losses, slopes and
+    masks as egeria_sp_loss_batch + egeria_plasticity_step on a second context, one restart, the
+    window halved, and the state survives export / import."""
+    ds, b, W = [4096, 2048, 1001], 40, 4
+    flags = eg.FLAG_EQUAL_SPLIT
+    fused = eg.Context(ds, b, W, 0.5, flags, device=DEV)       # a generous T: modules freeze at evaluation W
+    split = eg.Context(ds, b, W, 0.5, flags, device=DEV)
+    masks = []
+    for k in range(14):
+        rate = 0.1 if k < 7 else 0.01
+        at, ar = [], []
+        for m, d in enumerate(ds):
+            t, r = wl.make_pair(b, d, "relu", 0.3, seed=900 + 10 * k + m, device=DEV)
+            at.append(t)
+            ar.append(r)
+        for c in (fused, split):
+            c.egeria_plasticity_set_lr(rate)
+        l1, s1, m1 = fused.egeria_plasticity_evaluate(at, ar)
+        l2 = split.egeria_sp_loss_batch(at, ar)
+        s2, m2 = split.egeria_plasticity_step(l2)
+        assert l1.cpu().numpy().tobytes() == l2.cpu().numpy().tobytes()
+        assert s1.cpu().numpy().tobytes() == s2.cpu().numpy().tobytes()
+        assert m1.cpu().numpy().tobytes() == m2.cpu().numpy().tobytes()
+        masks.append(m1.cpu().numpy().tolist())
+        if k == 9:                                              # carry on from a checkpoint
+            saved = fused.egeria_plasticity_export()
+            fused.close()
+            fused = eg.Context(ds, b, W, 0.5, flags, device=DEV)
+            fused.egeria_plasticity_import(saved)
+    # frozen at evaluation W = 4; restart at 7 (the first evaluation under 0.01); W = 2: frozen again at 10
+    assert masks[3] == [0, 0, 0] and masks[4] == [1, 1, 1] and masks[6] == [1, 1, 1]
+    assert masks[7] == [0, 0, 0] and masks[9] == [0, 0, 0] and masks[10] == [1, 1, 1]
+    assert fused.egeria_plasticity_restarts() == 1 and fused.egeria_plasticity_window() == 2
+    fused.close()
+    split.close()
 
 
 def test_bootstrap_detector_matches_oracle():
