@@ -216,8 +216,49 @@ __device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const 
     return row_term<NC, true>(p, m, i, lane, gT, gR);
 }
 
-// One warp, once every row term of module m is in p.rowloss and visible: the loss (Eq. 1),
-// then optionally one evaluation of the freezing rule.
+// The rows' terms of one module are added up in ONE 64-bit integer that also counts the rows, so
+// that a single atomic add per warp both delivers its terms and tells it whether it was the last
+// (the value it gets back plus its own is then the complete sum: no scratch to re-read), and so
+// that the sum does not depend on the order of arrival (integer addition is associative):
+//   bits  0..45  sum of the terms in units of 2^-35 (a term is at most 4: both rows have unit norm;
+//                256 rows x 4 x 2^35 = 2^45)
+//   bits 46..54  rows whose term was not a finite number in [0, 4.5]  (NaN / Inf in the inputs)
+//   bits 55..63  rows delivered
+// A term is rounded to the nearest multiple of 2^-35 = 2.9e-11; over b rows and divided by b^2
+// that is at most 1.5e-11 / b on the loss.
+constexpr double kRowAccScale = 34359738368.0;  // 2^35
+constexpr int kRowAccBadShift = 46, kRowAccCountShift = 55;
+
+__device__ __forceinline__ unsigned long long row_acc_of(double term) {
+    unsigned long long v = 1ull << kRowAccCountShift;
+    if (term >= 0.0 && term <= 4.5) {  // false for NaN
+        if (term > 4.0) term = 4.0;
+        v += (unsigned long long)__double2ll_rn(term * kRowAccScale);
+    } else {
+        v += 1ull << kRowAccBadShift;
+    }
+    return v;
+}
+__device__ __forceinline__ int row_acc_rows(unsigned long long acc) { return (int)(acc >> kRowAccCountShift); }
+// Sum of the terms, NaN if any row's term was not a number in range.
+__device__ __forceinline__ double row_acc_sum(unsigned long long acc) {
+    if ((acc >> kRowAccBadShift) & 0x1ffull) return NAN;
+    return (double)(long long)(acc & ((1ull << kRowAccBadShift) - 1)) / kRowAccScale;
+}
+
+// One warp, with the sum of all row terms of module m: the loss (Eq. 1), then optionally one
+// evaluation of the freezing rule from the state loaded in L.
+__device__ __forceinline__ void finalize_module_finish(const FinCommon &p, int m, double sum_terms, StepLoaded &L,
+                                                       int lane) {
+    const double b = (double)p.b;
+    const float loss = (float)(sum_terms / (b * b));
+    if (lane == 0) p.out_losses[m] = loss;
+    if (p.fuse_step)
+        plasticity_rule_step(p.st, L, m, p.M, p.rule_flags, p.rule_serial, loss, p.lr, p.out_slopes, p.out_mask, lane);
+}
+
+// One warp, once every row term of module m is in p.rowloss and visible (the modules of the
+// CUDA-core kernel): add them in a fixed order, then as above.
 __device__ __forceinline__ void finalize_module_total(const FinCommon &p, int m, int lane) {
     const int b = p.b;
     double v[kMaxB / 32];
@@ -232,10 +273,7 @@ __device__ __forceinline__ void finalize_module_total(const FinCommon &p, int m,
 #pragma unroll
     for (int j = 0; j < kMaxB / 32; ++j) s += v[j];
     s = warp_sum_f64(s);
-    const float loss = (float)(s / ((double)b * (double)b));
-    if (lane == 0) p.out_losses[m] = loss;
-    if (p.fuse_step)
-        plasticity_rule_step(p.st, L, m, p.M, p.rule_flags, p.rule_serial, loss, p.lr, p.out_slopes, p.out_mask, lane);
+    finalize_module_finish(p, m, s, L, lane);
 }
 
 struct FinParams {

@@ -178,51 +178,14 @@ __device__ __forceinline__ bool next_chunk(int &k, int q, int lane, int b, float
     return false;
 }
 
-// One warp: wait until `total` units of the module are complete, to help finish it.  The first
-// warp of the CTA to get here polls the counter (a counter that every waiting warp of every CTA
-// polled would be a hot spot); the others watch its verdict in shared memory (*state: 0 nobody
-// polls yet, 1 being polled, 2 complete, 3 gave up).  The wait is a courtesy, not a dependency:
-// the CTA that delivers the module's last unit finishes every row nobody else has claimed, so a
-// CTA that stops waiting (false) loses nothing but parallelism.  That keeps the kernel correct
-// when not all of its CTAs are resident together.
-__device__ __forceinline__ bool wait_units_done(const int32_t *units_done, int total, volatile int *abort_flag,
-                                                int *state, int lane) {
-    int v = 0;
-    if (lane == 0) {
-        if (atomicCAS(state, 0, 1) == 0) {
-            v = 2;
-            const uint64_t t0 = ptx::globaltimer_ns();
-            while (ld_acquire(units_done) < total) {
-                if (*abort_flag || ptx::globaltimer_ns() - t0 > kHelpWaitNs) {
-                    v = 3;
-                    break;
-                }
-                __nanosleep(100);
-            }
-            __threadfence_block();
-            *reinterpret_cast<volatile int *>(state) = v;
-        } else {
-            const uint64_t t0 = ptx::globaltimer_ns();
-            while ((v = *reinterpret_cast<volatile int *>(state)) == 1) {
-                if (ptx::globaltimer_ns() - t0 > 2 * kHelpWaitNs) {
-                    v = 3;
-                    break;
-                }
-                __nanosleep(50);
-            }
-        }
-    }
-    return __shfl_sync(0xffffffffu, v, 0) == 2;
-}
-
 // One warp: take rows of module m from its cursor until none is left.  The claim of the next
-// row is in flight while the current one is worked on; the rows are published together.
+// row is in flight while the current one is worked on; the rows' terms are delivered together.
 // `stage` is kFinStageBytes of shared memory for this warp alone.
 template <int NC>
 __device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int lane, float *stage) {
     const int b = p.fin.b;
     FinCounters *c = p.ctr + m;
-    int mine = 0;
+    unsigned long long mine = 0;  // this warp's rows and their terms, packed (row_acc_of)
     int r = 0;
     if (lane == 0) r = atomicAdd(&c->row_cursor, 1);
     const SideInfo sT = p.fin.sides[2 * m], sR = p.fin.sides[2 * m + 1];  // in flight with the claim
@@ -231,21 +194,19 @@ __device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int
         int r_next = 0;
         if (lane == 0) r_next = atomicAdd(&c->row_cursor, 1);
         const double term = finalize_row_staged<NC>(p.fin, sT, sR, m, r, lane, stage);
-        if (lane == 0) p.fin.rowloss[(int64_t)m * kMaxB + r] = term;
-        ++mine;
+        mine += row_acc_of(term);
         r = __shfl_sync(0xffffffffu, r_next, 0);
     }
     if (mine == 0) return;
-    int before = 0;
-    if (lane == 0) {
-        __threadfence();
-        before = atomicAdd(&c->rows_done, mine);
-    }
+    // One atomic add delivers the terms and says whether these were the module's last rows; what
+    // the rule needs is loaded meanwhile (only the last warp uses it).
+    unsigned long long before = 0;
+    if (lane == 0) before = atomicAdd(&c->row_acc, mine);
+    StepLoaded L;
+    if (p.fin.fuse_step) L = plasticity_step_load(p.fin.st, m, lane);
     before = __shfl_sync(0xffffffffu, before, 0);
-    if (before + mine == b) {
-        __threadfence();
-        finalize_module_total(p.fin, m, lane);
-    }
+    const unsigned long long all = before + mine;
+    if (row_acc_rows(all) == b) finalize_module_finish(p.fin, m, row_acc_sum(all), L, lane);
 }
 }  // namespace detail
 
@@ -265,7 +226,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     volatile uint32_t *tmem_holder =
         reinterpret_cast<volatile uint32_t *>(bars + 2 * Cfg::kStages + 2 * Cfg::kAccStages);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
-    int *wait_state = reinterpret_cast<int *>(const_cast<uint32_t *>(tmem_holder) + 2);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -289,7 +249,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             ptx::mbar_init(accempty0 + 8 * s, kEpiWarps);  // one arrival per epilogue warp
         }
         *abort_flag = 0;
-        *wait_state = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
     }
@@ -517,34 +476,60 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             static_assert(kEpiWarps * kFinStageBytes <= Cfg::kStages * Cfg::kStageBytes, "ring too small to stage");
             float *stage = reinterpret_cast<float *>(smem_aligned + (warp - 2) * kFinStageBytes);
             ptx::fence_proxy_async();  // the ring was last touched by TMA and the tensor cores
-            const int m_last = (u_end > u_begin) ? p.units[u_end - 1].module : -1;
-            int prev_m = -1;
-            for (int ui = u_begin; ui < u_end; ++ui) {
-                const int m = p.units[ui].module;
-                if (m == prev_m) continue;
-                prev_m = m;
-                const int total = p.fin.sides[2 * m].module_units;
-                // With many CTAs on a module and few rows, most claims would find nothing and only
-                // crowd the cursor: as many warps of this CTA as its share of the rows, plus one.
-                const int ctas_on_m = Cfg::kStacked ? total : (total + 1) / 2;
-                if (warp - 2 > (b + ctas_on_m - 1) / ctas_on_m) continue;
-                bool ready;
-                if (m == m_last) {
-                    ready = detail::wait_units_done(&p.ctr[m].units_done, total, abort_flag, wait_state, lane);
-                } else {
-                    int done = 0;
-                    if (lane == 0) done = detail::ld_acquire(&p.ctr[m].units_done);
-                    ready = (__shfl_sync(0xffffffffu, done, 0) >= total);
+            // The modules this CTA worked on, 32 units at a time: lane j looks after the module of
+            // unit j (the first unit of each module only; a module's units are adjacent).  The warp
+            // polls their counters together, finishes rows wherever a module is complete and has
+            // rows nobody has claimed -- warps start at different modules, so that a CTA whose range
+            // covers parts of several modules works on all of them at once -- and waits (a while)
+            // for those that are not complete yet.  The wait is a courtesy, see above.
+            for (int base = u_begin; base < u_end; base += 32) {
+                int my_m = -1, my_total = 0;
+                if (base + lane < u_end) {
+                    my_m = p.units[base + lane].module;
+                    if (base + lane > u_begin && p.units[base + lane - 1].module == my_m) my_m = -1;
                 }
-                if (ready) {
-                    __threadfence();
-                    detail::finish_module_rows<Cfg::kNC>(p, m, lane, stage);
+                if (my_m >= 0) {
+                    my_total = p.fin.sides[2 * my_m].module_units;
+                    // With many CTAs on a module and few rows, most claims would find nothing and only
+                    // crowd the cursor: as many warps of this CTA as its share of the rows, plus one.
+                    const int ctas_on_m = Cfg::kStacked ? my_total : (my_total + 1) / 2;
+                    if (warp - 2 > (b + ctas_on_m - 1) / ctas_on_m) my_m = -1;
+                }
+                uint32_t pending = __ballot_sync(0xffffffffu, my_m >= 0);
+                uint64_t t_wait = ptx::globaltimer_ns();
+                while (pending) {
+                    bool ready = false;
+                    int left = 0;
+                    if ((pending >> lane) & 1u) {
+                        const int done = detail::ld_acquire(&p.ctr[my_m].units_done);
+                        const int cur = detail::ld_acquire(&p.ctr[my_m].row_cursor);
+                        ready = (done >= my_total);
+                        left = b - cur;
+                    }
+                    pending &= ~__ballot_sync(0xffffffffu, ready && left <= 0);  // complete, every row claimed
+                    const uint32_t cand = __ballot_sync(0xffffffffu, ready && left > 0);
+                    if (cand) {
+                        const int pick = (int)__fns(cand, 0, 1 + (warp - 2) % __popc(cand));
+                        const int m = __shfl_sync(0xffffffffu, my_m, pick);
+                        __threadfence();
+                        detail::finish_module_rows<Cfg::kNC>(p, m, lane, stage);  // returns when no row is left to claim
+                        pending &= ~(1u << pick);
+                        t_wait = ptx::globaltimer_ns();
+                    } else if (pending) {
+                        int stop = 0;
+                        if (lane == 0) stop = (*abort_flag != 0) || (ptx::globaltimer_ns() - t_wait > kHelpWaitNs);
+                        if (__shfl_sync(0xffffffffu, stop, 0)) break;
+                        __nanosleep(100);
+                    }
                 }
             }
             // Then look at all the other modules, a few times: where one is complete and still has
             // many rows nobody has claimed (few CTAs worked on it, so its rows go slowly), lend a
             // hand to the one with the most rows left.
-            for (int round = 0; round < 3; ++round) {
+            // (With fewer rows in all than half the epilogue warps of the grid there is nothing to
+            // lend a hand with, and the look itself would be the last thing the kernel waits for.)
+            const int help_rounds = (2 * (int64_t)b * p.M < (int64_t)gridDim.x * kEpiWarps) ? 0 : 3;
+            for (int round = 0; round < help_rounds; ++round) {
                 int best_left = 0, best_m = -1;
                 for (int mm = lane; mm < p.M; mm += 32) {
                     const SideInfo si = p.fin.sides[2 * mm];

@@ -77,8 +77,9 @@ struct FinCounters {
     int32_t pad0[31];
     int32_t row_cursor;  // next row of G nobody has claimed yet
     int32_t pad1[31];
-    int32_t rows_done;   // rows whose term of the loss is in the row scratch
-    int32_t pad2[31];
+    unsigned long long row_acc;  // the rows' terms of the loss so far and how many rows they are (packed:
+                                 // one atomic add per warp carries both, see finalize.cuh)
+    int32_t pad2[30];
 };
 
 // Per-module pointers for the CUDA-core kernel.
