@@ -35,8 +35,28 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the evaluation kernel, from the ncu
 # captures summarised under profiles/ (gpt2_medium: a 6-module launch scaled x4 by the modules
-# processed).  Valid for the kernel as captured; set to None when the kernel changes.
-NCU_TRAFFIC_BYTES = {"gpt2_medium": 6476067000, "resnet50": 1419185000}
+# processed), with the hash of the kernel sources they were taken from: the figure is reported only
+# while the sources still hash to that (kernel_sources_hash below), else null.
+NCU_TRAFFIC_BYTES = {"gpt2_medium": (6476067000, "stale"), "resnet50": (1419185000, "stale")}
+NOMINAL_HBM_GBS = 8000.0     # the "about 8 TB/s" the target is stated against
+
+
+def kernel_sources_hash() -> str:
+    """sha256 (first 16 hex digits) over the CUDA sources of the library, in name order."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted((ROOT / "paper_2201_06227_b200" / "csrc").iterdir()):
+        if f.suffix in (".cu", ".cuh", ".h"):
+            h.update(f.name.encode())
+            h.update(f.read_bytes())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(name: str):
+    entry = NCU_TRAFFIC_BYTES.get(name)
+    if entry is None or entry[1] != kernel_sources_hash():
+        return None
+    return entry[0]
 
 
 # ----------------------------------------------------------------------------- helpers
@@ -122,6 +142,40 @@ def oracle_sample(w: wl.Workload, budget_s: float = 12.0, max_modules: int = 4):
             "sample": f"modules 0..{done - 1} of {w.M} ({w.name}), float64 SP loss, {spent:.1f} s"}, spent, done
 
 
+def oracle_full_step(w: wl.Workload, budget_s: float = 30.0, one_thread: bool = False):
+    """The CPU oracle on one whole evaluation of the workload (every module), or on as many modules
+    as fit the budget; optionally again on one thread."""
+    import oracle
+    oracle.build()
+    cores = oracle.num_threads()
+
+    def run(max_s):
+        done, spent = 0, 0.0
+        for l in range(w.M):
+            at, ar = wl.make_module(w, l, "cpu")
+            ta, tr = wl.bf16_bits(at), wl.bf16_bits(ar)
+            t0 = time.perf_counter()
+            oracle.sp_loss(ta, tr)
+            spent += time.perf_counter() - t0
+            done += 1
+            if spent >= max_s:
+                break
+        return done, spent
+
+    done, spent = run(budget_s)
+    out = {"value": done / spent, "unit": UNIT, "cores": cores, "kind": "oracle", "modules_timed": done,
+           "whole_step": done == w.M, "seconds": spent}
+    if one_thread:
+        oracle.set_num_threads(1)
+        try:
+            d1, s1 = run(budget_s)
+        finally:
+            oracle.set_num_threads(cores)
+        out["value_1thread"] = d1 / s1
+        out["modules_timed_1thread"] = d1
+    return out
+
+
 # ----------------------------------------------------------------------------- reference arm (the oracle)
 
 def run_reference(args):
@@ -130,11 +184,14 @@ def run_reference(args):
         return
     w = wl.WORKLOADS[args.workload]
     per_step_budget = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
+    # the small workloads are cheap enough for every step to be a whole evaluation
+    whole = w.input_bytes < 2e9 and args.steps + args.warmup <= 30
     for _ in range(args.warmup):
         oracle_sample(w, budget_s=per_step_budget, max_modules=1)
     spent_total, done_total, cores, sample = 0.0, 0, 1, ""
     for _ in range(args.steps):
-        cb, spent, done = oracle_sample(w, budget_s=per_step_budget, max_modules=2)
+        cb, spent, done = oracle_sample(w, budget_s=1e9 if whole else per_step_budget,
+                                        max_modules=w.M if whole else 2)
         spent_total += spent
         done_total += done
         cores, sample = cb["cores"], cb["sample"]
@@ -144,7 +201,8 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * spent_total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": {"workload": w.name, "b": w.b, "modules": w.M,
-                                        "note": "each step is a bounded sample (first modules) of the workload"},
+                                        "note": ("each step is one whole evaluation" if whole else
+                                                 "each step is a bounded sample (first modules) of the workload")},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -185,7 +243,7 @@ def n_sets_for(w: wl.Workload) -> int:
     return min(16, max(2, int(np.ceil(8 * 126e6 / w.input_bytes))))
 
 
-def measure_other(eg, name, device, stream, steps, warmup):
+def measure_other(eg, name, device, stream, steps, warmup, oracle_too=False, front_only=False):
     """Short device-timed run of another named workload (context for the headline line)."""
     w = wl.WORKLOADS[name]
     n_sets = n_sets_for(w)
@@ -207,14 +265,69 @@ def measure_other(eg, name, device, stream, steps, warmup):
     ev1.record(stream)
     torch.cuda.synchronize(device)
     ms = ev0.elapsed_time(ev1) / steps
+    # the same with ONE input set evaluated again and again: for a workload that fits the 126 MB L2
+    # (or nearly) the reads then come partly from L2 -- labelled as such, never the headline
+    warm_ms = None
+    if n_sets > 1:
+        ev0.record(stream)
+        for i in range(steps):
+            step(0)
+        ev1.record(stream)
+        torch.cuda.synchronize(device)
+        warm_ms = ev0.elapsed_time(ev1) / steps
     ctx.check_device_status()
     ctx.close()
     peak, _ = hbm_peak()
     gram_s = gram_ms / max(1, calls) * 1e-3
-    return {"b": w.b, "modules": w.M, "input_bytes_per_step": w.input_bytes, "ms_per_step": ms,
-            "value": w.M / (ms * 1e-3), "gram_kernel_ms": gram_s * 1e3,
-            "gram_GBps": w.input_bytes / gram_s / 1e9, "roofline_frac": w.input_bytes / gram_s / 1e9 / peak,
-            "step_frac_of_hbm_roofline": (w.input_bytes / (peak * 1e9)) / (ms * 1e-3), "input_sets": n_sets}
+    out = {"b": w.b, "modules": w.M, "input_bytes_per_step": w.input_bytes, "ms_per_step": ms,
+           "value": w.M / (ms * 1e-3), "gram_kernel_ms": gram_s * 1e3,
+           "gram_GBps": w.input_bytes / gram_s / 1e9, "roofline_frac": w.input_bytes / gram_s / 1e9 / peak,
+           "step_frac_of_hbm_roofline": (w.input_bytes / (peak * 1e9)) / (ms * 1e-3),
+           "step_frac_nominal_8TBs": (w.input_bytes / (NOMINAL_HBM_GBS * 1e9)) / (ms * 1e-3),
+           "input_sets": n_sets, "warm_l2_ms_per_step (one input set, not from HBM)": warm_ms}
+    if oracle_too:
+        # the oracle on one whole evaluation of this workload, on the host's cores (and on one of them
+        # where that takes seconds): a reported baseline, not a target
+        out["cpu_baseline"] = oracle_full_step(w, one_thread=(w.input_bytes < 2e8))
+    if front_only:
+        # frontmost policy with the monitored module chosen on the device: the cost of one evaluation
+        # while module 0 is the front, beside the cost of evaluating every module
+        del sets, step
+        torch.cuda.empty_cache()
+        out["front_only"] = measure_front_only(eg, w, device, stream, steps, warmup, ms)
+    return out
+
+
+def measure_front_only(eg, w, device, stream, steps, warmup, full_ms):
+    at, ar = [], []
+    for l in range(w.M):
+        t, r = wl.make_pair(w.b, w.d[l], w.kind, w.sigma_of(l), w.seed_of(l), device)
+        at.append(t)
+        ar.append(r)
+    # a tolerance of zero: nothing ever freezes, module 0 stays the monitored one
+    ctx = eg.Context(list(w.d), w.b, w.W, 0.0, eg.FLAG_FRONTMOST | eg.FLAG_FRONT_ONLY, device=device)
+    losses = torch.empty(w.M, dtype=torch.float32, device=device)
+    slopes = torch.empty(w.M, dtype=torch.float64, device=device)
+    mask = torch.empty(w.M, dtype=torch.uint8, device=device)
+    pa, pr = ctx._ptr_array(at, w.b, True), ctx._ptr_array(ar, w.b, True)
+    sp = int(stream.cuda_stream)
+    # a second module-0 buffer pair to alternate with would not change the picture: 205 MB > L2
+    for _ in range(warmup + 12):
+        ctx.plasticity_evaluate_raw(pa, pr, w.b, losses.data_ptr(), slopes.data_ptr(), mask.data_ptr(), sp)
+    torch.cuda.synchronize(device)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(steps):
+        ctx.plasticity_evaluate_raw(pa, pr, w.b, losses.data_ptr(), slopes.data_ptr(), mask.data_ptr(), sp)
+    ev1.record(stream)
+    torch.cuda.synchronize(device)
+    ms = ev0.elapsed_time(ev1) / steps
+    ctx.check_device_status()
+    ctx.close()
+    share = w.d[0] / w.sum_d
+    return {"monitored_module": 0, "ms_per_step": ms, "all_modules_ms_per_step": full_ms,
+            "cost_ratio": ms / full_ms, "module_share_of_bytes": share,
+            "frac_of_hbm_roofline": (4 * w.b * w.d[0] / (hbm_peak()[0] * 1e9)) / (ms * 1e-3)}
 
 
 def time_workload(eg, w, device, steps, warmup, n_sets, stream, time_gram=True, sets=None):
@@ -385,18 +498,23 @@ def run_ours(args):
     achieved = w.input_bytes / gram_s / 1e9 if gram_s > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "gram_tc_kernel (Gram + finalisation + freezing rule)", "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(w.name) if not args.modules else None,
+                "frac_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "traffic": ncu_traffic(w.name) if not args.modules else None,
+                "kernel_sources_hash": kernel_sources_hash(),
                 "algorithmic_bytes_per_launch": w.input_bytes,
                 "avg_launch_ms": gram_s * 1e3, "launches_timed": gram_calls}
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
-        cpu_baseline, _, _ = oracle_sample(w)
+        cpu_baseline = oracle_full_step(w, budget_s=25.0)
+        cpu_baseline["sample"] = (f"modules 0..{cpu_baseline['modules_timed'] - 1} of {w.M} ({w.name}), float64 SP loss, "
+                                  f"{cpu_baseline['seconds']:.1f} s")
     others = None
     if world == 1 and not args.no_others:
         ctx.close()
         del sets, step
         torch.cuda.empty_cache()
-        others = {n: measure_other(eg, n, device, stream, 20, 5) for n in wl.ORDER if n != w.name}
+        others = {n: measure_other(eg, n, device, stream, 20, 5, oracle_too=not args.no_cpu_baseline,
+                                   front_only=(n == "resnet50")) for n in wl.ORDER if n != w.name}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps,
@@ -412,6 +530,12 @@ def run_ours(args):
         "cpu_baseline": cpu_baseline, "other_workloads": others,
     }
     line["roofline"]["step_frac"] = (w.input_bytes / (peak * 1e9)) / (elapsed_ms * 1e-3 / args.steps)
+    # time x median SM clock, headline and sustained: how much of the difference is the clock
+    if clocks and clocks.get("sm_mhz"):
+        line["clocks"]["ms_x_mhz_per_step"] = elapsed_ms / args.steps * clocks["sm_mhz"]
+    if sustained and sustained["clocks"].get("sm_mhz"):
+        sustained["clocks"]["ms_x_mhz_per_step"] = sustained["ms_per_step"] * sustained["clocks"]["sm_mhz"]
+        sustained["step_frac_nominal_8TBs"] = (w.input_bytes / (NOMINAL_HBM_GBS * 1e9)) / (sustained["ms_per_step"] * 1e-3)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()

@@ -93,7 +93,21 @@ enum {
      * state.  out_mask is then a prefix mask (1 for the frozen modules) and
      * out_slopes holds this evaluation's slope for the monitored module, the
      * final slope of every frozen one and +inf for those not monitored yet. */
-    EGERIA_FLAG_FRONTMOST = 128u
+    EGERIA_FLAG_FRONTMOST = 128u,
+    /* With EGERIA_FLAG_FRONTMOST: egeria_plasticity_evaluate computes the loss of the monitored
+     * module ONLY [Sec. 3: only the activation of the frontmost module that is not frozen is
+     * collected; Algorithm 1 is called with that one module].  Which module that is, is decided
+     * on the device when the kernel starts (it reads the front the previous evaluation left), so
+     * the caller never reads anything back: the work split of every possible front is kept on
+     * the device, each spreading its one module over the whole GPU, and an evaluation costs
+     * about that module's share of a full one.  Only out_losses[front] is written; out_mask
+     * and out_slopes are reported as under EGERIA_FLAG_FRONTMOST.  The pointers of ALL modules
+     * must still be valid (any of them may be the front), and every module must qualify for
+     * the TMA + tcgen05 kernel (d_l a multiple of 8, 16-byte aligned pointers), else
+     * EGERIA_ERR_UNSUPPORTED_SHAPE.  Once every module is frozen an evaluation does no work
+     * beyond reporting the mask.  egeria_sp_loss_batch and the subset calls are not affected
+     * (the subset form of the evaluation is refused: EGERIA_ERR_INVALID_ARG). */
+    EGERIA_FLAG_FRONT_ONLY = 256u
 };
 
 #define EGERIA_MAX_B 256          /* largest supported mini-batch size */

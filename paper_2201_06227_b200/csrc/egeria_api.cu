@@ -42,10 +42,16 @@ struct Layout {
     size_t tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides;
 };
 
-static int64_t units_cap(int M, int b_max) {
+// Units of one device-side plan: all modules in one split, or (front-only contexts) one split per
+// possible front, each over a single module.
+static int64_t units_cap(int M, int b_max, uint32_t flags) {
     int64_t cap = 0;
     for (int mode = 0; mode <= mode_of_b(b_max); ++mode) {
-        const int64_t u = max_units(M, mode, kMaxCtas);
+        int64_t u = max_units(M, mode, kMaxCtas);
+        if (flags & EGERIA_FLAG_FRONT_ONLY) {
+            const int64_t f = (int64_t)M * max_units(1, mode, kMaxCtas);
+            if (f > u) u = f;
+        }
         if (u > cap) cap = u;
     }
     return cap;
@@ -65,8 +71,8 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
         off = 0;
         L.tmaps = take((size_t)2 * M * sizeof(CUtensorMap));
         L.modules = take((size_t)M * sizeof(ModulePtrs));
-        L.units = take((size_t)units_cap(M, b_max) * sizeof(Unit));
-        L.cta_begin_tc = take((kMaxCtas + 1) * sizeof(int32_t));
+        L.units = take((size_t)units_cap(M, b_max, flags) * sizeof(Unit));
+        L.cta_begin_tc = take((size_t)((flags & EGERIA_FLAG_FRONT_ONLY) ? M : 1) * (kMaxCtas + 1) * sizeof(int32_t));
         L.cta_begin_simt = take((kMaxCtas + 1) * sizeof(int32_t));
         L.sides = take((size_t)2 * M * sizeof(SideInfo));
         L.plan_stride = off;
@@ -151,6 +157,7 @@ struct egeria_ctx {
     // device-side plans, least recently used one is replaced
     struct PlanEntry {
         int b = -1;
+        bool front_only = false;  // one split per possible front (plan.units is their concatenation)
         int weights_version = 0;
         std::vector<const void *> At, Ar;
         Plan plan;
@@ -287,6 +294,7 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     *out = nullptr;
     egeria_status s = check_shapes(M, d, b_max, W);
     if (s != EGERIA_OK) return s;
+    if ((flags & EGERIA_FLAG_FRONT_ONLY) && !(flags & EGERIA_FLAG_FRONTMOST)) return EGERIA_ERR_INVALID_ARG;
     Layout L;
     make_layout(M, d, b_max, W, flags, L);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % EGERIA_WORKSPACE_ALIGN) != 0 ||
@@ -470,13 +478,14 @@ static void poll_calibration(egeria_ctx *ctx) {
 
 // Select (or build and upload) the device-side plan for this (b, pointers).
 static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const void *const *At, const void *const *Ar,
-                                  int b) {
+                                  int b, bool front_only) {
     const int M = ctx->M;
     const size_t pbytes = (size_t)M * sizeof(void *);
     int lru = 0;
     for (int i = 0; i < kPlanSlots; ++i) {
         egeria_ctx::PlanEntry &e = ctx->plans[i];
-        if (e.b == b && e.weights_version == ctx->weights_version && memcmp(e.At.data(), At, pbytes) == 0 &&
+        if (e.b == b && e.front_only == front_only && e.weights_version == ctx->weights_version &&
+            memcmp(e.At.data(), At, pbytes) == 0 &&
             memcmp(e.Ar.data(), Ar, pbytes) == 0) {
             e.last_use = ++ctx->use_clock;
             ctx->cur = i;
@@ -498,11 +507,44 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
                              (reinterpret_cast<uintptr_t>(Ar[m]) % 16 == 0) && (ctx->d[m] % 8 == 0);
         tc_ok[m] = (aligned && !(ctx->flags & EGERIA_FLAG_FORCE_SIMT)) ? 1 : 0;
     }
-    build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), e.plan,
-               ctx->weights_version > 0 ? ctx->weights.data() : nullptr);
+    const float *weights = ctx->weights_version > 0 ? ctx->weights.data() : nullptr;
+    std::vector<int32_t> front_cta_begin;  // front-only: [M][kMaxCtas + 1] into the concatenated units
+    if (!front_only) {
+        build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), e.plan, weights);
+    } else {
+        // One split per possible front: module f alone over all CTAs.  Slots are numbered from 0 in
+        // each (only one of them runs in a launch).
+        for (int m = 0; m < M; ++m)
+            if (tc_ok[m] != 1) return EGERIA_ERR_UNSUPPORTED_SHAPE;
+        Plan &all = e.plan;
+        all = Plan{};
+        all.mode = mode_of_b(b);
+        all.n_ctas = ctx->n_ctas;
+        all.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, {0, 0}});
+        all.all_ctas_busy_tc = true;
+        front_cta_begin.assign((size_t)M * (kMaxCtas + 1), 0);
+        std::vector<uint8_t> only(M);
+        Plan one;
+        for (int f = 0; f < M; ++f) {
+            for (int m = 0; m < M; ++m) only[m] = (m == f) ? 1 : 2;
+            build_plan(M, ctx->d.data(), b, ctx->n_ctas, only.data(), one, weights);
+            const int32_t base = (int32_t)all.units.size();
+            all.units.insert(all.units.end(), one.units.begin(), one.units.end());
+            for (int c = 0; c <= ctx->n_ctas; ++c)
+                front_cta_begin[(size_t)f * (kMaxCtas + 1) + c] = base + one.cta_begin_tc[c];
+            all.sides[2 * (size_t)f] = one.sides[2 * (size_t)f];
+            all.sides[2 * (size_t)f + 1] = one.sides[2 * (size_t)f + 1];
+            all.all_ctas_busy_tc = all.all_ctas_busy_tc && one.all_ctas_busy_tc;
+            if ((size_t)one.units.size() * slot_floats_of_mode(one.mode) * sizeof(float) > ctx->L.slot_bytes_cap)
+                return EGERIA_ERR_WORKSPACE;
+        }
+        all.n_units_tc = (int)all.units.size();
+        all.cta_begin_tc.assign(ctx->n_ctas + 1, 0);
+        all.cta_begin_simt.assign(ctx->n_ctas + 1, 0);
+    }
     const Plan &P = e.plan;
     const Layout &L = ctx->L;
-    if ((size_t)P.units.size() * slot_floats_of_mode(P.mode) * sizeof(float) > L.slot_bytes_cap ||
+    if ((!front_only && (size_t)P.units.size() * slot_floats_of_mode(P.mode) * sizeof(float) > L.slot_bytes_cap) ||
         L.units + P.units.size() * sizeof(Unit) > L.cta_begin_tc)
         return EGERIA_ERR_WORKSPACE;
 
@@ -532,7 +574,10 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
         if (s != EGERIA_OK) return s;
     }
     if (!P.units.empty()) memcpy(img + L.units, P.units.data(), P.units.size() * sizeof(Unit));
-    memcpy(img + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t));
+    if (front_only)
+        memcpy(img + L.cta_begin_tc, front_cta_begin.data(), front_cta_begin.size() * sizeof(int32_t));
+    else
+        memcpy(img + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t));
     memcpy(img + L.cta_begin_simt, P.cta_begin_simt.data(), P.cta_begin_simt.size() * sizeof(int32_t));
     memcpy(img + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo));
     // From pageable memory the runtime stages the bytes before returning, so `pack` may be reused.
@@ -542,6 +587,7 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
         ctx->plan_upload_pending[lru] = true;
     }
     e.b = b;
+    e.front_only = front_only;
     e.weights_version = ctx->weights_version;
     e.At.assign(At, At + M);
     e.Ar.assign(Ar, Ar + M);
@@ -651,7 +697,9 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
     egeria_status s = set_attrs(ctx);
     if (s != EGERIA_OK) return s;
     poll_calibration(ctx);
-    s = refresh_plan(ctx, stream, At, Ar, b);
+    const bool front_only = fuse_step && (ctx->flags & EGERIA_FLAG_FRONT_ONLY);
+    if (front_only && active) return EGERIA_ERR_INVALID_ARG;
+    s = refresh_plan(ctx, stream, At, Ar, b, front_only);
     if (s != EGERIA_OK) return s;
 
     const Layout &L = ctx->L;
@@ -694,6 +742,8 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         tp.tmaps = reinterpret_cast<const CUtensorMap *>(region + L.tmaps);
         tp.units = reinterpret_cast<const Unit *>(region + L.units);
         tp.cta_begin = reinterpret_cast<const int32_t *>(region + L.cta_begin_tc);
+        tp.front_word = front_only ? ctx->slope_state().front : nullptr;
+        tp.cta_stride = kMaxCtas + 1;
         tp.slots = ctx->at<float>(L.slots);
         tp.status = ctx->at<int32_t>(L.status);
         FinCounters *sets = ctx->at<FinCounters>(L.fin_ctr);
@@ -1161,6 +1211,8 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         tp.tmaps = reinterpret_cast<const CUtensorMap *>(ws + L.tmaps);
         tp.units = reinterpret_cast<const Unit *>(ws + L.units);
         tp.cta_begin = reinterpret_cast<const int32_t *>(ws + L.cta_begin_tc);
+        tp.front_word = nullptr;
+        tp.cta_stride = 0;
         tp.slots = reinterpret_cast<float *>(ws + L.slots);
         tp.status = ticket + 1;
         tp.ctr = reinterpret_cast<FinCounters *>(ticket + 2);

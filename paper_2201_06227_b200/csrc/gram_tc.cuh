@@ -67,6 +67,11 @@ struct TcParams {
     const CUtensorMap *tmaps;  // [2 * M]: A_T and A_R of every module (device memory)
     const Unit *units;         // tensor-core units
     const int32_t *cta_begin;  // [gridDim.x + 1]
+    // Front-only evaluation (else nullptr): the word that holds the number of frozen modules; the
+    // work split of front f starts at cta_begin + f * cta_stride, and with every module frozen
+    // there is no work.
+    const unsigned long long *front_word;
+    int32_t cta_stride;
     float *slots;              // partial Gram slots
     int32_t *status;           // device status word
     FinCounters *ctr;          // [M] progress counters of this launch (all zero at launch)
@@ -229,8 +234,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int u_begin = p.cta_begin[blockIdx.x];
-    const int u_end = p.cta_begin[blockIdx.x + 1];
+    int u_begin = 0, u_end = 0;
+    bool all_frozen = false;  // front-only evaluation with nothing left to monitor
+    {
+        const int32_t *cta_begin = p.cta_begin;
+        if (p.front_word) {
+            const int front = (int)(uint32_t)*reinterpret_cast<const volatile unsigned long long *>(p.front_word);
+            all_frozen = (front >= p.M);
+            cta_begin += (int64_t)(all_frozen ? 0 : front) * p.cta_stride;
+        }
+        if (!all_frozen) {
+            u_begin = cta_begin[blockIdx.x];
+            u_end = cta_begin[blockIdx.x + 1];
+        }
+    }
 
     // The counters of the next launch start at zero (nobody reads that set during this launch).
     {
@@ -468,6 +485,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             __threadfence();
             detail::epi_bar_sync();
             if (epi_leader) atomicAdd(&p.ctr[u.module].units_done, 1);
+        }
+        if (all_frozen && blockIdx.x == 0 && warp == 2) {
+            // nothing is monitored any more: the rule only reports (prefix mask of ones, final slopes)
+            StepLoaded L = plasticity_step_load(p.fin.st, p.M - 1, lane);
+            plasticity_rule_step(p.fin.st, L, p.M - 1, p.M, p.fin.rule_flags, p.fin.rule_serial, 0.f, p.fin.lr,
+                                 p.fin.out_slopes, p.fin.out_mask, lane);
         }
         if (!aborted) {
             // All of this CTA's units are in and its pipeline is idle, so the operand ring is free:

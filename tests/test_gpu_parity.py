@@ -974,6 +974,83 @@ def test_unfreeze_inside_the_fused_evaluation():
     split.close()
 
 
+def test_front_only_evaluation_follows_the_front_on_the_device():
+    """EGERIA_FLAG_FRONT_ONLY: every evaluation computes the monitored module only, chosen on the
+    device.  Decisions against oracle.frontmost_replay on the oracle's own losses of the same
+    activations; the loss written is the front module's and nothing else is touched; after a
+    restart by the unfreezing rule the front is module 0 again."""
+    ds, b, W, K = [4096, 2048, 8192, 1024, 4160], 40, 2, 18
+    M = len(ds)
+    T = 0.5                                                    # generous: a module freezes W evaluations after its start
+    fo = eg.Context(ds, b, W, T, eg.FLAG_FRONTMOST | eg.FLAG_FRONT_ONLY, device=DEV)
+    full = eg.Context(ds, b, W, T, eg.FLAG_FRONTMOST, device=DEV)
+    losses = torch.full((M,), -9.0, dtype=torch.float32, device=DEV)
+    slopes = torch.zeros(M, dtype=torch.float64, device=DEV)
+    mask = torch.zeros(M, dtype=torch.uint8, device=DEV)
+    sp = int(torch.cuda.current_stream().cuda_stream)
+    hist = np.zeros((M, K), dtype=np.float32)
+    got_masks, fronts = [], []
+    front = 0
+    for c in (fo, full):
+        c.egeria_plasticity_set_lr(0.1)
+    for k in range(K):
+        at, ar = [], []
+        for m, d in enumerate(ds):
+            t, r = wl.make_pair(b, d, "relu", 0.3, seed=1200 + 10 * k + m, device=DEV)
+            at.append(t)
+            ar.append(r)
+            hist[m, k] = oracle.sp_loss(wl.bf16_bits(t), wl.bf16_bits(r))
+        losses.fill_(-9.0)
+        launches = fo.egeria_launch_count()
+        fo.plasticity_evaluate_raw(fo._ptr_array(at, b, True), fo._ptr_array(ar, b, True), b, losses.data_ptr(),
+                                   slopes.data_ptr(), mask.data_ptr(), sp)
+        l1, s1, m1 = full.egeria_plasticity_evaluate(at, ar)
+        got = losses.cpu().numpy()
+        assert fo.egeria_launch_count() == launches + 1            # one kernel, whatever the front
+        if front < M:
+            assert_loss_close(got[front:front + 1], hist[front:front + 1, k].astype(np.float64), f"evaluation {k}")
+            assert np.all(np.delete(got, front) == -9.0)           # only the monitored module was computed
+        else:
+            assert np.all(got == -9.0)
+        assert mask.cpu().numpy().tolist() == m1.cpu().numpy().tolist()
+        got_masks.append(mask.cpu().numpy().tolist())
+        fronts.append(front)
+        front = int(mask.cpu().numpy().sum())
+    ref = oracle.frontmost_replay(hist, W, np.full(M, T))
+    assert ref["frozen"] == M                                      # all frozen within the history ...
+    assert fronts == ref["monitored"].tolist()
+    for k in range(K):
+        want = [int(0 <= ref["freeze_eval"][m] <= k) for m in range(M)]
+        assert got_masks[k] == want, f"evaluation {k}"
+    assert got_masks[-1] == [1] * M                                # ... and an evaluation then only reports
+    fo.check_device_status()
+    # the learning rate falls tenfold: everything restarts, the device goes back to module 0
+    fo.egeria_plasticity_set_lr(0.01)
+    for k in range(3):
+        losses.fill_(-9.0)
+        fo.plasticity_evaluate_raw(fo._ptr_array(at, b, True), fo._ptr_array(ar, b, True), b, losses.data_ptr(),
+                                   slopes.data_ptr(), mask.data_ptr(), sp)
+        got = losses.cpu().numpy()
+        if k == 0:
+            assert np.all(got == -9.0) and mask.cpu().numpy().tolist() == [0] * M    # the restart itself
+        else:
+            assert got[0] > 0 and np.all(got[1:] == -9.0)
+    assert fo.egeria_plasticity_restarts() == 1
+    fo.check_device_status()
+    fo.close()
+    full.close()
+    # a module that cannot take the tensor-core kernel is refused, as is the subset form
+    bad = eg.Context([4096, 1001], b, W, T, eg.FLAG_FRONTMOST | eg.FLAG_FRONT_ONLY, device=DEV)
+    pair = [wl.make_pair(b, d, "relu", 0.3, seed=5, device=DEV) for d in (4096, 1001)]
+    with pytest.raises(eg.EgeriaError) as e:
+        bad.egeria_plasticity_evaluate([p[0] for p in pair], [p[1] for p in pair])
+    assert e.value.status == eg.ERR_UNSUPPORTED_SHAPE
+    bad.close()
+    with pytest.raises(eg.EgeriaError) as e:
+        eg.Context([4096], b, W, T, eg.FLAG_FRONT_ONLY, device=DEV)       # needs the frontmost policy
+    assert e.value.status == eg.ERR_INVALID_ARG
+
+
 def test_bootstrap_detector_matches_oracle():
     rng = np.random.default_rng(11)
     H, W = 120, 8
