@@ -751,6 +751,12 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         tp.ctr = sets + (size_t)set * ctx->M;
         tp.ctr_next = sets + (size_t)(set ^ 1u) * ctx->M;
         tp.M = ctx->M;
+        tp.n_active = 0;
+        if (front_only) {
+            tp.n_active = 1;
+        } else {
+            for (int m = 0; m < ctx->M; ++m) tp.n_active += (P.sides[2 * (size_t)m].tensor_core && P.sides[2 * (size_t)m].module_units > 0);
+        }
         tp.fin = fc;
         const bool log_it = !ctx->calibrated && ctx->host_log && ctx->calib_enqueued < kCalibLaunches &&
                             P.all_ctas_busy_tc;
@@ -1222,6 +1228,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         tp.test_stall = 0;
         tp.wait_limit_ns = kWaitLimitNs;
         tp.M = 1;
+        tp.n_active = 1;
         tp.fin = fc;
         if (launch_tc_mode(P.mode, kStaticCtas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
     } else {

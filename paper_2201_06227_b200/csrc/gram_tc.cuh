@@ -86,6 +86,7 @@ struct TcParams {
     uint32_t test_stall;
     uint64_t wait_limit_ns;    // limit of every bounded wait of this launch (kWaitLimitNs, shorter for the hook)
     int32_t M;
+    int32_t n_active;          // tensor-core modules this launch evaluates (front-only: 1)
     FinCommon fin;             // slots, sides, b, outputs, freezing-rule state
 };
 
@@ -551,7 +552,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             // hand to the one with the most rows left.
             // (With fewer rows in all than half the epilogue warps of the grid there is nothing to
             // lend a hand with, and the look itself would be the last thing the kernel waits for.)
-            const int help_rounds = (2 * (int64_t)b * p.M < (int64_t)gridDim.x * kEpiWarps) ? 0 : 3;
+            const int help_rounds = (2 * (int64_t)b * p.n_active < (int64_t)gridDim.x * kEpiWarps) ? 0 : 3;
             for (int round = 0; round < help_rounds; ++round) {
                 int best_left = 0, best_m = -1;
                 for (int mm = lane; mm < p.M; mm += 32) {
