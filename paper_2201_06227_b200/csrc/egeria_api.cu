@@ -138,6 +138,22 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
+typedef CUresult (*ReplaceAddressFn)(CUtensorMap *, void *);
+
+// A work split as built for one (b, kind of evaluation, split weights, which modules take which
+// kernel): it does not depend on where the activations are, so a caller whose buffers move from
+// call to call gets it from here instead of having it rebuilt.
+struct BuiltPlan {
+    int b = -1;
+    bool front_only = false;
+    int weights_version = -1;
+    std::vector<uint8_t> tc_ok;
+    Plan plan;
+    std::vector<int32_t> front_cta_begin;
+    uint64_t last_use = 0;
+};
+constexpr int kBuiltPlans = 4;
+
 }  // namespace egeria
 
 using namespace egeria;
@@ -153,7 +169,14 @@ struct egeria_ctx {
     Layout L{};
     int n_ctas = 0;
     EncodeTiledFn encode = nullptr;
+    ReplaceAddressFn replace_address = nullptr;  // may be missing: then every map is encoded afresh
     bool attrs_set = false;
+    BuiltPlan built[kBuiltPlans];
+    // Tensor maps of every (module, side) for tmpl_b rows, encoded once; a new pointer set copies
+    // them and only swaps the address in.
+    std::vector<CUtensorMap> tmpl;
+    std::vector<uint8_t> tmpl_valid;
+    int tmpl_b = -1;
     // device-side plans, least recently used one is replaced
     struct PlanEntry {
         int b = -1;
@@ -327,6 +350,12 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
         return EGERIA_ERR_CUDA;
     }
     ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapReplaceAddress", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess && fn)
+        ctx->replace_address = reinterpret_cast<ReplaceAddressFn>(fn);
+    else
+        (void)cudaGetLastError();
 
     if (flags & EGERIA_FLAG_HOST_STAGING) {
         size_t off = L.staging;  // same walk as make_layout
@@ -476,6 +505,47 @@ static void poll_calibration(egeria_ctx *ctx) {
     if (ctx->calib_round >= kCalibRounds) ctx->calibrated = true;
 }
 
+// The work split for b rows: all evaluated modules in one split, or (front-only) one split per
+// possible front, each with module f alone over all CTAs, their units concatenated (slots are
+// numbered from 0 in each: only one of them runs in a launch).
+static egeria_status build_split(egeria_ctx *ctx, int b, bool front_only, const std::vector<uint8_t> &tc_ok,
+                                 const float *weights, BuiltPlan &out) {
+    const int M = ctx->M;
+    out.front_cta_begin.clear();
+    if (!front_only) {
+        build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), out.plan, weights);
+        return EGERIA_OK;
+    }
+    for (int m = 0; m < M; ++m)
+        if (tc_ok[m] != 1) return EGERIA_ERR_UNSUPPORTED_SHAPE;
+    Plan &all = out.plan;
+    all = Plan{};
+    all.mode = mode_of_b(b);
+    all.n_ctas = ctx->n_ctas;
+    all.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, {0, 0}});
+    all.all_ctas_busy_tc = true;
+    out.front_cta_begin.assign((size_t)M * (kMaxCtas + 1), 0);
+    std::vector<uint8_t> only(M);
+    Plan one;
+    for (int f = 0; f < M; ++f) {
+        for (int m = 0; m < M; ++m) only[m] = (m == f) ? 1 : 2;
+        build_plan(M, ctx->d.data(), b, ctx->n_ctas, only.data(), one, weights);
+        const int32_t base = (int32_t)all.units.size();
+        all.units.insert(all.units.end(), one.units.begin(), one.units.end());
+        for (int c = 0; c <= ctx->n_ctas; ++c)
+            out.front_cta_begin[(size_t)f * (kMaxCtas + 1) + c] = base + one.cta_begin_tc[c];
+        all.sides[2 * (size_t)f] = one.sides[2 * (size_t)f];
+        all.sides[2 * (size_t)f + 1] = one.sides[2 * (size_t)f + 1];
+        all.all_ctas_busy_tc = all.all_ctas_busy_tc && one.all_ctas_busy_tc;
+        if ((size_t)one.units.size() * slot_floats_of_mode(one.mode) * sizeof(float) > ctx->L.slot_bytes_cap)
+            return EGERIA_ERR_WORKSPACE;
+    }
+    all.n_units_tc = (int)all.units.size();
+    all.cta_begin_tc.assign(ctx->n_ctas + 1, 0);
+    all.cta_begin_simt.assign(ctx->n_ctas + 1, 0);
+    return EGERIA_OK;
+}
+
 // Select (or build and upload) the device-side plan for this (b, pointers).
 static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const void *const *At, const void *const *Ar,
                                   int b, bool front_only) {
@@ -508,40 +578,31 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
         tc_ok[m] = (aligned && !(ctx->flags & EGERIA_FLAG_FORCE_SIMT)) ? 1 : 0;
     }
     const float *weights = ctx->weights_version > 0 ? ctx->weights.data() : nullptr;
-    std::vector<int32_t> front_cta_begin;  // front-only: [M][kMaxCtas + 1] into the concatenated units
-    if (!front_only) {
-        build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), e.plan, weights);
-    } else {
-        // One split per possible front: module f alone over all CTAs.  Slots are numbered from 0 in
-        // each (only one of them runs in a launch).
-        for (int m = 0; m < M; ++m)
-            if (tc_ok[m] != 1) return EGERIA_ERR_UNSUPPORTED_SHAPE;
-        Plan &all = e.plan;
-        all = Plan{};
-        all.mode = mode_of_b(b);
-        all.n_ctas = ctx->n_ctas;
-        all.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, {0, 0}});
-        all.all_ctas_busy_tc = true;
-        front_cta_begin.assign((size_t)M * (kMaxCtas + 1), 0);
-        std::vector<uint8_t> only(M);
-        Plan one;
-        for (int f = 0; f < M; ++f) {
-            for (int m = 0; m < M; ++m) only[m] = (m == f) ? 1 : 2;
-            build_plan(M, ctx->d.data(), b, ctx->n_ctas, only.data(), one, weights);
-            const int32_t base = (int32_t)all.units.size();
-            all.units.insert(all.units.end(), one.units.begin(), one.units.end());
-            for (int c = 0; c <= ctx->n_ctas; ++c)
-                front_cta_begin[(size_t)f * (kMaxCtas + 1) + c] = base + one.cta_begin_tc[c];
-            all.sides[2 * (size_t)f] = one.sides[2 * (size_t)f];
-            all.sides[2 * (size_t)f + 1] = one.sides[2 * (size_t)f + 1];
-            all.all_ctas_busy_tc = all.all_ctas_busy_tc && one.all_ctas_busy_tc;
-            if ((size_t)one.units.size() * slot_floats_of_mode(one.mode) * sizeof(float) > ctx->L.slot_bytes_cap)
-                return EGERIA_ERR_WORKSPACE;
+    BuiltPlan *bp = nullptr;
+    {
+        int oldest = 0;
+        for (int i = 0; i < kBuiltPlans; ++i) {
+            BuiltPlan &c = ctx->built[i];
+            if (c.b == b && c.front_only == front_only && c.weights_version == ctx->weights_version && c.tc_ok == tc_ok) {
+                bp = &c;
+                break;
+            }
+            if (c.last_use < ctx->built[oldest].last_use) oldest = i;
         }
-        all.n_units_tc = (int)all.units.size();
-        all.cta_begin_tc.assign(ctx->n_ctas + 1, 0);
-        all.cta_begin_simt.assign(ctx->n_ctas + 1, 0);
+        if (!bp) {
+            bp = &ctx->built[oldest];
+            bp->b = -1;
+            egeria_status bs = build_split(ctx, b, front_only, tc_ok, weights, *bp);
+            if (bs != EGERIA_OK) return bs;
+            bp->b = b;
+            bp->front_only = front_only;
+            bp->weights_version = ctx->weights_version;
+            bp->tc_ok = tc_ok;
+        }
+        bp->last_use = ++ctx->use_clock;
     }
+    e.plan = bp->plan;
+    const std::vector<int32_t> &front_cta_begin = bp->front_cta_begin;
     const Plan &P = e.plan;
     const Layout &L = ctx->L;
     if ((!front_only && (size_t)P.units.size() * slot_floats_of_mode(P.mode) * sizeof(float) > L.slot_bytes_cap) ||
@@ -566,12 +627,27 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
     const int box_rows = pitch_of_mode(P.mode);  // rows of one TMA box: all rows of one side
     CUtensorMap *maps = reinterpret_cast<CUtensorMap *>(img + L.tmaps);
     ModulePtrs *mods = reinterpret_cast<ModulePtrs *>(img + L.modules);
+    if (ctx->tmpl_b != b) {  // the maps kept as templates are for another batch size
+        ctx->tmpl.assign(2 * (size_t)M, CUtensorMap{});
+        ctx->tmpl_valid.assign(2 * (size_t)M, 0);
+        ctx->tmpl_b = b;
+    }
     for (int m = 0; m < M; ++m) {
         mods[m] = ModulePtrs{At[m], Ar[m], ctx->d[m]};
         if (tc_ok[m] != 1) continue;
-        egeria_status s = encode_map(ctx, &maps[2 * m], At[m], b, ctx->d[m], box_rows);
-        if (s == EGERIA_OK) s = encode_map(ctx, &maps[2 * m + 1], Ar[m], b, ctx->d[m], box_rows);
-        if (s != EGERIA_OK) return s;
+        const void *base[2] = {At[m], Ar[m]};
+        for (int side = 0; side < 2; ++side) {
+            const size_t k = 2 * (size_t)m + side;
+            if (ctx->replace_address && ctx->tmpl_valid[k]) {
+                // same shape, new place: copy the map and swap the address in (no re-encoding)
+                maps[k] = ctx->tmpl[k];
+                if (ctx->replace_address(&maps[k], const_cast<void *>(base[side])) == CUDA_SUCCESS) continue;
+            }
+            egeria_status s = encode_map(ctx, &maps[k], base[side], b, ctx->d[m], box_rows);
+            if (s != EGERIA_OK) return s;
+            ctx->tmpl[k] = maps[k];
+            ctx->tmpl_valid[k] = 1;
+        }
     }
     if (!P.units.empty()) memcpy(img + L.units, P.units.data(), P.units.size() * sizeof(Unit));
     if (front_only)
