@@ -341,6 +341,14 @@ egeria_status egeria_debug_plan_weighted(int M, const int64_t *d, int b, int n_c
                                          const float *weights, int32_t *out_units, int max_units,
                                          int *n_units);
 
+/* Test hook: the help planned for the end of a launch, pure host arithmetic.  The rows of a
+ * module are finished by the warps of the thread blocks that worked on it, so a module that got
+ * few blocks has many rows per warp; some warps of the blocks of the well-off modules are told to
+ * start with such a module's rows instead.  Writes, for every CTA c < n_ctas, out_help[2 c] = the
+ * module it lends warps to (-1: none) and out_help[2 c + 1] = how many of its twelve epilogue
+ * warps. */
+egeria_status egeria_debug_plan_help(int M, const int64_t *d, int b, int n_ctas, int32_t *out_help);
+
 /* Test hook for the bounded waits: the NEXT evaluation kernel of this context (tensor-core
  * modules) runs with every wait limited to one millisecond instead of two seconds, and with one
  * hand-shake of its first thread block left out on purpose, so that the waits that depend on it

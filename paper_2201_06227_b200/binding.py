@@ -32,7 +32,7 @@ EXPORTS = [
     "egeria_split_weights", "egeria_status_string", "egeria_bootstrap_step", "egeria_bootstrap_replay",
     "egeria_bootstrap_reset", "egeria_plasticity_state_bytes", "egeria_plasticity_export", "egeria_plasticity_import",
     "egeria_sp_loss_subset", "egeria_plasticity_evaluate_subset",
-    "egeria_sp_loss_static_status", "egeria_debug_stall_next", "egeria_plasticity_set_lr", "egeria_plasticity_restarts", "egeria_plasticity_replay_lr",
+    "egeria_sp_loss_static_status", "egeria_debug_stall_next", "egeria_debug_plan_help", "egeria_plasticity_set_lr", "egeria_plasticity_restarts", "egeria_plasticity_replay_lr",
 ]
 
 
@@ -94,6 +94,7 @@ def lib() -> ctypes.CDLL:
     L.egeria_sp_loss_static.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_int64, vp]
     L.egeria_sp_loss_static_status.argtypes = []
     L.egeria_debug_stall_next.argtypes = [vp, ctypes.c_int]
+    L.egeria_debug_plan_help.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int32)]
     L.egeria_launch_count.argtypes = [vp]
     L.egeria_launch_count.restype = ctypes.c_int64
     L.egeria_status_string.argtypes = [ctypes.c_int]
@@ -136,6 +137,15 @@ def egeria_debug_plan(d: Sequence[int], b: int, n_ctas: int) -> np.ndarray:
                                  out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), cap, ctypes.byref(n))
     _check(st, "egeria_debug_plan")
     return out[: n.value].copy()
+
+
+def egeria_debug_plan_help(d: Sequence[int], b: int, n_ctas: int) -> np.ndarray:
+    """Rows {module helped (-1: none), warps lent} per CTA: the help planned for the end of a launch."""
+    out = np.zeros((n_ctas, 2), dtype=np.int32)
+    st = lib().egeria_debug_plan_help(len(d), _i64(d), int(b), int(n_ctas),
+                                      out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)))
+    _check(st, "egeria_debug_plan_help")
+    return out
 
 
 def egeria_debug_plan_weighted(d: Sequence[int], b: int, n_ctas: int, weights) -> np.ndarray:

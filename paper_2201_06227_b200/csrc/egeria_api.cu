@@ -39,7 +39,7 @@ struct Layout {
     // Device-side plans (tensor maps, pointers, unit table, per-CTA ranges, slot ranges): kPlanSlots
     // regions of plan_stride bytes from plan0; the offsets below are relative to a region.
     size_t plan0, plan_stride;
-    size_t tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides;
+    size_t tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides, cta_help;
 };
 
 // Units of one device-side plan: all modules in one split, or (front-only contexts) one split per
@@ -75,6 +75,7 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
         L.cta_begin_tc = take((size_t)((flags & EGERIA_FLAG_FRONT_ONLY) ? M : 1) * (kMaxCtas + 1) * sizeof(int32_t));
         L.cta_begin_simt = take((kMaxCtas + 1) * sizeof(int32_t));
         L.sides = take((size_t)2 * M * sizeof(SideInfo));
+        L.cta_help = take((size_t)kMaxCtas * sizeof(CtaHelp));
         L.plan_stride = off;
         off = saved;
         L.plan0 = take(L.plan_stride * kPlanSlots);
@@ -307,6 +308,21 @@ egeria_status egeria_debug_plan_weighted(int M, const int64_t *d, int b, int n_c
         row[2] = u.kb0;
         row[3] = u.nkb;
         row[4] = u.cta;
+    }
+    return EGERIA_OK;
+}
+
+egeria_status egeria_debug_plan_help(int M, const int64_t *d, int b, int n_ctas, int32_t *out_help) {
+    if (!out_help || n_ctas < 1) return EGERIA_ERR_INVALID_ARG;
+    egeria_status s = check_shapes(M, d, b, 1);
+    if (s != EGERIA_OK) return s;
+    std::vector<uint8_t> tc_ok(M);
+    for (int m = 0; m < M; ++m) tc_ok[m] = (d[m] % 8 == 0);
+    Plan plan;
+    build_plan(M, d, b, n_ctas, tc_ok.data(), plan, nullptr);
+    for (int c = 0; c < n_ctas; ++c) {
+        out_help[2 * c] = plan.cta_help[c].module;
+        out_help[2 * c + 1] = plan.cta_help[c].warps;
     }
     return EGERIA_OK;
 }
@@ -656,6 +672,8 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
         memcpy(img + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t));
     memcpy(img + L.cta_begin_simt, P.cta_begin_simt.data(), P.cta_begin_simt.size() * sizeof(int32_t));
     memcpy(img + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo));
+    if (!front_only && !P.cta_help.empty())  // (the image is zeroed: no help planned otherwise)
+        memcpy(img + L.cta_help, P.cta_help.data(), P.cta_help.size() * sizeof(CtaHelp));
     // From pageable memory the runtime stages the bytes before returning, so `pack` may be reused.
     EG_CUDA(cudaMemcpyAsync(ctx->plan_region(lru), img, L.plan_stride, cudaMemcpyHostToDevice, stream));
     if (ctx->pinned_plans) {
@@ -818,6 +836,7 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         tp.tmaps = reinterpret_cast<const CUtensorMap *>(region + L.tmaps);
         tp.units = reinterpret_cast<const Unit *>(region + L.units);
         tp.cta_begin = reinterpret_cast<const int32_t *>(region + L.cta_begin_tc);
+        tp.cta_help = front_only ? nullptr : reinterpret_cast<const CtaHelp *>(region + L.cta_help);
         tp.front_word = front_only ? ctx->slope_state().front : nullptr;
         tp.cta_stride = kMaxCtas + 1;
         tp.slots = ctx->at<float>(L.slots);
@@ -1293,6 +1312,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         tp.tmaps = reinterpret_cast<const CUtensorMap *>(ws + L.tmaps);
         tp.units = reinterpret_cast<const Unit *>(ws + L.units);
         tp.cta_begin = reinterpret_cast<const int32_t *>(ws + L.cta_begin_tc);
+        tp.cta_help = nullptr;
         tp.front_word = nullptr;
         tp.cta_stride = 0;
         tp.slots = reinterpret_cast<float *>(ws + L.slots);

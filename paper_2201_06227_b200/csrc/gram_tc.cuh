@@ -67,6 +67,7 @@ struct TcParams {
     const CUtensorMap *tmaps;  // [2 * M]: A_T and A_R of every module (device memory)
     const Unit *units;         // tensor-core units
     const int32_t *cta_begin;  // [gridDim.x + 1]
+    const CtaHelp *cta_help;   // [gridDim.x] planned help at the end of the launch, or nullptr
     // Front-only evaluation (else nullptr): the word that holds the number of frozen modules; the
     // work split of front f starts at cta_begin + f * cta_stride, and with every module frozen
     // there is no work.
@@ -433,6 +434,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         const int part = (warp - 2) >> 2;  // which third of the quarter's columns this warp drains
         const int b = p.fin.b;
         const bool epi_leader = (threadIdx.x == 64);
+        // asked for now, needed at the end of the launch
+        const CtaHelp planned_help = p.cta_help ? p.cta_help[blockIdx.x] : CtaHelp{-1, 0};
         uint32_t acc = 0, acc_phase = 0;
         bool aborted = false;
         for (int ui = u_begin; ui < u_end; ++ui) {
@@ -500,6 +503,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             static_assert(kEpiWarps * kFinStageBytes <= Cfg::kStages * Cfg::kStageBytes, "ring too small to stage");
             float *stage = reinterpret_cast<float *>(smem_aligned + (warp - 2) * kFinStageBytes);
             ptx::fence_proxy_async();  // the ring was last touched by TMA and the tensor cores
+            // Planned help first: the last few warps of a CTA whose own module has warps to spare
+            // start with the rows of a module that is short of them (see CtaHelp), once that module
+            // is complete; the wait for it is a courtesy like the others.
+            {
+                const CtaHelp h = planned_help;
+                if (h.warps > 0 && warp - 2 >= kEpiWarps - h.warps) {
+                    const int total = p.fin.sides[2 * h.module].module_units;
+                    const uint64_t t_wait = ptx::globaltimer_ns();
+                    int state = 0;  // 1 complete, 2 gave up
+                    while (state == 0) {
+                        if (lane == 0) {
+                            if (detail::ld_acquire(&p.ctr[h.module].units_done) >= total)
+                                state = 1;
+                            else if (*abort_flag || ptx::globaltimer_ns() - t_wait > kHelpWaitNs)
+                                state = 2;
+                        }
+                        state = __shfl_sync(0xffffffffu, state, 0);
+                        if (state == 0) __nanosleep(100);
+                    }
+                    if (state == 1) {
+                        __threadfence();
+                        detail::finish_module_rows<Cfg::kNC>(p, h.module, lane, stage);
+                    }
+                }
+            }
             // The modules this CTA worked on, 32 units at a time: lane j looks after the module of
             // unit j (the first unit of each module only; a module's units are adjacent).  The warp
             // polls their counters together, finishes rows wherever a module is complete and has

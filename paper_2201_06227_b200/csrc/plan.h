@@ -70,6 +70,16 @@ struct CtaLog {
     uint32_t pad;
 };
 
+// End-of-launch help, planned on the host.  The rows of a module are finished by the warps of the
+// CTAs that worked on it; a module that got few CTAs (a small one) has many rows per warp, a big
+// one less than one.  So some warps of the CTAs of big modules are told to start with a small
+// module's rows instead: `warps` of this CTA's epilogue warps (the last ones) first help `module`
+// (-1, 0: nobody).
+struct CtaHelp {
+    int32_t module;
+    int32_t warps;
+};
+
 // Progress counters of one module inside the tensor-core kernel (zero before a launch).  Each
 // is polled or bumped by many CTAs at the end of a launch, so each has a 128-byte line of its own.
 struct FinCounters {
@@ -98,6 +108,7 @@ struct Plan {
     std::vector<int32_t> cta_begin_tc;    // [n_ctas + 1] into units[0 .. n_units_tc)
     std::vector<int32_t> cta_begin_simt;  // [n_ctas + 1] into units[n_units_tc ..), relative to 0
     std::vector<SideInfo> sides;    // [2 * M]
+    std::vector<CtaHelp> cta_help;  // [n_ctas] which module some warps of the CTA lend a hand to first
 };
 
 inline int64_t kblocks_of(int64_t d) { return (d + kKBlock - 1) / kKBlock; }
@@ -182,13 +193,76 @@ inline void split_tiles(const std::vector<Tile> &tiles, int n_ctas, int slot0, s
     }
     cta_begin[n_ctas] = (int)units.size() - base;
 }
+// Who lends a hand to whom at the end of a launch (CtaHelp).  A CTA's warps are credited to the
+// modules it worked on in proportion to its blocks there; a module's need is its b rows at the
+// launch's average rows per warp.  CTAs whose main module has more warps than it needs give the
+// surplus share of their warps (at most two thirds) to the module that lacks the most at that
+// point.  Nothing is planned when no module has more than 1.5 times the average rows per warp.
+inline void plan_help(Plan &plan, int M, int b, int warps_per_cta) {
+    const int n_ctas = plan.n_ctas;
+    plan.cta_help.assign(n_ctas, CtaHelp{-1, 0});
+    std::vector<double> have(M, 0.0);
+    std::vector<int> main_module(n_ctas, -1);
+    for (int c = 0; c < n_ctas; ++c) {
+        const int u0 = plan.cta_begin_tc[c], u1 = plan.cta_begin_tc[c + 1];
+        int64_t blocks = 0, best = 0;
+        for (int u = u0; u < u1; ++u) blocks += plan.units[u].nkb;
+        std::vector<int64_t> per;  // blocks per module, in unit order (few entries)
+        std::vector<int> mods;
+        for (int u = u0; u < u1; ++u) {
+            const int m = plan.units[u].module;
+            if (mods.empty() || mods.back() != m) {
+                mods.push_back(m);
+                per.push_back(0);
+            }
+            per.back() += plan.units[u].nkb;
+        }
+        for (size_t k = 0; k < mods.size(); ++k) {
+            have[mods[k]] += (double)warps_per_cta * (double)per[k] / (double)blocks;
+            if (per[k] > best) {
+                best = per[k];
+                main_module[c] = mods[k];
+            }
+        }
+    }
+    double rows = 0.0, warps = 0.0;
+    for (int m = 0; m < M; ++m)
+        if (have[m] > 0.0) {
+            rows += b;
+            warps += have[m];
+        }
+    if (warps <= 0.0) return;
+    const double rho = rows / warps;  // rows per warp if every warp took its share
+    std::vector<double> lack(M, 0.0);
+    bool worth = false;
+    for (int m = 0; m < M; ++m) {
+        if (have[m] <= 0.0) continue;
+        lack[m] = b / rho - have[m];  // warps the module is short of (negative: it has some to spare)
+        if (b / have[m] > 1.5 * rho && b / have[m] > 1.5) worth = true;
+    }
+    if (!worth) return;
+    for (int c = 0; c < n_ctas; ++c) {
+        const int mm = main_module[c];
+        if (mm < 0 || lack[mm] >= 0.0) continue;
+        int give = (int)(warps_per_cta * (-lack[mm]) / have[mm]);
+        const int cap = 2 * warps_per_cta / 3;
+        if (give > cap) give = cap;
+        if (give < 1) continue;
+        int to = -1;
+        for (int m = 0; m < M; ++m)
+            if (lack[m] > 0.5 && (to < 0 || lack[m] > lack[to])) to = m;
+        if (to < 0) break;
+        plan.cta_help[c] = CtaHelp{to, give};
+        lack[to] -= give;
+    }
+}
 }  // namespace detail
 
 // tc_ok[m]: 1 = module m takes the TMA + tcgen05 kernel, 0 = the CUDA-core kernel, 2 = module m
 // is not evaluated in this plan (no units, never finished).  weights: see split_tiles (applies
 // to the tensor-core split only).
 inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t *tc_ok, Plan &plan,
-                       const float *weights = nullptr) {
+                       const float *weights = nullptr, int warps_per_cta = 12) {
     plan.mode = mode_of_b(b);
     plan.n_ctas = n_ctas;
     plan.units.clear();
@@ -227,6 +301,7 @@ inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t
         t.tensor_core = r.tensor_core = (tc_ok[m] == 1) ? 1 : 0;
         t.module_units = r.module_units = units;
     }
+    detail::plan_help(plan, M, b, warps_per_cta);
 }
 
 }  // namespace egeria

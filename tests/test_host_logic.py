@@ -208,3 +208,32 @@ def test_plan_rejects_bad_arguments():
     assert L.egeria_debug_plan(1, eg._i64([8]), 8, 0, p, 4, ctypes.byref(n)) == eg.ERR_INVALID_ARG
     assert L.egeria_debug_plan(1, eg._i64([8]), 400, 4, p, 4, ctypes.byref(n)) == eg.ERR_UNSUPPORTED_SHAPE
     assert L.egeria_debug_plan(1, eg._i64([8]), 8, 4, None, 4, ctypes.byref(n)) == eg.ERR_INVALID_ARG
+
+
+def test_planned_help_goes_from_well_off_modules_to_needy_ones():
+    """End-of-launch help (CtaHelp): CTAs whose module has more warps than rows to do lend some to
+    the modules that have many rows per warp; balanced workloads plan none."""
+    for name in ("bert_base", "gpt2_medium", "tiny"):
+        w = wl.WORKLOADS[name]
+        assert not (eg.egeria_debug_plan_help(list(w.d), w.b, 148)[:, 1] > 0).any(), name
+    w = wl.WORKLOADS["resnet56"]
+    d, n = list(w.d), 148
+    units = eg.egeria_debug_plan(d, w.b, n)
+    help_ = eg.egeria_debug_plan_help(d, w.b, n)
+    blocks = np.zeros((n, len(d)))
+    for m, _, _, nkb, c in units:
+        blocks[c, m] += nkb
+    have = (12.0 * blocks / blocks.sum(axis=1, keepdims=True)).sum(axis=0)      # warps credited to each module
+    rows_per_warp = w.b / have
+    donors = np.nonzero(help_[:, 1] > 0)[0]
+    assert len(donors) > 20
+    assert np.all(help_[donors, 1] <= 8) and np.all(help_[help_[:, 1] == 0, 0] == -1)
+    avg = w.b * len(d) / have.sum()
+    for c in donors:
+        own = int(np.argmax(blocks[c]))
+        assert rows_per_warp[own] < avg < rows_per_warp[help_[c, 0]]         # from the well-off to the needy
+    got = np.bincount(help_[donors, 0], weights=help_[donors, 1], minlength=len(d))
+    after = w.b / (have + got - np.bincount([int(np.argmax(blocks[c])) for c in donors],
+                                            weights=help_[donors, 1], minlength=len(d)))
+    assert after.max() < 0.6 * rows_per_warp.max()                             # the worst module is much better off
+    assert after.max() / after.min() < 1.6
