@@ -18,7 +18,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libegeria.so"
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 FLAG_SIGNED_SLOPE, FLAG_FORCE_SIMT, FLAG_KEEP_GRAMS, FLAG_HOST_STAGING, FLAG_TIME_GRAM = 1, 2, 4, 8, 16
-FLAG_EQUAL_SPLIT, FLAG_AUTO_T, FLAG_FRONTMOST, FLAG_FRONT_ONLY = 32, 64, 128, 256
+FLAG_EQUAL_SPLIT, FLAG_AUTO_T, FLAG_FRONTMOST, FLAG_FRONT_ONLY, FLAG_OVERLAP = 32, 64, 128, 256, 512
 MAX_B = 256
 WORKSPACE_ALIGN = 1024
 

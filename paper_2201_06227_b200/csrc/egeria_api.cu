@@ -702,22 +702,32 @@ static cudaError_t launch_finalize(const FinParams &fp, int M, int b, cudaStream
     return cudaGetLastError();
 }
 
-static cudaError_t launch_tc_mode(int mode, int n_ctas, cudaStream_t stream, const TcParams &tp) {
+// Launched as a programmatic dependent of whatever kernel precedes it in the stream: if that is an
+// evaluation kernel of this library (which says early that its dependents may start), this launch
+// begins while that one is finishing; after any other kernel nothing changes.
+template <int MODE>
+static cudaError_t launch_tc(int n_ctas, cudaStream_t stream, const TcParams &tp, bool overlap) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_ctas);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = TcCfg<MODE>::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, gram_tc_kernel<MODE>, tp);
+}
+
+// overlap: EGERIA_FLAG_OVERLAP (the caller's promise about the inputs; see egeria.h).
+static cudaError_t launch_tc_mode(int mode, int n_ctas, cudaStream_t stream, const TcParams &tp, bool overlap = false) {
     switch (mode) {
-        case kStacked32:
-            gram_tc_kernel<kStacked32><<<n_ctas, kTcThreads, TcCfg<kStacked32>::kSmemBytes, stream>>>(tp);
-            break;
-        case kStacked64:
-            gram_tc_kernel<kStacked64><<<n_ctas, kTcThreads, TcCfg<kStacked64>::kSmemBytes, stream>>>(tp);
-            break;
-        case kSingle1:
-            gram_tc_kernel<kSingle1><<<n_ctas, kTcThreads, TcCfg<kSingle1>::kSmemBytes, stream>>>(tp);
-            break;
-        default:
-            gram_tc_kernel<kSingle2><<<n_ctas, kTcThreads, TcCfg<kSingle2>::kSmemBytes, stream>>>(tp);
-            break;
+        case kStacked32: return launch_tc<kStacked32>(n_ctas, stream, tp, overlap);
+        case kStacked64: return launch_tc<kStacked64>(n_ctas, stream, tp, overlap);
+        case kSingle1: return launch_tc<kSingle1>(n_ctas, stream, tp, overlap);
+        default: return launch_tc<kSingle2>(n_ctas, stream, tp, overlap);
     }
-    return cudaGetLastError();
 }
 
 static cudaError_t set_tc_attrs() {
@@ -860,7 +870,8 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         tp.test_stall = ctx->stall_next;
         tp.wait_limit_ns = ctx->stall_next ? kTestWaitLimitNs : kWaitLimitNs;
         ctx->stall_next = 0;
-        if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
+        if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp, (ctx->flags & EGERIA_FLAG_OVERLAP) != 0) != cudaSuccess)
+            return EGERIA_ERR_CUDA;
         if (log_it) {
             const int k = ctx->calib_enqueued;
             EG_CUDA(cudaMemcpyAsync(ctx->host_log + (size_t)k * kMaxCtas, tp.log, (size_t)ctx->n_ctas * sizeof(CtaLog),

@@ -26,6 +26,13 @@
 // and split its columns.
 // Every wait is bounded; on expiry the CTA raises its abort flag, records
 // EGERIA_ERR_TIMEOUT in the status word, drains what is in flight and returns.
+//
+// Back-to-back evaluations overlap (programmatic dependent launch): the activations are inputs
+// that no evaluation writes, so a CTA of the next launch may start streaming on an SM as soon as
+// this launch's CTA there has ended, while other CTAs of this launch are still finishing their
+// modules.  Everything the launches share -- partial slots, progress counters, the rule's state,
+// the outputs, the status word, the log -- is touched only after grid_dependency_wait(), i.e. once
+// the launch before has ended entirely.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -241,6 +248,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     {
         const int32_t *cta_begin = p.cta_begin;
         if (p.front_word) {
+            ptx::grid_dependency_wait();
             const int front = (int)(uint32_t)*reinterpret_cast<const volatile unsigned long long *>(p.front_word);
             all_frozen = (front >= p.M);
             cta_begin += (int64_t)(all_frozen ? 0 : front) * p.cta_stride;
@@ -251,12 +259,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         }
     }
 
-    // The counters of the next launch start at zero (nobody reads that set during this launch).
-    {
-        int32_t *z = reinterpret_cast<int32_t *>(p.ctr_next);
-        const int n = p.M * (int)(sizeof(FinCounters) / sizeof(int32_t));
-        for (int i = blockIdx.x * kTcThreads + threadIdx.x; i < n; i += gridDim.x * kTcThreads) z[i] = 0;
-    }
+    // The launch after this one may begin (its CTAs get an SM when one of ours ends).  A front-only
+    // launch reads the front the launch before it wrote, so it waits for that one here and now.
+    ptx::grid_launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < Cfg::kStages; ++s) {
@@ -412,6 +417,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 }
             }
             if (p.log) {
+                ptx::grid_dependency_wait();  // the log is shared with the launch before
                 CtaLog e;
                 e.serial = p.serial;
                 e.duration_ns = (uint32_t)(ptx::globaltimer_ns() - t_entry);
@@ -438,6 +444,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         const CtaHelp planned_help = p.cta_help ? p.cta_help[blockIdx.x] : CtaHelp{-1, 0};
         uint32_t acc = 0, acc_phase = 0;
         bool aborted = false;
+        bool prior_done = false;  // the launch before has ended: the shared workspace is ours
+        // Once the launch before has ended: the counters of the NEXT launch start at zero (the set
+        // this launch does not use; the launch before used it until its end).
+        auto claim_workspace = [&]() {
+            if (prior_done) return;
+            ptx::grid_dependency_wait();
+            prior_done = true;
+            int32_t *z = reinterpret_cast<int32_t *>(p.ctr_next);
+            const int n = p.M * (int)(sizeof(FinCounters) / sizeof(int32_t));
+            for (int i = blockIdx.x * kEpiThreads + (threadIdx.x - 64); i < n; i += gridDim.x * kEpiThreads) z[i] = 0;
+        };
         for (int ui = u_begin; ui < u_end; ++ui) {
             const Unit u = p.units[ui];
             const bool got = ptx::mbar_wait_bounded(accfull0 + 8 * acc, acc_phase, abort_flag, p.wait_limit_ns);
@@ -445,6 +462,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 aborted = true;
                 break;
             }
+            claim_workspace();  // the first unit's streaming is over by now; usually so is the launch before
             ptx::tc_fence_after_sync();
             float *slot = p.slots + (int64_t)u.slot * p.fin.slot_floats;
             const uint32_t t_row = tmem_base + acc * Cfg::kAccCols + ((uint32_t)(q * 32) << 16);
@@ -490,6 +508,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             detail::epi_bar_sync();
             if (epi_leader) atomicAdd(&p.ctr[u.module].units_done, 1);
         }
+        claim_workspace();  // (CTAs without a unit, and the counters' clearing if the wait above gave up)
         if (all_frozen && blockIdx.x == 0 && warp == 2) {
             // nothing is monitored any more: the rule only reports (prefix mask of ones, final slopes)
             StepLoaded L = plasticity_step_load(p.fin.st, p.M - 1, lane);
@@ -615,7 +634,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     __syncthreads();
     ptx::tc_fence_after_sync();
     if (warp == 1) ptx::tmem_dealloc(tmem_base, Cfg::kTmemCols);
-    if (threadIdx.x == 0 && *abort_flag) atomicMax(p.status, kStatusTimeout);
+    if (threadIdx.x == 0 && *abort_flag) {
+        ptx::grid_dependency_wait();
+        atomicMax(p.status, kStatusTimeout);
+    }
 }
 
 }  // namespace egeria

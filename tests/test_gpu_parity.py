@@ -428,6 +428,51 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_recovers(kind)
     ctx.close()
 
 
+@pytest.mark.parametrize("b,ds,extra", [(32, [98304] * 6, 0), (128, [16384, 8192, 4096, 4096, 520 * 8], 0),
+                                        (64, [200704, 100352, 8200], 0), (256, [65536, 32768], 0),
+                                        (40, [4096, 2048, 8192, 1024], "front_only")])
+def test_overlapped_evaluations_give_the_same_results(b, ds, extra):
+    """EGERIA_FLAG_OVERLAP: consecutive evaluations overlap on the GPU (the next one streams while
+    the previous one finishes its modules).  Enqueued back to back without any synchronisation,
+    on inputs that alternate between two sets, every evaluation must give bit for bit what the
+    same sequence gives without the flag -- losses, slopes and masks (the rule's state is carried
+    from evaluation to evaluation) -- and the first one must match the oracle."""
+    n_eval, M = 24, len(ds)
+    sets = []
+    for k in range(2):
+        at, ar = [], []
+        for m, d in enumerate(ds):
+            t, r = wl.make_pair(b, d, "relu" if m % 2 else "normal", 0.05 + 0.1 * k + 0.02 * m, seed=8000 + 10 * k + m, device=DEV)
+            at.append(t)
+            ar.append(r)
+        sets.append((at, ar))
+    base = eg.FLAG_EQUAL_SPLIT | ((eg.FLAG_FRONTMOST | eg.FLAG_FRONT_ONLY) if extra == "front_only" else 0)
+    T = 0.5 if extra == "front_only" else 1e-3
+    results = {}
+    for name, flags in (("plain", base), ("overlapped", base | eg.FLAG_OVERLAP)):
+        ctx = eg.Context(ds, b, 3, T, flags, device=DEV)
+        outs = [(torch.full((M,), -1.0, dtype=torch.float32, device=DEV), torch.zeros(M, dtype=torch.float64, device=DEV),
+                 torch.zeros(M, dtype=torch.uint8, device=DEV)) for _ in range(n_eval)]
+        sp = int(torch.cuda.current_stream().cuda_stream)
+        ptrs = [(ctx._ptr_array(at, b, True), ctx._ptr_array(ar, b, True)) for at, ar in sets]
+        for k in range(n_eval):                                  # no synchronisation in between
+            pa, pr = ptrs[k % 2]
+            ctx.plasticity_evaluate_raw(pa, pr, b, outs[k][0].data_ptr(), outs[k][1].data_ptr(), outs[k][2].data_ptr(), sp)
+        torch.cuda.synchronize()
+        ctx.check_device_status()
+        results[name] = [tuple(t.cpu().numpy().copy() for t in o) for o in outs]
+        ctx.close()
+    for k in range(n_eval):
+        for j in range(3):
+            assert results["plain"][k][j].tobytes() == results["overlapped"][k][j].tobytes(), (k, j)
+    if extra != "front_only":
+        ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in sets[0][0]], [wl.bf16_bits(r) for r in sets[0][1]])
+        assert_loss_close(results["overlapped"][0][0], ref)
+        assert results["overlapped"][-1][2].all()                # constant alternating readings: everything froze
+    else:
+        assert results["overlapped"][-1][2].all()
+
+
 def test_changing_b_and_pointers_between_calls():
     ctx = eg.Context([4096, 264], 128, 5, 1e-3, device=DEV)
     for b in (128, 8, 70, 8):
