@@ -108,19 +108,21 @@ enum {
      * beyond reporting the mask.  egeria_sp_loss_batch and the subset calls are not affected
      * (the subset form of the evaluation is refused: EGERIA_ERR_INVALID_ARG). */
     EGERIA_FLAG_FRONT_ONLY = 256u,
-    /* Let consecutive evaluations of this context overlap on the GPU (programmatic dependent
-     * launch): a thread block of the next evaluation starts reading its activations on an SM as
-     * soon as the previous evaluation's block there has ended, while other blocks of the
-     * previous evaluation are still finishing their modules; everything the evaluations share
-     * (workspace, outputs, the rule's state) is touched only after the previous evaluation has
-     * ended entirely, so results are the same.  THE CALLER PROMISES, by setting this flag, that
-     * the activations passed to an evaluation are not written by the KERNEL that precedes that
-     * evaluation in the stream (they were complete before it; e.g. several mini-batches'
-     * activations collected first and evaluated one after the other): the evaluation starts
-     * reading them before that kernel is known to have ended.  (Copies are not kernels: an
-     * evaluation still waits for a copy enqueued before it.)  Without the flag an evaluation
-     * starts when everything before it in the stream has ended, as any kernel does.
-     * Has no effect under EGERIA_FLAG_TIME_GRAM (the timing events keep the kernels apart). */
+    /* Let consecutive evaluations of this context overlap on the GPU.  Every evaluation kernel
+     * is launched as a programmatic dependent of the kernel before it in the stream: its thread
+     * blocks set themselves up while that kernel's last blocks are still running, and then WAIT
+     * for that kernel to have ended before they read an activation or touch the workspace.
+     * With this flag the wait before the first read of the activations is left out: a thread
+     * block of the next evaluation starts streaming on an SM as soon as the previous
+     * evaluation's block there has ended, while other blocks of the previous evaluation are
+     * still finishing their modules; everything the evaluations share (workspace, outputs, the
+     * rule's state) is still touched only after the previous evaluation has ended entirely, so
+     * results are the same.  THE CALLER PROMISES, by setting this flag, that the activations
+     * passed to an evaluation are not written by the KERNEL that precedes that evaluation in
+     * the stream (they were complete before it; e.g. several mini-batches' activations
+     * collected first and evaluated one after the other).  (Copies are not kernels: an
+     * evaluation still waits for a copy enqueued before it.)  Has no effect under
+     * EGERIA_FLAG_TIME_GRAM (the timing events keep the kernels apart). */
     EGERIA_FLAG_OVERLAP = 512u
 };
 

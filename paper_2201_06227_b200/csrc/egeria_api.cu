@@ -702,11 +702,13 @@ static cudaError_t launch_finalize(const FinParams &fp, int M, int b, cudaStream
     return cudaGetLastError();
 }
 
-// Launched as a programmatic dependent of whatever kernel precedes it in the stream: if that is an
-// evaluation kernel of this library (which says early that its dependents may start), this launch
-// begins while that one is finishing; after any other kernel nothing changes.
+// Launched as a programmatic dependent of whatever kernel precedes it in the stream: its CTAs may
+// become resident and set themselves up (barriers, tensor memory, their share of the plan) while
+// that kernel's last CTAs are still running -- an evaluation kernel of this library says so early,
+// any other kernel implicitly as its CTAs end.  The kernel itself waits (griddepcontrol.wait) before
+// it reads an activation or touches anything in the workspace, so nothing is consumed early.
 template <int MODE>
-static cudaError_t launch_tc(int n_ctas, cudaStream_t stream, const TcParams &tp, bool overlap) {
+static cudaError_t launch_tc(int n_ctas, cudaStream_t stream, const TcParams &tp) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_ctas);
     cfg.blockDim = dim3(kTcThreads);
@@ -716,17 +718,16 @@ static cudaError_t launch_tc(int n_ctas, cudaStream_t stream, const TcParams &tp
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = overlap ? 1 : 0;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gram_tc_kernel<MODE>, tp);
 }
 
-// overlap: EGERIA_FLAG_OVERLAP (the caller's promise about the inputs; see egeria.h).
-static cudaError_t launch_tc_mode(int mode, int n_ctas, cudaStream_t stream, const TcParams &tp, bool overlap = false) {
+static cudaError_t launch_tc_mode(int mode, int n_ctas, cudaStream_t stream, const TcParams &tp) {
     switch (mode) {
-        case kStacked32: return launch_tc<kStacked32>(n_ctas, stream, tp, overlap);
-        case kStacked64: return launch_tc<kStacked64>(n_ctas, stream, tp, overlap);
-        case kSingle1: return launch_tc<kSingle1>(n_ctas, stream, tp, overlap);
-        default: return launch_tc<kSingle2>(n_ctas, stream, tp, overlap);
+        case kStacked32: return launch_tc<kStacked32>(n_ctas, stream, tp);
+        case kStacked64: return launch_tc<kStacked64>(n_ctas, stream, tp);
+        case kSingle1: return launch_tc<kSingle1>(n_ctas, stream, tp);
+        default: return launch_tc<kSingle2>(n_ctas, stream, tp);
     }
 }
 
@@ -867,11 +868,11 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
                             P.all_ctas_busy_tc;
         tp.log = log_it ? ctx->at<CtaLog>(L.cta_log) : nullptr;
         tp.serial = ctx->tc_launches + 1;
+        tp.early_inputs = (ctx->flags & EGERIA_FLAG_OVERLAP) ? 1u : 0u;
         tp.test_stall = ctx->stall_next;
         tp.wait_limit_ns = ctx->stall_next ? kTestWaitLimitNs : kWaitLimitNs;
         ctx->stall_next = 0;
-        if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp, (ctx->flags & EGERIA_FLAG_OVERLAP) != 0) != cudaSuccess)
-            return EGERIA_ERR_CUDA;
+        if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
         if (log_it) {
             const int k = ctx->calib_enqueued;
             EG_CUDA(cudaMemcpyAsync(ctx->host_log + (size_t)k * kMaxCtas, tp.log, (size_t)ctx->n_ctas * sizeof(CtaLog),
@@ -1332,6 +1333,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         tp.ctr_next = tp.ctr + 1;
         tp.log = nullptr;
         tp.serial = 0;
+        tp.early_inputs = 0;
         tp.test_stall = 0;
         tp.wait_limit_ns = kWaitLimitNs;
         tp.M = 1;

@@ -27,12 +27,14 @@
 // Every wait is bounded; on expiry the CTA raises its abort flag, records
 // EGERIA_ERR_TIMEOUT in the status word, drains what is in flight and returns.
 //
-// Back-to-back evaluations overlap (programmatic dependent launch): the activations are inputs
-// that no evaluation writes, so a CTA of the next launch may start streaming on an SM as soon as
-// this launch's CTA there has ended, while other CTAs of this launch are still finishing their
-// modules.  Everything the launches share -- partial slots, progress counters, the rule's state,
-// the outputs, the status word, the log -- is touched only after grid_dependency_wait(), i.e. once
-// the launch before has ended entirely.
+// The kernel is launched as a programmatic dependent of the kernel before it in the stream: a CTA
+// gets an SM as soon as that kernel's CTA there has ended and sets itself up while that kernel's
+// last CTAs are still running.  Nothing that kernel may have produced is consumed early: the
+// producer executes grid_dependency_wait() before its first load, and everything the launches of a
+// context share -- partial slots, progress counters, the rule's state, the outputs, the status
+// word, the log -- is touched only after it as well.  If the caller vouches that the activations
+// were complete before the preceding kernel (early_inputs), the producer does not wait: the next
+// evaluation then streams while this one is still finishing its modules.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -91,6 +93,9 @@ struct TcParams {
     // CTA 0 stops after its first stage, so no accumulator is ever complete and (given more blocks
     // than pipeline stages) the producer runs out of free stages with loads in flight behind it.
     // Either way the waits run out, the CTA leaves through the give-up path and the kernel returns.
+    // 1: the activations were complete before the kernel that precedes this launch in the stream
+    // (the caller's promise, EGERIA_FLAG_OVERLAP), so the loads need not wait for that kernel.
+    uint32_t early_inputs;
     uint32_t test_stall;
     uint64_t wait_limit_ns;    // limit of every bounded wait of this launch (kWaitLimitNs, shorter for the hook)
     int32_t M;
@@ -288,6 +293,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            // Whatever wrote the activations must have ended before the first load -- unless the caller
+            // vouches that it was not the kernel before this one.
+            if (!p.early_inputs) ptx::grid_dependency_wait();
             const uint64_t policy = ptx::l2_policy_evict_first();
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0;
