@@ -180,7 +180,7 @@ double egeria_oracle_smooth(const double *P, int64_t i, int64_t W) {
 }
 
 /* Ordinary least squares slope of y[0..n-1] against x = 0..n-1
- * [Sec. 4.2.2 "linear least-squares regression"]. n < 2 has no line: +inf. */
+ * [Sec. 4.2.2: the smoothed plasticity is fitted with a least-squares line]. n < 2 has no line: +inf. */
 double egeria_oracle_ols_slope(const double *y, int64_t n) {
     if (n < 2) return INFINITY;
     double xm = 0.0, ym = 0.0;
@@ -384,7 +384,7 @@ int64_t egeria_oracle_bootstrap_replay(const float *loss, int64_t H, int64_t W, 
  * halved for the refreezing.
  *
  * Readings taken where the text leaves room:
- *   - "since the frontmost layers' freeze": the learning rate in force at the first freeze
+ *   - which freeze the drop is counted from: the learning rate in force at the first freeze
  *     after the start or after the last restart is remembered (lr_ref);
  *   - the test runs at the end of every evaluation, after the freeze step, as in Algorithm 1:
  *     restart iff lr_i <= lr_ref / 10 * (1 + 1e-6).  The slack of one part in a million lets a
