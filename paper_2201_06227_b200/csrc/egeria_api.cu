@@ -9,6 +9,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>  // header-only; a no-op unless a profiler is attached
+
 #include "../../include/egeria.h"
 #include "finalize.cuh"
 #include "gram_simt.cuh"
@@ -28,9 +30,37 @@ constexpr uint64_t kTestWaitLimitNs = 1000000ull;  // 1 ms: wait limit of a laun
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// A named range around the host side of a call, for timelines (Nsight Systems and the like).
+struct HostRange {
+    explicit HostRange(const char *name) { nvtxRangePushA(name); }
+    ~HostRange() { nvtxRangePop(); }
+};
+
+// Host-side check of a work split before it goes to the device: every unit lies inside its tile
+// and its slot inside the reserved slots, every CTA's range is a contiguous piece of the unit
+// table, every (module, side) has its slots in a row.  A split that fails is never uploaded.
+static bool plan_is_sane(const Plan &P, int M, const int64_t *d, int n_ctas, int64_t slot_cap) {
+    const int n_tc = P.n_units_tc, n_all = (int)P.units.size();
+    if (n_tc < 0 || n_tc > n_all) return false;
+    if ((int)P.cta_begin_tc.size() != n_ctas + 1 || (int)P.cta_begin_simt.size() != n_ctas + 1) return false;
+    if (P.cta_begin_tc[0] != 0 || P.cta_begin_tc[n_ctas] != n_tc) return false;
+    if (P.cta_begin_simt[0] != 0 || P.cta_begin_simt[n_ctas] != n_all - n_tc) return false;
+    for (int c = 0; c < n_ctas; ++c)
+        if (P.cta_begin_tc[c] > P.cta_begin_tc[c + 1] || P.cta_begin_simt[c] > P.cta_begin_simt[c + 1]) return false;
+    for (const Unit &u : P.units) {
+        if (u.module < 0 || u.module >= M || u.side < 0 || u.side > 2) return false;
+        if (u.kb0 < 0 || u.nkb < 1 || (int64_t)u.kb0 + u.nkb > kblocks_of(d[u.module])) return false;
+        if (u.slot < 0 || u.slot >= slot_cap || u.cta < 0 || u.cta >= n_ctas) return false;
+    }
+    if ((int)P.sides.size() != 2 * M) return false;
+    for (const SideInfo &si : P.sides)
+        if (si.n_slots < 0 || si.first_slot < 0 || (int64_t)si.first_slot + si.n_slots > slot_cap) return false;
+    return true;
+}
+
 // Offsets of everything the library keeps in the caller's workspace.
 struct Layout {
-    size_t status, cta_log, rowloss, tickets, fin_ctr, T, losses, keep, slots, staging, total;
+    size_t status, cta_log, rowloss, tickets, fin_ctr, T, losses, keep, chunk, slots, staging, total;
     // the freezing-rule state, one contiguous region [rule0, rule_end) (what export / import copy)
     size_t rule0, raw, plist, n_evals, counter, freeze_eval, last_slope, Tauto, smax, front, unfreeze, boot_raw,
         boot_plist, boot_ints, rule_end;
@@ -104,6 +134,20 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
     L.losses = take((size_t)M * sizeof(float));
     L.keep = off;
     if (flags & EGERIA_FLAG_KEEP_GRAMS) take((size_t)M * 2 * b_max * b_max * sizeof(float));
+    {
+        // scratch of the two-level finalisation (one module evaluated alone): rows x chunks x both
+        // sides x columns, float64; the chunk count is bounded by the units one module can have
+        size_t bytes = 0;
+        for (int mode = 0; mode <= mode_of_b(b_max) && mode <= kStacked64; ++mode) {  // used at b <= 64 only
+            const int nc = pitch_of_mode(mode) / 32;
+            const int chunk_slots = kFinStageBytes / (32 * nc * 4) / 2;
+            const size_t chunks = (size_t)(max_units(1, mode, kMaxCtas) + chunk_slots - 1) / chunk_slots;
+            const size_t rows = (size_t)(pitch_of_mode(mode) < b_max ? pitch_of_mode(mode) : b_max);
+            const size_t v = rows * chunks * 2 * 32 * nc * sizeof(double);
+            if (v > bytes) bytes = v;
+        }
+        L.chunk = take(bytes);
+    }
     size_t slot_bytes = 0;
     for (int mode = 0; mode <= mode_of_b(b_max); ++mode) {
         const size_t s = (size_t)max_units(M, mode, kMaxCtas) * slot_floats_of_mode(mode) * sizeof(float);
@@ -530,7 +574,8 @@ static egeria_status build_split(egeria_ctx *ctx, int b, bool front_only, const 
     out.front_cta_begin.clear();
     if (!front_only) {
         build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), out.plan, weights);
-        return EGERIA_OK;
+        const int64_t slot_cap = (int64_t)(ctx->L.slot_bytes_cap / (slot_floats_of_mode(out.plan.mode) * sizeof(float)));
+        return plan_is_sane(out.plan, M, ctx->d.data(), ctx->n_ctas, slot_cap) ? EGERIA_OK : EGERIA_ERR_WORKSPACE;
     }
     for (int m = 0; m < M; ++m)
         if (tc_ok[m] != 1) return EGERIA_ERR_UNSUPPORTED_SHAPE;
@@ -546,6 +591,9 @@ static egeria_status build_split(egeria_ctx *ctx, int b, bool front_only, const 
     for (int f = 0; f < M; ++f) {
         for (int m = 0; m < M; ++m) only[m] = (m == f) ? 1 : 2;
         build_plan(M, ctx->d.data(), b, ctx->n_ctas, only.data(), one, weights);
+        if (!plan_is_sane(one, M, ctx->d.data(), ctx->n_ctas,
+                          (int64_t)(ctx->L.slot_bytes_cap / (slot_floats_of_mode(one.mode) * sizeof(float)))))
+            return EGERIA_ERR_WORKSPACE;
         const int32_t base = (int32_t)all.units.size();
         all.units.insert(all.units.end(), one.units.begin(), one.units.end());
         for (int c = 0; c <= ctx->n_ctas; ++c)
@@ -833,6 +881,7 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
     fc.out_losses = out_losses;
     fc.rowloss = ctx->at<double>(L.rowloss);
     fc.keep = (ctx->flags & EGERIA_FLAG_KEEP_GRAMS) ? ctx->at<float>(L.keep) : nullptr;
+    fc.chunk_sums = ctx->at<double>(L.chunk);
     fc.fuse_step = fuse_step ? 1 : 0;
     fc.lr = ctx->lr;
     fc.rule_flags = ctx->rule_flags();
@@ -914,12 +963,14 @@ extern "C" {
 
 egeria_status egeria_sp_loss_batch(egeria_ctx *ctx, void *cuda_stream, const void *const *At, const void *const *Ar,
                                    int b, const int64_t *d, float *out_losses) {
+    HostRange range("egeria_sp_loss_batch");
     return sp_loss_impl(ctx, cuda_stream, At, Ar, b, d, out_losses, false, nullptr, nullptr);
 }
 
 egeria_status egeria_plasticity_evaluate(egeria_ctx *ctx, void *cuda_stream, const void *const *At,
                                          const void *const *Ar, int b, const int64_t *d, float *out_losses,
                                          double *out_slopes, uint8_t *out_mask) {
+    HostRange range("egeria_plasticity_evaluate");
     return sp_loss_impl(ctx, cuda_stream, At, Ar, b, d, out_losses, true, out_slopes, out_mask);
 }
 
@@ -941,6 +992,7 @@ egeria_status egeria_sp_loss_batch_host(egeria_ctx *ctx, void *cuda_stream, cons
     if (!ctx || !At_host || !Ar_host || !d || !out_losses_host) return EGERIA_ERR_INVALID_ARG;
     if (!(ctx->flags & EGERIA_FLAG_HOST_STAGING)) return EGERIA_ERR_WORKSPACE;
     if (b < 2 || b > ctx->b_max) return EGERIA_ERR_INVALID_ARG;
+    HostRange range("egeria_sp_loss_batch_host");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     for (int m = 0; m < ctx->M; ++m) {
         if (d[m] != ctx->d[m] || !At_host[m] || !Ar_host[m]) return EGERIA_ERR_INVALID_ARG;
@@ -961,6 +1013,7 @@ egeria_status egeria_sp_loss_batch_host(egeria_ctx *ctx, void *cuda_stream, cons
 egeria_status egeria_plasticity_step(egeria_ctx *ctx, void *cuda_stream, const float *losses, double *out_slopes,
                                      uint8_t *out_mask) {
     if (!ctx || !losses) return EGERIA_ERR_INVALID_ARG;
+    HostRange range("egeria_plasticity_step");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     ctx->last_stream = stream;
     ctx->rule_evals++;
@@ -1311,6 +1364,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     fc.out_losses = out_loss;
     fc.rowloss = reinterpret_cast<double *>(ws + L.rowloss);
     fc.keep = nullptr;
+    fc.chunk_sums = nullptr;
     fc.fuse_step = 0;
     fc.lr = NAN;
     fc.rule_flags = 0;

@@ -30,6 +30,7 @@ struct FinCommon {
     float *out_losses;      // [M]
     double *rowloss;        // [M][kMaxB] scratch
     float *keep;            // [M][2][b*b] normalised matrices, or nullptr
+    double *chunk_sums;     // scratch of the two-level finalisation (one module evaluated alone), or nullptr
     // fused freezing-rule step (fuse_step != 0): Algorithm 1 on the loss just computed
     int32_t fuse_step;
     int32_t rule_flags;     // RuleFlags
@@ -213,6 +214,115 @@ __device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const 
 #pragma unroll
     for (int c = 0; c < NC; ++c)
         if (fin_col<NC>(lane, c) >= b) gT[c] = gR[c] = 0.0;
+    return row_term<NC, true>(p, m, i, lane, gT, gR);
+}
+
+// ---- Two levels, for a module evaluated alone.  Such a module is cut over all CTAs, so a row of G
+// has a hundred or more partial rows per side, while there are far fewer rows than warps: one warp
+// per row would add them one after the other for tens of microseconds with most warps idle.
+// Instead a task is (row, chunk): a warp adds the row's partials of kChunk consecutive slots per
+// side (one pass of its stage) and leaves the two float64 sums in scratch; the warp that delivers
+// a row's last chunk adds the chunk sums in chunk order and finishes the row.  Which warp does
+// what does not change any sum, so the result is as reproducible as the one-level one.
+
+// Slots per side in one chunk: half the stage each for T and R.
+template <int NC>
+__host__ __device__ constexpr int fin_chunk_slots() { return kFinStageBytes / (32 * NC * 4) / 2; }
+// Doubles of scratch one (row, chunk) task leaves: both sides, this row, every column.
+template <int NC>
+__host__ __device__ constexpr int fin_chunk_doubles() { return 2 * 32 * NC; }
+
+// One warp: chunk `ch` of row i: fetch, add, store to scratch[(i * n_chunks + ch)].
+template <int NC>
+__device__ __forceinline__ void finalize_row_chunk(const FinCommon &p, const SideInfo &sT, const SideInfo &sR, int i,
+                                                   int ch, int n_chunks, int lane, float *stage) {
+    constexpr int kPitch = 32 * NC;
+    constexpr int kPieces = kPitch / 4;
+    constexpr int kLanesPerRow = kPieces < 32 ? kPieces : 32;
+    constexpr int kRowsPerIssue = 32 / kLanesPerRow;
+    constexpr int kIssuesPerRow = (kPieces + 31) / 32;
+    constexpr int kChunk = fin_chunk_slots<NC>();
+    const float *rowT = p.slots + (int64_t)sT.first_slot * p.slot_floats + sT.side_off + (int64_t)i * kPitch;
+    const float *rowR = p.slots + (int64_t)sR.first_slot * p.slot_floats + sR.side_off + (int64_t)i * kPitch;
+    const int t0 = ch * kChunk, r0 = ch * kChunk;
+    const int nT = (sT.n_slots - t0 < kChunk) ? (sT.n_slots - t0 > 0 ? sT.n_slots - t0 : 0) : kChunk;
+    const int nR = (sR.n_slots - r0 < kChunk) ? (sR.n_slots - r0 > 0 ? sR.n_slots - r0 : 0) : kChunk;
+    const int G = nT + nR;
+    const uint32_t stage_addr = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
+    const int sub = lane / kLanesPerRow, piece = lane % kLanesPerRow;
+    for (int sl0 = 0; sl0 < G; sl0 += kRowsPerIssue) {
+        const int sl = sl0 + sub;
+        if (sl < G) {
+            const float *src = (sl < nT) ? rowT + (int64_t)(t0 + sl) * p.slot_floats
+                                         : rowR + (int64_t)(r0 + sl - nT) * p.slot_floats;
+#pragma unroll
+            for (int q = 0; q < kIssuesPerRow; ++q) {
+                const int off = 4 * (piece + 32 * q);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_addr + (sl * kPitch + off) * 4),
+                             "l"(src + off)
+                             : "memory");
+            }
+        }
+    }
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    double gT[NC], gR[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) gT[c] = gR[c] = 0.0;
+    for (int sl = 0; sl < G; ++sl) {
+        const float *row = stage + sl * kPitch;
+        float v[NC];
+        if (NC >= 4) {
+#pragma unroll
+            for (int h = 0; h < NC / 4; ++h) {
+                const float4 t = *reinterpret_cast<const float4 *>(row + 128 * h + 4 * lane);
+                v[4 * h] = t.x;
+                v[4 * h + 1] = t.y;
+                v[4 * h + 2] = t.z;
+                v[4 * h + 3] = t.w;
+            }
+        } else if (NC == 2) {
+            const float2 t = *reinterpret_cast<const float2 *>(row + 2 * lane);
+            v[0] = t.x;
+            v[NC - 1] = t.y;
+        } else {
+            v[0] = row[lane];
+        }
+        if (sl < nT) {
+#pragma unroll
+            for (int c = 0; c < NC; ++c) gT[c] += (double)v[c];
+        } else {
+#pragma unroll
+            for (int c = 0; c < NC; ++c) gR[c] += (double)v[c];
+        }
+    }
+    __syncwarp();  // the stage is free again
+    double *out = p.chunk_sums + ((int64_t)i * n_chunks + ch) * fin_chunk_doubles<NC>();
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {  // [side][c][lane]: consecutive lanes, consecutive doubles
+        out[c * 32 + lane] = gT[c];
+        out[(NC + c) * 32 + lane] = gR[c];
+    }
+}
+
+// One warp, once all chunks of row i are in scratch and visible: add them in chunk order and
+// finish the row.  Returns the row's term (all lanes).
+template <int NC>
+__device__ __forceinline__ double finalize_row_from_chunks(const FinCommon &p, int m, int i, int n_chunks, int lane) {
+    double gT[NC], gR[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) gT[c] = gR[c] = 0.0;
+    const double *in = p.chunk_sums + (int64_t)i * n_chunks * fin_chunk_doubles<NC>();
+    for (int ch = 0; ch < n_chunks; ++ch, in += fin_chunk_doubles<NC>()) {
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            gT[c] += __ldcg(in + c * 32 + lane);
+            gR[c] += __ldcg(in + (NC + c) * 32 + lane);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+        if (fin_col<NC>(lane, c) >= p.b) gT[c] = gR[c] = 0.0;
     return row_term<NC, true>(p, m, i, lane, gT, gR);
 }
 

@@ -197,6 +197,20 @@ __device__ __forceinline__ bool next_chunk(int &k, int q, int lane, int b, float
     return false;
 }
 
+// What module m's row cursor counts up to: its b rows, or, when it is finished in two levels (a
+// module evaluated alone, cut into many partials, b <= 64), its (row, chunk) tasks.  (At b > 64 the
+// chunk sums are 2 to 4 KB per task and the scratch traffic eats the gain: measured 22 -> 22 us at
+// b = 128, 92 -> 98 us at b = 256, against 66 -> 55 us at b = 64 and 27 -> 23 us at b = 32.)
+template <int NC>
+__device__ __forceinline__ int module_tasks(const TcParams &p, int m) {
+    const int nT = p.fin.sides[2 * m].n_slots, nR = p.fin.sides[2 * m + 1].n_slots;
+    const int most = nT > nR ? nT : nR;
+    constexpr int kChunk = fin_chunk_slots<NC>();
+    if (NC <= 2 && p.n_active == 1 && p.fin.chunk_sums && most > kChunk)
+        return p.fin.b * ((most + kChunk - 1) / kChunk);
+    return p.fin.b;
+}
+
 // One warp: take rows of module m from its cursor until none is left.  The claim of the next
 // row is in flight while the current one is worked on; the rows' terms are delivered together.
 // `stage` is kFinStageBytes of shared memory for this warp alone.
@@ -209,12 +223,37 @@ __device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int
     if (lane == 0) r = atomicAdd(&c->row_cursor, 1);
     const SideInfo sT = p.fin.sides[2 * m], sR = p.fin.sides[2 * m + 1];  // in flight with the claim
     r = __shfl_sync(0xffffffffu, r, 0);
-    while (r < b) {
-        int r_next = 0;
-        if (lane == 0) r_next = atomicAdd(&c->row_cursor, 1);
-        const double term = finalize_row_staged<NC>(p.fin, sT, sR, m, r, lane, stage);
-        mine += row_acc_of(term);
-        r = __shfl_sync(0xffffffffu, r_next, 0);
+    constexpr int kChunk = fin_chunk_slots<NC>();
+    const int most = sT.n_slots > sR.n_slots ? sT.n_slots : sR.n_slots;
+    if (NC <= 2 && p.n_active == 1 && p.fin.chunk_sums && most > kChunk) {
+        // A module evaluated alone: (row, chunk) tasks, see finalize_row_chunk.  The cursor counts
+        // tasks; task v is chunk v % n_chunks of row v / n_chunks.
+        const int n_chunks = (most + kChunk - 1) / kChunk;
+        const int n_tasks = b * n_chunks;
+        while (r < n_tasks) {
+            int r_next = 0;
+            if (lane == 0) r_next = atomicAdd(&c->row_cursor, 1);
+            const int row = r / n_chunks, ch = r % n_chunks;
+            finalize_row_chunk<NC>(p.fin, sT, sR, row, ch, n_chunks, lane, stage);
+            __threadfence();  // every lane's sums, before the count
+            __syncwarp();
+            int done = 0;
+            if (lane == 0) done = atomicAdd(&c->row_chunks_done[row], 1);
+            done = __shfl_sync(0xffffffffu, done, 0);
+            if (done == n_chunks - 1) {
+                __threadfence();
+                mine += row_acc_of(finalize_row_from_chunks<NC>(p.fin, m, row, n_chunks, lane));
+            }
+            r = __shfl_sync(0xffffffffu, r_next, 0);
+        }
+    } else {
+        while (r < b) {
+            int r_next = 0;
+            if (lane == 0) r_next = atomicAdd(&c->row_cursor, 1);
+            const double term = finalize_row_staged<NC>(p.fin, sT, sR, m, r, lane, stage);
+            mine += row_acc_of(term);
+            r = __shfl_sync(0xffffffffu, r_next, 0);
+        }
     }
     if (mine == 0) return;
     // One atomic add delivers the terms and says whether these were the module's last rows; what
@@ -562,17 +601,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             // covers parts of several modules works on all of them at once -- and waits (a while)
             // for those that are not complete yet.  The wait is a courtesy, see above.
             for (int base = u_begin; base < u_end; base += 32) {
-                int my_m = -1, my_total = 0;
+                int my_m = -1, my_total = 0, my_tasks = b;
                 if (base + lane < u_end) {
                     my_m = p.units[base + lane].module;
                     if (base + lane > u_begin && p.units[base + lane - 1].module == my_m) my_m = -1;
                 }
                 if (my_m >= 0) {
                     my_total = p.fin.sides[2 * my_m].module_units;
+                    my_tasks = detail::module_tasks<Cfg::kNC>(p, my_m);
                     // With many CTAs on a module and few rows, most claims would find nothing and only
-                    // crowd the cursor: as many warps of this CTA as its share of the rows, plus one.
+                    // crowd the cursor: as many warps of this CTA as its share of the rows (or of the
+                    // (row, chunk) tasks), plus one.
                     const int ctas_on_m = Cfg::kStacked ? my_total : (my_total + 1) / 2;
-                    if (warp - 2 > (b + ctas_on_m - 1) / ctas_on_m) my_m = -1;
+                    if (warp - 2 > (my_tasks + ctas_on_m - 1) / ctas_on_m) my_m = -1;
                 }
                 uint32_t pending = __ballot_sync(0xffffffffu, my_m >= 0);
                 uint64_t t_wait = ptx::globaltimer_ns();
@@ -583,7 +624,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                         const int done = detail::ld_acquire(&p.ctr[my_m].units_done);
                         const int cur = detail::ld_acquire(&p.ctr[my_m].row_cursor);
                         ready = (done >= my_total);
-                        left = b - cur;
+                        left = my_tasks - cur;
                     }
                     pending &= ~__ballot_sync(0xffffffffu, ready && left <= 0);  // complete, every row claimed
                     const uint32_t cand = __ballot_sync(0xffffffffu, ready && left > 0);
@@ -615,7 +656,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                     if (!si.tensor_core || si.module_units == 0) continue;
                     const int done = detail::ld_acquire(&p.ctr[mm].units_done);
                     const int cur = detail::ld_acquire(&p.ctr[mm].row_cursor);
-                    const int left = (done >= si.module_units) ? b - cur : 0;
+                    const int left = (done >= si.module_units) ? detail::module_tasks<Cfg::kNC>(p, mm) - cur : 0;
                     if (left > best_left) {
                         best_left = left;
                         best_m = mm;

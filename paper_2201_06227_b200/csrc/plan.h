@@ -90,6 +90,7 @@ struct FinCounters {
     unsigned long long row_acc;  // the rows' terms of the loss so far and how many rows they are (packed:
                                  // one atomic add per warp carries both, see finalize.cuh)
     int32_t pad2[30];
+    int32_t row_chunks_done[256];  // two-level finalisation: chunks of each row whose sums are in scratch
 };
 
 // Per-module pointers for the CUDA-core kernel.

@@ -69,6 +69,18 @@ def test_single_module_tensor_core_path(b, d):
     compare_with_oracle([at], [ar], what=f"b={b} d={d}")
 
 
+@pytest.mark.parametrize("b,d", [(8, 64 * 148 * 9), (32, 64 * 148 * 12 + 72), (33, 64 * 148 * 9), (64, 64 * 148 * 10),
+                                 (128, 64 * 148 * 5), (256, 64 * 148 * 4)])
+def test_single_module_cut_over_every_cta(b, d):
+    """One module alone over all 148 CTAs: a row of G has 148 partial rows per side.  At b <= 64
+    the finalisation then runs in two levels ((row, chunk) tasks, chunk sums in scratch); entries
+    and loss against the oracle, and the same bits on a second evaluation."""
+    at, ar = wl.make_pair(b, d, "relu" if b % 2 else "normal", 0.25, seed=31 * b + 7, device=DEV)
+    losses = compare_with_oracle([at], [ar], flags=eg.FLAG_EQUAL_SPLIT, what=f"alone b={b} d={d}")
+    again, _ = run_gpu([at], [ar], flags=eg.FLAG_EQUAL_SPLIT)
+    assert again.tobytes() == losses.tobytes()
+
+
 @pytest.mark.parametrize("b,d", [(2, 1), (5, 7), (8, 100), (64, 1001), (100, 333), (130, 250), (256, 65)])
 def test_single_module_cuda_core_path_for_unaligned_d(b, d):
     at, ar = wl.make_pair(b, d, "normal", 0.3, seed=77 + b + d, device=DEV)
