@@ -365,6 +365,20 @@ egeria_status egeria_debug_plan_weighted(int M, const int64_t *d, int b, int n_c
  * warps. */
 egeria_status egeria_debug_plan_help(int M, const int64_t *d, int b, int n_ctas, int32_t *out_help);
 
+/* Test hook: how the end of a launch is cut into tasks and who starts with which, pure host
+ * arithmetic for the split egeria_debug_plan returns (only_module >= 0: that module evaluated
+ * alone, as in a front-only evaluation).  A task is a row of G, or, for a module evaluated alone
+ * at b <= 64 and cut into more partials than one pass of a warp's staging area holds, a (row,
+ * chunk) pair.  Writes
+ *   out_first[c * 12 + w]  the task epilogue warp w of CTA c starts with, (module << 16) | task,
+ *                          or -1 (host int32 [n_ctas * 12]);
+ *   out_tasks[2 m], out_tasks[2 m + 1]  module m's tasks and how many of them have a warp of their
+ *                          own from the start; the module's cursor hands out the rest (host int32 [2 M]);
+ *   *out_validate          1 if the kernel would tell an arrived partial row by its contents (every
+ *                          task has its own warp and fits one pass), 0 if by the unit counters. */
+egeria_status egeria_debug_plan_tasks(int M, const int64_t *d, int b, int n_ctas, int only_module,
+                                      int32_t *out_first, int32_t *out_tasks, int *out_validate);
+
 /* Test hook for the bounded waits: the NEXT evaluation kernel of this context (tensor-core
  * modules) runs with every wait limited to one millisecond instead of two seconds, and with one
  * hand-shake of its first thread block left out on purpose, so that the waits that depend on it

@@ -32,7 +32,7 @@ EXPORTS = [
     "egeria_split_weights", "egeria_status_string", "egeria_bootstrap_step", "egeria_bootstrap_replay",
     "egeria_bootstrap_reset", "egeria_plasticity_state_bytes", "egeria_plasticity_export", "egeria_plasticity_import",
     "egeria_sp_loss_subset", "egeria_plasticity_evaluate_subset",
-    "egeria_sp_loss_static_status", "egeria_debug_stall_next", "egeria_debug_plan_help", "egeria_plasticity_set_lr", "egeria_plasticity_restarts", "egeria_plasticity_replay_lr",
+    "egeria_sp_loss_static_status", "egeria_debug_stall_next", "egeria_debug_plan_help", "egeria_debug_plan_tasks", "egeria_plasticity_set_lr", "egeria_plasticity_restarts", "egeria_plasticity_replay_lr",
 ]
 
 
@@ -95,6 +95,9 @@ def lib() -> ctypes.CDLL:
     L.egeria_sp_loss_static_status.argtypes = []
     L.egeria_debug_stall_next.argtypes = [vp, ctypes.c_int]
     L.egeria_debug_plan_help.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int32)]
+    L.egeria_debug_plan_tasks.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                          ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
+                                          ctypes.POINTER(ctypes.c_int)]
     L.egeria_launch_count.argtypes = [vp]
     L.egeria_launch_count.restype = ctypes.c_int64
     L.egeria_status_string.argtypes = [ctypes.c_int]
@@ -146,6 +149,19 @@ def egeria_debug_plan_help(d: Sequence[int], b: int, n_ctas: int) -> np.ndarray:
                                       out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)))
     _check(st, "egeria_debug_plan_help")
     return out
+
+
+def egeria_debug_plan_tasks(d: Sequence[int], b: int, n_ctas: int, only_module: int = -1):
+    """How the end of a launch is cut into tasks: (first[n_ctas, 12] = (module << 16) | task or -1,
+    tasks[M, 2] = {tasks, tasks with a warp of their own}, validate)."""
+    first = np.zeros((n_ctas, 12), dtype=np.int32)
+    tasks = np.zeros((len(d), 2), dtype=np.int32)
+    v = ctypes.c_int(0)
+    st = lib().egeria_debug_plan_tasks(len(d), _i64(d), int(b), int(n_ctas), int(only_module),
+                                       first.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                       tasks.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), ctypes.byref(v))
+    _check(st, "egeria_debug_plan_tasks")
+    return first, tasks, bool(v.value)
 
 
 def egeria_debug_plan_weighted(d: Sequence[int], b: int, n_ctas: int, weights) -> np.ndarray:

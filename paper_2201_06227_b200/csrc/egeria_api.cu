@@ -66,10 +66,13 @@ struct Layout {
         boot_plist, boot_ints, rule_end;
     size_t replay_raw, replay_plist;  // windows of egeria_plasticity_replay_lr ([M][W] doubles each)
     size_t slot_bytes_cap;  // bytes reserved for partial slots
+    size_t slot_set_bytes;  // launches that validate partial rows by their contents (b <= 128) alternate
+                            // between the sets [0, slot_set_bytes) and [slot_set_bytes, 2 slot_set_bytes)
     // Device-side plans (tensor maps, pointers, unit table, per-CTA ranges, slot ranges): kPlanSlots
     // regions of plan_stride bytes from plan0; the offsets below are relative to a region.
     size_t plan0, plan_stride;
-    size_t tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides, cta_help;
+    size_t tmaps, modules, units, cta_begin_tc, cta_begin_simt, sides, cta_help, first_task;
+    size_t first_task_bytes;
 };
 
 // Units of one device-side plan: all modules in one split, or (front-only contexts) one split per
@@ -106,6 +109,8 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
         L.cta_begin_simt = take((kMaxCtas + 1) * sizeof(int32_t));
         L.sides = take((size_t)2 * M * sizeof(SideInfo));
         L.cta_help = take((size_t)kMaxCtas * sizeof(CtaHelp));
+        L.first_task_bytes = (size_t)((flags & EGERIA_FLAG_FRONT_ONLY) ? M : 1) * kMaxCtas * kEpiWarps * sizeof(int32_t);
+        L.first_task = take(L.first_task_bytes);
         L.plan_stride = off;
         off = saved;
         L.plan0 = take(L.plan_stride * kPlanSlots);
@@ -148,11 +153,15 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
         }
         L.chunk = take(bytes);
     }
-    size_t slot_bytes = 0;
+    size_t slot_bytes = 0, set_bytes = 0;
     for (int mode = 0; mode <= mode_of_b(b_max); ++mode) {
         const size_t s = (size_t)max_units(M, mode, kMaxCtas) * slot_floats_of_mode(mode) * sizeof(float);
         if (s > slot_bytes) slot_bytes = s;
+        if (mode <= kSingle1 && s > set_bytes) set_bytes = s;
     }
+    set_bytes = align_up(set_bytes, 256);
+    if (2 * set_bytes > slot_bytes) slot_bytes = 2 * set_bytes;
+    L.slot_set_bytes = set_bytes;
     L.slot_bytes_cap = slot_bytes;
     L.slots = take(slot_bytes);
     L.staging = off;
@@ -195,6 +204,8 @@ struct BuiltPlan {
     std::vector<uint8_t> tc_ok;
     Plan plan;
     std::vector<int32_t> front_cta_begin;
+    std::vector<int32_t> front_first_task;  // [M][kMaxCtas * kEpiWarps]
+    int slot_units = 0;  // partial slots a launch of this plan may write (front-only: of the largest front)
     uint64_t last_use = 0;
 };
 constexpr int kBuiltPlans = 4;
@@ -229,6 +240,7 @@ struct egeria_ctx {
         int weights_version = 0;
         std::vector<const void *> At, Ar;
         Plan plan;
+        int slot_units = 0;  // partial slots a launch of this plan may write
         uint64_t last_use = 0;
     };
     PlanEntry plans[kPlanSlots];
@@ -244,6 +256,9 @@ struct egeria_ctx {
     int64_t launches = 0;
     uint32_t tc_launches = 0;  // selects the set of progress counters the next tensor-core launch uses
     uint32_t rule_evals = 0;   // evaluations of the freezing rule enqueued so far (the serial of the last one)
+    bool slots_dirty = false;  // a launch that does not validate rows has left its partials in the slots
+    int val_set = 0;           // set of slots the next launch that validates rows uses
+    size_t set_dirty[2] = {0, 0};  // bytes from the start of each set that a launch wrote and nobody has emptied
     uint32_t stall_next = 0;   // test hook: give-up path of the next tensor-core launch (egeria_debug_stall_next)
     // Split weights: one per CTA, from the streaming rates the CTAs report (SMs do not all get
     // the same share of HBM bandwidth; the CTA -> SM placement repeats from launch to launch).
@@ -371,6 +386,24 @@ egeria_status egeria_debug_plan_help(int M, const int64_t *d, int b, int n_ctas,
     return EGERIA_OK;
 }
 
+egeria_status egeria_debug_plan_tasks(int M, const int64_t *d, int b, int n_ctas, int only_module, int32_t *out_first,
+                                      int32_t *out_tasks, int *out_validate) {
+    if (!out_first || !out_tasks || !out_validate || n_ctas < 1 || only_module >= M) return EGERIA_ERR_INVALID_ARG;
+    egeria_status s = check_shapes(M, d, b, 1);
+    if (s != EGERIA_OK) return s;
+    std::vector<uint8_t> tc_ok(M);
+    for (int m = 0; m < M; ++m) tc_ok[m] = (only_module >= 0 && m != only_module) ? 2 : (d[m] % 8 == 0);
+    Plan plan;
+    build_plan(M, d, b, n_ctas, tc_ok.data(), plan, nullptr, kEpiWarps, true);
+    memcpy(out_first, plan.first_task.data(), plan.first_task.size() * sizeof(int32_t));
+    for (int m = 0; m < M; ++m) {
+        out_tasks[2 * m] = plan.sides[2 * (size_t)m].n_tasks;
+        out_tasks[2 * m + 1] = plan.sides[2 * (size_t)m].n_static;
+    }
+    *out_validate = plan.validate_rows ? 1 : 0;
+    return EGERIA_OK;
+}
+
 egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d, int b_max, int W, const float *T,
                                        float T_all, void *workspace, size_t workspace_bytes, uint32_t flags) {
     if (!out) return EGERIA_ERR_INVALID_ARG;
@@ -455,6 +488,7 @@ egeria_status egeria_plasticity_create(egeria_ctx **out, int M, const int64_t *d
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.cta_log, 0, kMaxCtas * sizeof(CtaLog));
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.tickets, 0, (size_t)M * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.fin_ctr, 0, (size_t)2 * M * sizeof(FinCounters));
+    if (e == cudaSuccess) e = cudaMemset(ctx->ws + L.slots, 0xff, L.slot_bytes_cap);  // every partial slot empty (kSlotEmpty)
     if (e == cudaSuccess) e = cudaMemcpy(ctx->ws + L.T, Th.data(), (size_t)M * sizeof(float), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) {
         plasticity_clear_kernel<<<(M + 127) / 128, 128>>>(ctx->slope_state(), M, W, 0);
@@ -572,8 +606,10 @@ static egeria_status build_split(egeria_ctx *ctx, int b, bool front_only, const 
                                  const float *weights, BuiltPlan &out) {
     const int M = ctx->M;
     out.front_cta_begin.clear();
+    out.front_first_task.clear();
     if (!front_only) {
-        build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), out.plan, weights);
+        build_plan(M, ctx->d.data(), b, ctx->n_ctas, tc_ok.data(), out.plan, weights, kEpiWarps, true);
+        out.slot_units = (int)out.plan.units.size();
         const int64_t slot_cap = (int64_t)(ctx->L.slot_bytes_cap / (slot_floats_of_mode(out.plan.mode) * sizeof(float)));
         return plan_is_sane(out.plan, M, ctx->d.data(), ctx->n_ctas, slot_cap) ? EGERIA_OK : EGERIA_ERR_WORKSPACE;
     }
@@ -583,14 +619,19 @@ static egeria_status build_split(egeria_ctx *ctx, int b, bool front_only, const 
     all = Plan{};
     all.mode = mode_of_b(b);
     all.n_ctas = ctx->n_ctas;
-    all.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, {0, 0}});
+    all.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, 0, 0});
     all.all_ctas_busy_tc = true;
     out.front_cta_begin.assign((size_t)M * (kMaxCtas + 1), 0);
+    out.front_first_task.assign((size_t)M * kMaxCtas * kEpiWarps, -1);
+    all.validate_rows = true;  // (one protocol for whichever front the device picks)
+    out.slot_units = 0;
     std::vector<uint8_t> only(M);
     Plan one;
     for (int f = 0; f < M; ++f) {
         for (int m = 0; m < M; ++m) only[m] = (m == f) ? 1 : 2;
-        build_plan(M, ctx->d.data(), b, ctx->n_ctas, only.data(), one, weights);
+        build_plan(M, ctx->d.data(), b, ctx->n_ctas, only.data(), one, weights, kEpiWarps, true);
+        memcpy(&out.front_first_task[(size_t)f * kMaxCtas * kEpiWarps], one.first_task.data(),
+               one.first_task.size() * sizeof(int32_t));
         if (!plan_is_sane(one, M, ctx->d.data(), ctx->n_ctas,
                           (int64_t)(ctx->L.slot_bytes_cap / (slot_floats_of_mode(one.mode) * sizeof(float)))))
             return EGERIA_ERR_WORKSPACE;
@@ -601,6 +642,8 @@ static egeria_status build_split(egeria_ctx *ctx, int b, bool front_only, const 
         all.sides[2 * (size_t)f] = one.sides[2 * (size_t)f];
         all.sides[2 * (size_t)f + 1] = one.sides[2 * (size_t)f + 1];
         all.all_ctas_busy_tc = all.all_ctas_busy_tc && one.all_ctas_busy_tc;
+        all.validate_rows = all.validate_rows && one.validate_rows;
+        if ((int)one.units.size() > out.slot_units) out.slot_units = (int)one.units.size();
         if ((size_t)one.units.size() * slot_floats_of_mode(one.mode) * sizeof(float) > ctx->L.slot_bytes_cap)
             return EGERIA_ERR_WORKSPACE;
     }
@@ -666,6 +709,7 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
         bp->last_use = ++ctx->use_clock;
     }
     e.plan = bp->plan;
+    e.slot_units = bp->slot_units;
     const std::vector<int32_t> &front_cta_begin = bp->front_cta_begin;
     const Plan &P = e.plan;
     const Layout &L = ctx->L;
@@ -722,6 +766,11 @@ static egeria_status refresh_plan(egeria_ctx *ctx, cudaStream_t stream, const vo
     memcpy(img + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo));
     if (!front_only && !P.cta_help.empty())  // (the image is zeroed: no help planned otherwise)
         memcpy(img + L.cta_help, P.cta_help.data(), P.cta_help.size() * sizeof(CtaHelp));
+    memset(img + L.first_task, 0xff, L.first_task_bytes);  // -1: no task
+    if (front_only)
+        memcpy(img + L.first_task, bp->front_first_task.data(), bp->front_first_task.size() * sizeof(int32_t));
+    else
+        memcpy(img + L.first_task, P.first_task.data(), P.first_task.size() * sizeof(int32_t));
     // From pageable memory the runtime stages the bytes before returning, so `pack` may be reused.
     EG_CUDA(cudaMemcpyAsync(ctx->plan_region(lru), img, L.plan_stride, cudaMemcpyHostToDevice, stream));
     if (ctx->pinned_plans) {
@@ -756,7 +805,7 @@ static cudaError_t launch_finalize(const FinParams &fp, int M, int b, cudaStream
 // any other kernel implicitly as its CTAs end.  The kernel itself waits (griddepcontrol.wait) before
 // it reads an activation or touches anything in the workspace, so nothing is consumed early.
 template <int MODE>
-static cudaError_t launch_tc(int n_ctas, cudaStream_t stream, const TcParams &tp) {
+static cudaError_t launch_tc(int n_ctas, cudaStream_t stream, const TcParams &tp, bool programmatic) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_ctas);
     cfg.blockDim = dim3(kTcThreads);
@@ -766,16 +815,17 @@ static cudaError_t launch_tc(int n_ctas, cudaStream_t stream, const TcParams &tp
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = programmatic ? 1 : 0;  // (not after a memset: an ordinary, fully serialised launch)
     return cudaLaunchKernelEx(&cfg, gram_tc_kernel<MODE>, tp);
 }
 
-static cudaError_t launch_tc_mode(int mode, int n_ctas, cudaStream_t stream, const TcParams &tp) {
+static cudaError_t launch_tc_mode(int mode, int n_ctas, cudaStream_t stream, const TcParams &tp,
+                                  bool programmatic = true) {
     switch (mode) {
-        case kStacked32: return launch_tc<kStacked32>(n_ctas, stream, tp);
-        case kStacked64: return launch_tc<kStacked64>(n_ctas, stream, tp);
-        case kSingle1: return launch_tc<kSingle1>(n_ctas, stream, tp);
-        default: return launch_tc<kSingle2>(n_ctas, stream, tp);
+        case kStacked32: return launch_tc<kStacked32>(n_ctas, stream, tp, programmatic);
+        case kStacked64: return launch_tc<kStacked64>(n_ctas, stream, tp, programmatic);
+        case kSingle1: return launch_tc<kSingle1>(n_ctas, stream, tp, programmatic);
+        default: return launch_tc<kSingle2>(n_ctas, stream, tp, programmatic);
     }
 }
 
@@ -874,7 +924,35 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         EG_CUDA(cudaEventRecord(ev0, stream));
     }
     FinCommon fc;
-    fc.slots = ctx->at<float>(L.slots);
+    // How the finish learns that a partial row has arrived (Plan::validate_rows), and which slots
+    // the launch uses.  Launches that validate alternate between two sets of slots; each empties what
+    // the one before wrote into the other set (the tensor-core kernel does, so there must be one).
+    const size_t plan_slot_bytes = (size_t)ctx->plans[ctx->cur].slot_units * slot_floats * sizeof(float);
+    fc.sentinel = (P.validate_rows && P.n_units_tc > 0 && plan_slot_bytes <= L.slot_set_bytes) ? 1u : 0u;
+    fc.wait_limit_ns = ctx->stall_next ? kTestWaitLimitNs : kWaitLimitNs;
+    bool after_memset = false;
+    float *slot_base = ctx->at<float>(L.slots);
+    uint4 *empty_ptr = nullptr;
+    uint32_t empty_n = 0;
+    if (fc.sentinel) {
+        if (ctx->slots_dirty) {
+            // the launch before left what it wrote all over the slots (the other protocol)
+            EG_CUDA(cudaMemsetAsync(ctx->ws + L.slots, 0xff, L.slot_bytes_cap, stream));
+            ctx->slots_dirty = false;
+            ctx->set_dirty[0] = ctx->set_dirty[1] = 0;
+            after_memset = true;
+        }
+        const int set = ctx->val_set, other = set ^ 1;
+        slot_base = reinterpret_cast<float *>(ctx->ws + L.slots + (size_t)set * L.slot_set_bytes);
+        empty_ptr = reinterpret_cast<uint4 *>(ctx->ws + L.slots + (size_t)other * L.slot_set_bytes);
+        empty_n = (uint32_t)(ctx->set_dirty[other] / sizeof(uint4));
+        ctx->set_dirty[other] = 0;
+        if (plan_slot_bytes > ctx->set_dirty[set]) ctx->set_dirty[set] = plan_slot_bytes;
+        ctx->val_set = other;
+    } else if (!P.units.empty()) {
+        ctx->slots_dirty = true;
+    }
+    fc.slots = slot_base;
     fc.slot_floats = slot_floats;
     fc.sides = reinterpret_cast<const SideInfo *>(region + L.sides);
     fc.b = b;
@@ -899,7 +977,11 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         tp.cta_help = front_only ? nullptr : reinterpret_cast<const CtaHelp *>(region + L.cta_help);
         tp.front_word = front_only ? ctx->slope_state().front : nullptr;
         tp.cta_stride = kMaxCtas + 1;
-        tp.slots = ctx->at<float>(L.slots);
+        tp.first_task = reinterpret_cast<const int32_t *>(region + L.first_task);
+        tp.first_stride = kMaxCtas * kEpiWarps;
+        tp.empty_ptr = empty_ptr;
+        tp.empty_n = empty_n;
+        tp.slots = slot_base;
         tp.status = ctx->at<int32_t>(L.status);
         FinCounters *sets = ctx->at<FinCounters>(L.fin_ctr);
         const uint32_t set = ctx->tc_launches & 1u;
@@ -921,7 +1003,7 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         tp.test_stall = ctx->stall_next;
         tp.wait_limit_ns = ctx->stall_next ? kTestWaitLimitNs : kWaitLimitNs;
         ctx->stall_next = 0;
-        if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp) != cudaSuccess) return EGERIA_ERR_CUDA;
+        if (launch_tc_mode(P.mode, ctx->n_ctas, stream, tp, !after_memset) != cudaSuccess) return EGERIA_ERR_CUDA;
         if (log_it) {
             const int k = ctx->calib_enqueued;
             EG_CUDA(cudaMemcpyAsync(ctx->host_log + (size_t)k * kMaxCtas, tp.log, (size_t)ctx->n_ctas * sizeof(CtaLog),
@@ -938,7 +1020,7 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         sp.modules = reinterpret_cast<const ModulePtrs *>(region + L.modules);
         sp.units = reinterpret_cast<const Unit *>(region + L.units) + P.n_units_tc;
         sp.cta_begin = reinterpret_cast<const int32_t *>(region + L.cta_begin_simt);
-        sp.slots = ctx->at<float>(L.slots);
+        sp.slots = slot_base;
         sp.slot_floats = slot_floats;
         sp.b = b;
         sp.mode = P.mode;
@@ -1204,6 +1286,10 @@ egeria_status egeria_device_status(egeria_ctx *ctx) {
         // a kernel that gave up leaves its progress counters and tickets half-way: start afresh
         EG_CUDA(cudaMemset(ctx->ws + ctx->L.fin_ctr, 0, (size_t)2 * ctx->M * sizeof(FinCounters)));
         EG_CUDA(cudaMemset(ctx->ws + ctx->L.tickets, 0, (size_t)ctx->M * sizeof(int32_t)));
+        // ... and partial rows that were written and never read: every slot empty again
+        EG_CUDA(cudaMemset(ctx->ws + ctx->L.slots, 0xff, ctx->L.slot_bytes_cap));
+        ctx->slots_dirty = false;
+        ctx->set_dirty[0] = ctx->set_dirty[1] = 0;
         EG_CUDA(cudaMemset(ctx->ws + ctx->L.status, 0, sizeof(int32_t)));
     }
     if (word == kStatusTimeout) return EGERIA_ERR_TIMEOUT;
@@ -1314,7 +1400,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     const uint8_t tc_ok = (reinterpret_cast<uintptr_t>(At) % 16 == 0) && (reinterpret_cast<uintptr_t>(Ar) % 16 == 0) &&
                           (d % 8 == 0);
     Plan P;
-    build_plan(1, &d, b, kStaticCtas, &tc_ok, P);
+    build_plan(1, &d, b, kStaticCtas, &tc_ok, P, nullptr, kEpiWarps, false, false);  // every row from the cursor
     if ((int64_t)P.units.size() > max_units(1, kSingle1, kStaticCtas)) return EGERIA_ERR_WORKSPACE;
 
     CUtensorMap maps[2];
@@ -1357,8 +1443,10 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     const int64_t slot_floats = slot_floats_of_mode(P.mode);
     int32_t *ticket = reinterpret_cast<int32_t *>(ws + L.ticket);
     FinCommon fc;
-    fc.slots = reinterpret_cast<const float *>(ws + L.slots);
+    fc.slots = reinterpret_cast<float *>(ws + L.slots);
     fc.slot_floats = slot_floats;
+    fc.sentinel = 0u;  // counters and fences say when a partial is complete: the scratch needs no preparation
+    fc.wait_limit_ns = kWaitLimitNs;
     fc.sides = reinterpret_cast<const SideInfo *>(ws + L.sides);
     fc.b = b;
     fc.out_losses = out_loss;
@@ -1381,6 +1469,10 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         tp.cta_help = nullptr;
         tp.front_word = nullptr;
         tp.cta_stride = 0;
+        tp.first_task = nullptr;
+        tp.first_stride = 0;
+        tp.empty_ptr = nullptr;
+        tp.empty_n = 0;
         tp.slots = reinterpret_cast<float *>(ws + L.slots);
         tp.status = ticket + 1;
         tp.ctr = reinterpret_cast<FinCounters *>(ticket + 2);

@@ -22,9 +22,20 @@ constexpr int kFinRowsPerCta = kFinThreads / 32;
 constexpr int kMaxB = 256;
 constexpr double kNormEps = 1e-12;
 
+// What a partial slot holds where nothing has been written since it was last emptied: the
+// tensor-core kernel's finish can tell a partial row that has arrived from one that has not by its
+// values alone (no flag, no fence: every 4-byte element is its own flag).  The epilogue never
+// stores this pattern as a value (a NaN with these bits becomes the canonical one); launches that
+// work this way alternate between two sets of slots, and each empties, at its start, what the
+// launch before wrote into the other set.
+constexpr uint32_t kSlotEmpty = 0xffffffffu;
+constexpr uint32_t kCanonicalNan = 0x7fc00000u;
+
 struct FinCommon {
-    const float *slots;
+    float *slots;
     int64_t slot_floats;
+    uint32_t sentinel;      // 1: a partial row has arrived when none of its elements is kSlotEmpty (no counters)
+    uint64_t wait_limit_ns; // limit of the wait for partial rows that have not arrived
     const SideInfo *sides;  // [2 * M]
     int32_t b;
     float *out_losses;      // [M]
@@ -138,22 +149,110 @@ __device__ __forceinline__ double finalize_row(const FinCommon &p, const SideInf
     return row_term<NC, false>(p, m, i, lane, gT, gR);
 }
 
-constexpr int kFinStageBytes = 16384;  // warp-private shared memory of the staged variant
 
-// The same row with the partials staged through `stage` (kFinStageBytes of shared memory that
-// only this warp touches): every 16-byte piece of the row in every partial slot is fetched with
-// cp.async, all in flight together whatever the register budget, then added from shared memory
-// in ascending slot order (A_T's partials, then A_R's).  A lane owns the columns fin_col(lane, c).
-// The partial slots of the tensor-core modes have a row pitch of exactly 32 * NC floats.
-template <int NC>
-__device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const SideInfo sT, const SideInfo sR, int m,
-                                                      int i, int lane, float *stage) {
+// One warp: rows 0 .. G - 1 of the stage <- the partial rows src_of(0 .. G - 1) (32 * NC floats
+// each), every 16-byte piece fetched with cp.async, all in flight together whatever the register
+// budget.  With p.sentinel the rows need not have arrived yet: pieces that still hold kSlotEmpty
+// in the columns the epilogue writes (the first b, rounded up to 32) are fetched again until they
+// do not -- at most p.wait_limit_ns, then the CTA's abort flag is set and false returned.  (The
+// slots are put back to kSlotEmpty by the launch after this one, which uses another set of them.)
+template <int NC, class SrcOf>
+__device__ __forceinline__ bool fetch_partial_rows(const FinCommon &p, int G, SrcOf src_of, int lane, float *stage,
+                                                   volatile int *abort_flag) {
     constexpr int kPitch = 32 * NC;                          // floats per row of a partial
     constexpr int kPieces = kPitch / 4;                      // 16-byte pieces per row: 8, 16, 32, 64
-    constexpr int kCap = kFinStageBytes / (kPitch * 4);      // rows of partials the stage holds
     constexpr int kLanesPerRow = kPieces < 32 ? kPieces : 32;
     constexpr int kRowsPerIssue = 32 / kLanesPerRow;         // rows one cp.async of the warp covers
     constexpr int kIssuesPerRow = (kPieces + 31) / 32;
+    const uint32_t stage_addr = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
+    const int sub = lane / kLanesPerRow, piece = lane % kLanesPerRow;
+    for (int sl0 = 0; sl0 < G; sl0 += kRowsPerIssue) {
+        const int sl = sl0 + sub;
+        if (sl < G) {
+            const float *src = src_of(sl);
+#pragma unroll
+            for (int q = 0; q < kIssuesPerRow; ++q) {
+                const int off = 4 * (piece + 32 * q);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_addr + (sl * kPitch + off) * 4),
+                             "l"(src + off)
+                             : "memory");
+            }
+        }
+    }
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    if (!p.sentinel) return true;
+    const int written = (p.b + 31) & ~31;  // columns the epilogue stores
+    uint64_t t0 = 0;
+    for (;;) {
+        bool miss = false;
+        for (int sl0 = 0; sl0 < G; sl0 += kRowsPerIssue) {
+            const int sl = sl0 + sub;
+            if (sl < G) {
+#pragma unroll
+                for (int q = 0; q < kIssuesPerRow; ++q) {
+                    const int off = 4 * (piece + 32 * q);
+                    if (off < written) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(stage + sl * kPitch + off);
+                        if (v.x == kSlotEmpty || v.y == kSlotEmpty || v.z == kSlotEmpty || v.w == kSlotEmpty) {
+                            miss = true;
+                            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_addr +
+                                                                                           (sl * kPitch + off) * 4),
+                                         "l"(src_of(sl) + off)
+                                         : "memory");
+                        }
+                    }
+                }
+            }
+        }
+        if (!__any_sync(0xffffffffu, miss)) break;
+        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+        int stop = 0;
+        if (lane == 0) {
+            uint64_t now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            stop = (*abort_flag != 0) || (now - t0 > p.wait_limit_ns);
+            if (stop) *abort_flag = 1;
+        }
+        if (__shfl_sync(0xffffffffu, stop, 0)) return false;
+    }
+    return true;
+}
+
+// This lane's values of one staged partial row: the columns fin_col(lane, c).
+template <int NC>
+__device__ __forceinline__ void staged_row_values(const float *row, int lane, float (&v)[NC]) {
+    if (NC >= 4) {
+#pragma unroll
+        for (int h = 0; h < NC / 4; ++h) {
+            const float4 t = *reinterpret_cast<const float4 *>(row + 128 * h + 4 * lane);
+            v[4 * h] = t.x;
+            v[4 * h + 1] = t.y;
+            v[4 * h + 2] = t.z;
+            v[4 * h + 3] = t.w;
+        }
+    } else if (NC == 2) {
+        const float2 t = *reinterpret_cast<const float2 *>(row + 2 * lane);
+        v[0] = t.x;
+        v[NC - 1] = t.y;
+    } else {
+        v[0] = row[lane];
+    }
+}
+
+// One row with the partials staged through `stage` (kFinStageBytes of shared memory that only
+// this warp touches), a stage-full at a time, added from shared memory in ascending slot order
+// (A_T's partials, then A_R's).  A lane owns the columns fin_col(lane, c).  The partial slots of
+// the tensor-core modes have a row pitch of exactly 32 * NC floats.  `ok` = false (and nothing
+// to use) if the partial rows did not arrive in time.
+template <int NC>
+__device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const SideInfo sT, const SideInfo sR, int m,
+                                                      int i, int lane, float *stage, volatile int *abort_flag,
+                                                      bool &ok) {
+    constexpr int kPitch = 32 * NC;                          // floats per row of a partial
+    constexpr int kCap = kFinStageBytes / (kPitch * 4);      // rows of partials the stage holds
     const int b = p.b;
     double gT[NC], gR[NC];
 #pragma unroll
@@ -161,45 +260,21 @@ __device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const 
     const float *rowT = p.slots + (int64_t)sT.first_slot * p.slot_floats + sT.side_off + (int64_t)i * kPitch;
     const float *rowR = p.slots + (int64_t)sR.first_slot * p.slot_floats + sR.side_off + (int64_t)i * kPitch;
     const int nT = sT.n_slots, n_tot = sT.n_slots + sR.n_slots;
-    const uint32_t stage_addr = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
-    const int sub = lane / kLanesPerRow, piece = lane % kLanesPerRow;
+    ok = true;
     for (int s0 = 0; s0 < n_tot; s0 += kCap) {
         const int G = (n_tot - s0 < kCap) ? n_tot - s0 : kCap;
-        for (int sl0 = 0; sl0 < G; sl0 += kRowsPerIssue) {
-            const int sl = sl0 + sub;
-            if (sl < G) {
+        const int64_t slot_floats = p.slot_floats;
+        ok = fetch_partial_rows<NC>(
+            p, G,
+            [=](int sl) {
                 const int s = s0 + sl;
-                const float *src = (s < nT) ? rowT + (int64_t)s * p.slot_floats : rowR + (int64_t)(s - nT) * p.slot_floats;
-#pragma unroll
-                for (int q = 0; q < kIssuesPerRow; ++q) {
-                    const int off = 4 * (piece + 32 * q);
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_addr + (sl * kPitch + off) * 4),
-                                 "l"(src + off)
-                                 : "memory");
-                }
-            }
-        }
-        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-        __syncwarp();
+                return (s < nT) ? rowT + (int64_t)s * slot_floats : rowR + (int64_t)(s - nT) * slot_floats;
+            },
+            lane, stage, abort_flag);
+        if (!ok) return 0.0;
         for (int sl = 0; sl < G; ++sl) {
-            const float *row = stage + sl * kPitch;
             float v[NC];
-            if (NC >= 4) {
-#pragma unroll
-                for (int h = 0; h < NC / 4; ++h) {
-                    const float4 t = *reinterpret_cast<const float4 *>(row + 128 * h + 4 * lane);
-                    v[4 * h] = t.x;
-                    v[4 * h + 1] = t.y;
-                    v[4 * h + 2] = t.z;
-                    v[4 * h + 3] = t.w;
-                }
-            } else if (NC == 2) {
-                const float2 t = *reinterpret_cast<const float2 *>(row + 2 * lane);
-                v[0] = t.x;
-                v[NC - 1] = t.y;
-            } else {
-                v[0] = row[lane];
-            }
+            staged_row_values<NC>(stage + sl * kPitch, lane, v);
             if (s0 + sl < nT) {  // uniform over the warp
 #pragma unroll
                 for (int c = 0; c < NC; ++c) gT[c] += (double)v[c];
@@ -210,7 +285,7 @@ __device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const 
         }
         __syncwarp();  // everyone has read the stage before the next pass overwrites it
     }
-    // columns beyond b were never written by anyone: whatever was added there is dropped
+    // columns beyond b hold nothing of G: whatever was added there is dropped
 #pragma unroll
     for (int c = 0; c < NC; ++c)
         if (fin_col<NC>(lane, c) >= b) gT[c] = gR[c] = 0.0;
@@ -227,20 +302,18 @@ __device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const 
 
 // Slots per side in one chunk: half the stage each for T and R.
 template <int NC>
-__host__ __device__ constexpr int fin_chunk_slots() { return kFinStageBytes / (32 * NC * 4) / 2; }
+__host__ __device__ constexpr int fin_chunk_slots() { return kFinStageBytes / (32 * NC * 4) / 2; }  // = chunk_slots_of_mode
 // Doubles of scratch one (row, chunk) task leaves: both sides, this row, every column.
 template <int NC>
 __host__ __device__ constexpr int fin_chunk_doubles() { return 2 * 32 * NC; }
 
-// One warp: chunk `ch` of row i: fetch, add, store to scratch[(i * n_chunks + ch)].
+// One warp: chunk `ch` of row i: fetch, add, store to scratch[(i * n_chunks + ch)].  False if the
+// partial rows did not arrive in time.
 template <int NC>
-__device__ __forceinline__ void finalize_row_chunk(const FinCommon &p, const SideInfo &sT, const SideInfo &sR, int i,
-                                                   int ch, int n_chunks, int lane, float *stage) {
+__device__ __forceinline__ bool finalize_row_chunk(const FinCommon &p, const SideInfo &sT, const SideInfo &sR, int i,
+                                                   int ch, int n_chunks, int lane, float *stage,
+                                                   volatile int *abort_flag) {
     constexpr int kPitch = 32 * NC;
-    constexpr int kPieces = kPitch / 4;
-    constexpr int kLanesPerRow = kPieces < 32 ? kPieces : 32;
-    constexpr int kRowsPerIssue = 32 / kLanesPerRow;
-    constexpr int kIssuesPerRow = (kPieces + 31) / 32;
     constexpr int kChunk = fin_chunk_slots<NC>();
     const float *rowT = p.slots + (int64_t)sT.first_slot * p.slot_floats + sT.side_off + (int64_t)i * kPitch;
     const float *rowR = p.slots + (int64_t)sR.first_slot * p.slot_floats + sR.side_off + (int64_t)i * kPitch;
@@ -248,46 +321,20 @@ __device__ __forceinline__ void finalize_row_chunk(const FinCommon &p, const Sid
     const int nT = (sT.n_slots - t0 < kChunk) ? (sT.n_slots - t0 > 0 ? sT.n_slots - t0 : 0) : kChunk;
     const int nR = (sR.n_slots - r0 < kChunk) ? (sR.n_slots - r0 > 0 ? sR.n_slots - r0 : 0) : kChunk;
     const int G = nT + nR;
-    const uint32_t stage_addr = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
-    const int sub = lane / kLanesPerRow, piece = lane % kLanesPerRow;
-    for (int sl0 = 0; sl0 < G; sl0 += kRowsPerIssue) {
-        const int sl = sl0 + sub;
-        if (sl < G) {
-            const float *src = (sl < nT) ? rowT + (int64_t)(t0 + sl) * p.slot_floats
-                                         : rowR + (int64_t)(r0 + sl - nT) * p.slot_floats;
-#pragma unroll
-            for (int q = 0; q < kIssuesPerRow; ++q) {
-                const int off = 4 * (piece + 32 * q);
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_addr + (sl * kPitch + off) * 4),
-                             "l"(src + off)
-                             : "memory");
-            }
-        }
-    }
-    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-    __syncwarp();
+    const int64_t slot_floats = p.slot_floats;
+    if (!fetch_partial_rows<NC>(
+            p, G,
+            [=](int sl) {
+                return (sl < nT) ? rowT + (int64_t)(t0 + sl) * slot_floats : rowR + (int64_t)(r0 + sl - nT) * slot_floats;
+            },
+            lane, stage, abort_flag))
+        return false;
     double gT[NC], gR[NC];
 #pragma unroll
     for (int c = 0; c < NC; ++c) gT[c] = gR[c] = 0.0;
     for (int sl = 0; sl < G; ++sl) {
-        const float *row = stage + sl * kPitch;
         float v[NC];
-        if (NC >= 4) {
-#pragma unroll
-            for (int h = 0; h < NC / 4; ++h) {
-                const float4 t = *reinterpret_cast<const float4 *>(row + 128 * h + 4 * lane);
-                v[4 * h] = t.x;
-                v[4 * h + 1] = t.y;
-                v[4 * h + 2] = t.z;
-                v[4 * h + 3] = t.w;
-            }
-        } else if (NC == 2) {
-            const float2 t = *reinterpret_cast<const float2 *>(row + 2 * lane);
-            v[0] = t.x;
-            v[NC - 1] = t.y;
-        } else {
-            v[0] = row[lane];
-        }
+        staged_row_values<NC>(stage + sl * kPitch, lane, v);
         if (sl < nT) {
 #pragma unroll
             for (int c = 0; c < NC; ++c) gT[c] += (double)v[c];
@@ -303,6 +350,7 @@ __device__ __forceinline__ void finalize_row_chunk(const FinCommon &p, const Sid
         out[c * 32 + lane] = gT[c];
         out[(NC + c) * 32 + lane] = gR[c];
     }
+    return true;
 }
 
 // One warp, once all chunks of row i are in scratch and visible: add them in chunk order and

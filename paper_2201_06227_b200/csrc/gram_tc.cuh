@@ -20,6 +20,14 @@
 // always gets to this point after it, so every module is finished; and the result never
 // depends on which warp did what.
 //
+// The first task of every epilogue warp is planned on the host (Plan::first_task): no claim to
+// wait for.  Where that gives every row of the launch a warp of its own (Plan::validate_rows), the
+// finish does not go by the counters at all: a partial slot holds a bit pattern no value has
+// (kSlotEmpty) except between a launch's store and its read, so a warp fetches its row of every
+// partial until none of it is empty -- each 4-byte element is its own flag; no fence, no look
+// at a counter, no claim.  Such launches alternate between two sets of slots, and each puts
+// back to "empty", at its start, what the launch before wrote into the other set.
+//
 // Warp roles (448 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
 // owner, warps 2..13 = epilogue (TMEM -> registers -> global, then the finalisation); a warp
 // may read only the TMEM lane quarter (warp index mod 4), so three warps share each quarter
@@ -98,6 +106,11 @@ struct TcParams {
     uint32_t early_inputs;
     uint32_t test_stall;
     uint64_t wait_limit_ns;    // limit of every bounded wait of this launch (kWaitLimitNs, shorter for the hook)
+    uint4 *empty_ptr;          // the set of slots this launch does NOT use: what the launch before wrote there
+    uint32_t empty_n;          // ... is put back to kSlotEmpty at the start (empty_n 16-byte pieces; 0: nothing)
+    const int32_t *first_task; // [gridDim.x * kEpiWarps] the task each epilogue warp starts the finish with
+                               // ((module << 16) | task, -1: none), or nullptr; front-only: one table per front
+    int32_t first_stride;      // front-only: entries from one front's table to the next
     int32_t M;
     int32_t n_active;          // tensor-core modules this launch evaluates (front-only: 1)
     FinCommon fin;             // slots, sides, b, outputs, freezing-rule state
@@ -197,44 +210,39 @@ __device__ __forceinline__ bool next_chunk(int &k, int q, int lane, int b, float
     return false;
 }
 
-// What module m's row cursor counts up to: its b rows, or, when it is finished in two levels (a
-// module evaluated alone, cut into many partials, b <= 64), its (row, chunk) tasks.  (At b > 64 the
-// chunk sums are 2 to 4 KB per task and the scratch traffic eats the gain: measured 22 -> 22 us at
-// b = 128, 92 -> 98 us at b = 256, against 66 -> 55 us at b = 64 and 27 -> 23 us at b = 32.)
-template <int NC>
-__device__ __forceinline__ int module_tasks(const TcParams &p, int m) {
-    const int nT = p.fin.sides[2 * m].n_slots, nR = p.fin.sides[2 * m + 1].n_slots;
-    const int most = nT > nR ? nT : nR;
-    constexpr int kChunk = fin_chunk_slots<NC>();
-    if (NC <= 2 && p.n_active == 1 && p.fin.chunk_sums && most > kChunk)
-        return p.fin.b * ((most + kChunk - 1) / kChunk);
-    return p.fin.b;
+// Tasks of module m that its cursor hands out (the others have a warp each from the start).
+__device__ __forceinline__ int module_cursor_tasks(const TcParams &p, int m) {
+    const SideInfo si = p.fin.sides[2 * m];
+    return si.n_tasks - si.n_static;
 }
 
-// One warp: take rows of module m from its cursor until none is left.  The claim of the next
-// row is in flight while the current one is worked on; the rows' terms are delivered together.
-// `stage` is kFinStageBytes of shared memory for this warp alone.
+// One warp: do task `first` of module m (if not negative), then take tasks from the module's
+// cursor until none is left.  A task is a row of G, or -- a module evaluated alone and cut into many
+// partials at b <= 64, where one warp per row would add a hundred partial rows one after the
+// other with most warps idle -- a (row, chunk) pair (see finalize_row_chunk; measured 66 -> 55 us
+// at b = 64, 27 -> 23 us at b = 32; at b > 64 the chunk sums are 2 to 4 KB per task and the
+// scratch traffic eats the gain).  The claim of the next task is in flight while the current one
+// is worked on; the rows' terms are delivered together.  `stage` is kFinStageBytes of shared
+// memory for this warp alone.
 template <int NC>
-__device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int lane, float *stage) {
+__device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int lane, float *stage,
+                                                   volatile int *abort_flag, int first = -1) {
     const int b = p.fin.b;
     FinCounters *c = p.ctr + m;
     unsigned long long mine = 0;  // this warp's rows and their terms, packed (row_acc_of)
     int r = 0;
-    if (lane == 0) r = atomicAdd(&c->row_cursor, 1);
+    if (first < 0 && lane == 0) r = atomicAdd(&c->row_cursor, 1);
     const SideInfo sT = p.fin.sides[2 * m], sR = p.fin.sides[2 * m + 1];  // in flight with the claim
-    r = __shfl_sync(0xffffffffu, r, 0);
-    constexpr int kChunk = fin_chunk_slots<NC>();
-    const int most = sT.n_slots > sR.n_slots ? sT.n_slots : sR.n_slots;
-    if (NC <= 2 && p.n_active == 1 && p.fin.chunk_sums && most > kChunk) {
-        // A module evaluated alone: (row, chunk) tasks, see finalize_row_chunk.  The cursor counts
-        // tasks; task v is chunk v % n_chunks of row v / n_chunks.
-        const int n_chunks = (most + kChunk - 1) / kChunk;
-        const int n_tasks = b * n_chunks;
+    const int n_tasks = sT.n_tasks, n_static = sT.n_static;
+    r = (first < 0) ? n_static + __shfl_sync(0xffffffffu, r, 0) : first;
+    if (n_tasks > b) {
+        // (row, chunk) tasks: task v is chunk v % n_chunks of row v / n_chunks
+        const int n_chunks = n_tasks / b;
         while (r < n_tasks) {
             int r_next = 0;
             if (lane == 0) r_next = atomicAdd(&c->row_cursor, 1);
             const int row = r / n_chunks, ch = r % n_chunks;
-            finalize_row_chunk<NC>(p.fin, sT, sR, row, ch, n_chunks, lane, stage);
+            if (!finalize_row_chunk<NC>(p.fin, sT, sR, row, ch, n_chunks, lane, stage, abort_flag)) return;
             __threadfence();  // every lane's sums, before the count
             __syncwarp();
             int done = 0;
@@ -244,15 +252,17 @@ __device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int
                 __threadfence();
                 mine += row_acc_of(finalize_row_from_chunks<NC>(p.fin, m, row, n_chunks, lane));
             }
-            r = __shfl_sync(0xffffffffu, r_next, 0);
+            r = n_static + __shfl_sync(0xffffffffu, r_next, 0);
         }
     } else {
         while (r < b) {
             int r_next = 0;
             if (lane == 0) r_next = atomicAdd(&c->row_cursor, 1);
-            const double term = finalize_row_staged<NC>(p.fin, sT, sR, m, r, lane, stage);
+            bool ok;
+            const double term = finalize_row_staged<NC>(p.fin, sT, sR, m, r, lane, stage, abort_flag, ok);
+            if (!ok) return;
             mine += row_acc_of(term);
-            r = __shfl_sync(0xffffffffu, r_next, 0);
+            r = n_static + __shfl_sync(0xffffffffu, r_next, 0);
         }
     }
     if (mine == 0) return;
@@ -289,6 +299,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     const int lane = threadIdx.x & 31;
     int u_begin = 0, u_end = 0;
     bool all_frozen = false;  // front-only evaluation with nothing left to monitor
+    const int32_t *first_task = p.first_task;
     {
         const int32_t *cta_begin = p.cta_begin;
         if (p.front_word) {
@@ -296,6 +307,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             const int front = (int)(uint32_t)*reinterpret_cast<const volatile unsigned long long *>(p.front_word);
             all_frozen = (front >= p.M);
             cta_begin += (int64_t)(all_frozen ? 0 : front) * p.cta_stride;
+            if (first_task) first_task += (int64_t)(all_frozen ? 0 : front) * p.first_stride;
         }
         if (!all_frozen) {
             u_begin = cta_begin[blockIdx.x];
@@ -489,6 +501,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         const bool epi_leader = (threadIdx.x == 64);
         // asked for now, needed at the end of the launch
         const CtaHelp planned_help = p.cta_help ? p.cta_help[blockIdx.x] : CtaHelp{-1, 0};
+        const int my_first = (first_task && !all_frozen) ? first_task[blockIdx.x * kEpiWarps + (warp - 2)] : -1;
         uint32_t acc = 0, acc_phase = 0;
         bool aborted = false;
         bool prior_done = false;  // the launch before has ended: the shared workspace is ours
@@ -501,6 +514,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             int32_t *z = reinterpret_cast<int32_t *>(p.ctr_next);
             const int n = p.M * (int)(sizeof(FinCounters) / sizeof(int32_t));
             for (int i = blockIdx.x * kEpiThreads + (threadIdx.x - 64); i < n; i += gridDim.x * kEpiThreads) z[i] = 0;
+            // ... and the partial slots the launch before wrote and read are empty again for the
+            // launch after this one (this launch uses the other set)
+            const uint4 empty = make_uint4(kSlotEmpty, kSlotEmpty, kSlotEmpty, kSlotEmpty);
+            for (uint32_t i = blockIdx.x * kEpiThreads + (threadIdx.x - 64); i < p.empty_n; i += gridDim.x * kEpiThreads)
+                p.empty_ptr[i] = empty;
         };
         for (int ui = u_begin; ui < u_end; ++ui) {
             const Unit u = p.units[ui];
@@ -523,7 +541,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             while (have) {
                 ptx::tmem_ld_wait();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) v[c] = w[c];
+                for (int c = 0; c < 32; ++c) v[c] = (w[c] == kSlotEmpty) ? kCanonicalNan : w[c];  // never stored as a value
                 k += 3;
                 const bool have_next = detail::next_chunk<MODE>(k, q, lane, b, slot, nx);
                 if (have_next) ptx::tmem_ld_32x32(t_row + nx.col, w);
@@ -550,8 +568,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 acc_phase ^= 1u;
             }
 
-            // Publish the partial: every thread's stores, then one count for the unit.
-            __threadfence();
+            // Publish the partial: every thread's stores, then one count for the unit.  (Where the
+            // readers validate what they read, the count is a hint and needs no fence before it.)
+            if (!p.fin.sentinel) __threadfence();
             detail::epi_bar_sync();
             if (epi_leader) atomicAdd(&p.ctr[u.module].units_done, 1);
         }
@@ -569,12 +588,40 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             static_assert(kEpiWarps * kFinStageBytes <= Cfg::kStages * Cfg::kStageBytes, "ring too small to stage");
             float *stage = reinterpret_cast<float *>(smem_aligned + (warp - 2) * kFinStageBytes);
             ptx::fence_proxy_async();  // the ring was last touched by TMA and the tensor cores
-            // Planned help first: the last few warps of a CTA whose own module has warps to spare
+            // The task planned for this warp first (Plan::first_task): no cursor to ask, and no
+            // counter to wait for either -- the partial rows say themselves whether they are here.
+            if (my_first >= 0) {
+                const int fm = my_first >> 16;
+                bool go = true;
+                if (!p.fin.sentinel) {
+                    // ... by the counter, then: this task is nobody else's, so the wait is not a
+                    // courtesy and runs to the launch's limit
+                    const int total = p.fin.sides[2 * fm].module_units;
+                    const uint64_t t_wait = ptx::globaltimer_ns();
+                    int state = 0;  // 1 complete, 2 gave up
+                    while (state == 0) {
+                        if (lane == 0) {
+                            if (detail::ld_acquire(&p.ctr[fm].units_done) >= total)
+                                state = 1;
+                            else if (*abort_flag || ptx::globaltimer_ns() - t_wait > p.wait_limit_ns) {
+                                *abort_flag = 1;
+                                state = 2;
+                            }
+                        }
+                        state = __shfl_sync(0xffffffffu, state, 0);
+                        if (state == 0) __nanosleep(100);
+                    }
+                    go = (state == 1);
+                    __threadfence();
+                }
+                if (go) detail::finish_module_rows<Cfg::kNC>(p, fm, lane, stage, abort_flag, my_first & 0xffff);
+            }
+            // Planned help: the last few warps of a CTA whose own module has warps to spare
             // start with the rows of a module that is short of them (see CtaHelp), once that module
             // is complete; the wait for it is a courtesy like the others.
             {
                 const CtaHelp h = planned_help;
-                if (h.warps > 0 && warp - 2 >= kEpiWarps - h.warps) {
+                if (h.warps > 0 && warp - 2 >= kEpiWarps - h.warps && !(my_first >= 0 && (my_first >> 16) == h.module)) {
                     const int total = p.fin.sides[2 * h.module].module_units;
                     const uint64_t t_wait = ptx::globaltimer_ns();
                     int state = 0;  // 1 complete, 2 gave up
@@ -590,7 +637,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                     }
                     if (state == 1) {
                         __threadfence();
-                        detail::finish_module_rows<Cfg::kNC>(p, h.module, lane, stage);
+                        detail::finish_module_rows<Cfg::kNC>(p, h.module, lane, stage, abort_flag);
                     }
                 }
             }
@@ -608,12 +655,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 }
                 if (my_m >= 0) {
                     my_total = p.fin.sides[2 * my_m].module_units;
-                    my_tasks = detail::module_tasks<Cfg::kNC>(p, my_m);
+                    my_tasks = detail::module_cursor_tasks(p, my_m);
                     // With many CTAs on a module and few rows, most claims would find nothing and only
                     // crowd the cursor: as many warps of this CTA as its share of the rows (or of the
                     // (row, chunk) tasks), plus one.
                     const int ctas_on_m = Cfg::kStacked ? my_total : (my_total + 1) / 2;
-                    if (warp - 2 > (my_tasks + ctas_on_m - 1) / ctas_on_m) my_m = -1;
+                    if (my_tasks <= 0 || warp - 2 > (my_tasks + ctas_on_m - 1) / ctas_on_m) my_m = -1;
                 }
                 uint32_t pending = __ballot_sync(0xffffffffu, my_m >= 0);
                 uint64_t t_wait = ptx::globaltimer_ns();
@@ -632,7 +679,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                         const int pick = (int)__fns(cand, 0, 1 + (warp - 2) % __popc(cand));
                         const int m = __shfl_sync(0xffffffffu, my_m, pick);
                         __threadfence();
-                        detail::finish_module_rows<Cfg::kNC>(p, m, lane, stage);  // returns when no row is left to claim
+                        detail::finish_module_rows<Cfg::kNC>(p, m, lane, stage, abort_flag);  // returns when no row is left to claim
                         pending &= ~(1u << pick);
                         t_wait = ptx::globaltimer_ns();
                     } else if (pending) {
@@ -656,7 +703,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                     if (!si.tensor_core || si.module_units == 0) continue;
                     const int done = detail::ld_acquire(&p.ctr[mm].units_done);
                     const int cur = detail::ld_acquire(&p.ctr[mm].row_cursor);
-                    const int left = (done >= si.module_units) ? detail::module_tasks<Cfg::kNC>(p, mm) - cur : 0;
+                    const int left = (done >= si.module_units) ? si.n_tasks - si.n_static - cur : 0;
                     if (left > best_left) {
                         best_left = left;
                         best_m = mm;
@@ -673,7 +720,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 }
                 if (best_left < 2 * kEpiWarps) break;  // not worth a round trip: its own CTAs are about done
                 __threadfence();
-                detail::finish_module_rows<Cfg::kNC>(p, best_m, lane, stage);
+                detail::finish_module_rows<Cfg::kNC>(p, best_m, lane, stage, abort_flag);
             }
         }
     }

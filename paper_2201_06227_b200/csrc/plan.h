@@ -58,7 +58,9 @@ struct SideInfo {
     int32_t tensor_core;   // 1: the module's units belong to the tensor-core kernel, which also
                            //    finishes the module; 0: CUDA-core kernel + finalisation kernel
     int32_t module_units;  // work units of the whole module (both sides)
-    int32_t pad[2];
+    int32_t n_tasks;       // what the module's finish is cut into: its b rows, or (row, chunk) tasks
+    int32_t n_static;      // the first n_static tasks belong to warps named in Plan::first_task; the
+                           // module's cursor hands out the rest
 };
 
 // What one CTA of the tensor-core kernel reports about a launch: how long it streamed and how
@@ -110,7 +112,25 @@ struct Plan {
     std::vector<int32_t> cta_begin_simt;  // [n_ctas + 1] into units[n_units_tc ..), relative to 0
     std::vector<SideInfo> sides;    // [2 * M]
     std::vector<CtaHelp> cta_help;  // [n_ctas] which module some warps of the CTA lend a hand to first
+    // [n_ctas * warps_per_cta] the task an epilogue warp starts the finish with, without asking the
+    // module's cursor: (module << 16) | task, or -1
+    std::vector<int32_t> first_task;
+    // How the finish learns that a partial row has arrived.  false: from the units-done counter of
+    // its module, which a unit bumps after a fence.  true: from the row itself -- slots are
+    // "empty" (a bit pattern no value has) except between the store and the read of a launch, and
+    // the reader fetches until nothing it needs is empty.  That saves the fence, the look at the
+    // counter and the claim (2 to 3 us of a 10 to 40 us evaluation); it needs a second set of
+    // slots (a launch empties what the launch before wrote), so it is chosen for b <= 128, where
+    // the slots are small and the end of a launch is a large part of it, and where every task has
+    // a warp of its own from the start and its partial rows fit one pass of the warp's stage.
+    bool validate_rows = false;
 };
+
+// Bytes of shared memory one epilogue warp stages partial rows in at the end of a launch.
+constexpr int kFinStageBytes = 16384;
+// Two-level finish of a module evaluated alone (stacked modes): partial slots per side whose rows
+// one (row, chunk) task adds (half a stage per side).
+inline int chunk_slots_of_mode(int mode) { return kFinStageBytes / (pitch_of_mode(mode) * 4) / 2; }
 
 inline int64_t kblocks_of(int64_t d) { return (d + kKBlock - 1) / kKBlock; }
 
@@ -257,17 +277,78 @@ inline void plan_help(Plan &plan, int M, int b, int warps_per_cta) {
         lack[to] -= give;
     }
 }
+
+// The finish of each tensor-core module as tasks, and who starts with which (Plan::first_task).
+// A module evaluated alone in a stacked mode, cut into more partials per side than one chunk
+// holds, is finished in two levels if the caller has scratch for the chunk sums: its tasks are
+// (row, chunk) pairs, task v = chunk v % n_chunks of row v / n_chunks.  Otherwise a task is a row.
+// The warps of a CTA serve the modules it worked on in turn (warp w the (w mod j)-th of its j
+// modules), its planned-help warps the module they help; a module's tasks go to its servers one
+// each, warp 0 of every CTA first, so that they spread over the SMs.
+inline void plan_first_tasks(Plan &plan, int M, int b, int warps_per_cta, bool two_level_ok, bool static_tasks) {
+    const int n_ctas = plan.n_ctas;
+    plan.first_task.assign((size_t)n_ctas * warps_per_cta, -1);
+    int n_active = 0;
+    for (int m = 0; m < M; ++m)
+        if (plan.sides[2 * (size_t)m].tensor_core && plan.sides[2 * (size_t)m].module_units > 0) ++n_active;
+    for (int m = 0; m < M; ++m) {
+        SideInfo &t = plan.sides[2 * (size_t)m], &r = plan.sides[2 * (size_t)m + 1];
+        int tasks = b;
+        const int most = t.n_slots > r.n_slots ? t.n_slots : r.n_slots;
+        const int chunk = chunk_slots_of_mode(plan.mode);
+        if (two_level_ok && mode_is_stacked(plan.mode) && n_active == 1 && t.tensor_core && most > chunk)
+            tasks = b * ((most + chunk - 1) / chunk);
+        t.n_tasks = r.n_tasks = tasks;
+        t.n_static = r.n_static = 0;
+    }
+    plan.validate_rows = false;
+    if (!static_tasks) return;  // every task from the cursor
+    std::vector<std::vector<int32_t>> servers(M);
+    std::vector<std::vector<int>> mods(n_ctas);
+    for (int c = 0; c < n_ctas; ++c)
+        for (int u = plan.cta_begin_tc[c]; u < plan.cta_begin_tc[c + 1]; ++u) {
+            const int m = plan.units[u].module;
+            if (mods[c].empty() || mods[c].back() != m) mods[c].push_back(m);
+        }
+    for (int w = 0; w < warps_per_cta; ++w)
+        for (int c = 0; c < n_ctas; ++c) {
+            if (mods[c].empty()) continue;
+            const CtaHelp h = plan.cta_help.empty() ? CtaHelp{-1, 0} : plan.cta_help[c];
+            const int regular = warps_per_cta - (h.warps > 0 ? h.warps : 0);
+            const int m = (w >= regular) ? h.module : mods[c][(size_t)w % mods[c].size()];
+            if (m >= 0 && m < M) servers[m].push_back(c * warps_per_cta + w);
+        }
+    bool one_pass = true, all_static = true;
+    for (int m = 0; m < M; ++m) {
+        SideInfo &t = plan.sides[2 * (size_t)m], &r = plan.sides[2 * (size_t)m + 1];
+        if (!t.tensor_core || t.module_units == 0) continue;
+        int n = (int)servers[m].size();
+        if (n > t.n_tasks) n = t.n_tasks;
+        if (n > 0xffff) n = 0xffff;
+        for (int k = 0; k < n; ++k) plan.first_task[servers[m][k]] = (m << 16) | k;
+        t.n_static = r.n_static = n;
+        if (n < t.n_tasks) all_static = false;
+        int rows_per_task = t.n_slots + r.n_slots;  // partial rows a task fetches
+        if (t.n_tasks > b && rows_per_task > 2 * chunk_slots_of_mode(plan.mode)) rows_per_task = 2 * chunk_slots_of_mode(plan.mode);
+        if ((int64_t)rows_per_task * pitch_of_mode(plan.mode) * 4 > kFinStageBytes) one_pass = false;
+    }
+    // (measured slower that way: a row that takes several passes of the stage -- one big module
+    // alone at b = 128 -- 23.8 against 20.5 us; more rows than warps -- 27 modules at b = 128 --
+    // 40.2 against 38.5 us)
+    plan.validate_rows = n_active > 0 && plan.mode <= kSingle1 && one_pass && all_static;
+}
 }  // namespace detail
 
 // tc_ok[m]: 1 = module m takes the TMA + tcgen05 kernel, 0 = the CUDA-core kernel, 2 = module m
 // is not evaluated in this plan (no units, never finished).  weights: see split_tiles (applies
 // to the tensor-core split only).
 inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t *tc_ok, Plan &plan,
-                       const float *weights = nullptr, int warps_per_cta = 12) {
+                       const float *weights = nullptr, int warps_per_cta = 12, bool two_level_ok = false,
+                       bool static_tasks = true) {
     plan.mode = mode_of_b(b);
     plan.n_ctas = n_ctas;
     plan.units.clear();
-    plan.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, {0, 0}});
+    plan.sides.assign(2 * (size_t)M, SideInfo{0, 0, 0, 0, 0, 0, 0, 0});
     std::vector<detail::Tile> tc, simt;
     for (int m = 0; m < M; ++m) {
         if (tc_ok[m] == 2) continue;
@@ -303,6 +384,7 @@ inline void build_plan(int M, const int64_t *d, int b, int n_ctas, const uint8_t
         t.module_units = r.module_units = units;
     }
     detail::plan_help(plan, M, b, warps_per_cta);
+    detail::plan_first_tasks(plan, M, b, warps_per_cta, two_level_ok, static_tasks);
 }
 
 }  // namespace egeria

@@ -223,6 +223,28 @@ def test_nan_propagates_and_zero_rows_are_clamped():
     assert np.isnan(losses[0])
 
 
+@pytest.mark.parametrize("b,d", [(16, 256), (64, 64 * 148 * 3), (128, 4096)])
+def test_nan_of_any_bit_pattern_is_a_value_not_a_missing_row(b, d):
+    """The finish tells a partial row that has arrived from one that has not by its contents: the
+    bit pattern that means "not here yet" is a NaN.  Inputs that are NaNs with every payload bit set
+    (and infinities, whose products and differences are NaNs too) must come out as a NaN loss like
+    any other NaN -- not as a wait that runs out -- and leave the context as it was."""
+    at, ar = wl.make_pair(b, d, "normal", 0.2, seed=11 + b, device=DEV)
+    ctx = eg.Context([d], b, 5, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
+    good = ctx.egeria_sp_loss_batch([at], [ar]).cpu().numpy().copy()
+    for bits, where in ((-1, (1, 5)), (0x7F80, (0, 0)), (-128, (b - 1, d - 1))):   # 0xFFFF, +Inf, 0xFF80 = -Inf
+        n = at.clone()
+        n.view(torch.int16)[where] = bits
+        m = ar.clone()
+        m.view(torch.int16)[where] = bits
+        losses = ctx.egeria_sp_loss_batch([n], [m]).cpu().numpy()
+        assert ctx.egeria_device_status() == eg.OK
+        assert np.isnan(losses[0]), (hex(bits & 0xFFFF), losses)
+        again = ctx.egeria_sp_loss_batch([at], [ar]).cpu().numpy()
+        assert again.tobytes() == good.tobytes()
+    ctx.close()
+
+
 # ----------------------------------------------------------------------------- named workloads
 
 def test_tiny_workload_full():
@@ -416,26 +438,63 @@ def test_many_pointer_sets_enqueued_ahead_of_the_gpu():
 
 
 @pytest.mark.parametrize("kind", [1, 2])
-def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_recovers(kind):
+@pytest.mark.parametrize("b,ds", [(64, [64 * 148 * 40]), (128, [64 * 148 * 3] * 6), (128, [64 * 148 * 2] * 15),
+                                  (256, [64 * 148 * 8] * 3)])
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_recovers(kind, b, ds):
     """The give-up path of the evaluation kernel, in the form that returns: one hand-shake of the
     first thread block is left out for ONE launch whose waits are limited to a millisecond.  The
     kernel returns, the status word says EGERIA_ERR_TIMEOUT (once), and the next evaluation on
-    the same context matches the oracle."""
-    b, d = 64, 64 * 148 * 40                       # 40 blocks per thread block: more than the 12 pipeline stages
-    at, ar = wl.make_pair(b, d, "relu", 0.2, seed=4242, device=DEV)
-    ref = oracle.sp_loss(wl.bf16_bits(at), wl.bf16_bits(ar))
-    ctx = eg.Context([d], b, 5, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
-    good = ctx.egeria_sp_loss_batch([at], [ar]).cpu().numpy().copy()
-    assert_loss_close(good, [ref])
-    out = torch.full((1,), -5.0, dtype=torch.float32, device=DEV)
+    the same context matches the oracle.  Where the finish tells an arrived partial row by its
+    contents (the warps that wait for the first block's partial give up), and where it goes by the
+    unit counters (more rows than warps, or b = 256); the modules the first block did not work on
+    are finished all the same."""
+    # every thread block gets 36 to 60 blocks of 64 features: more than the 12 (6 at b = 256) pipeline stages
+    _, _, validate = eg.egeria_debug_plan_tasks(ds, b, 148)
+    assert validate == (b <= 128 and len(ds) < 15)
+    at, ar = [], []
+    for m, d in enumerate(ds):
+        t, r = wl.make_pair(b, d, "relu", 0.2, seed=4242 + m, device=DEV)
+        at.append(t)
+        ar.append(r)
+    ref = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+    ctx = eg.Context(ds, b, 5, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
+    good = ctx.egeria_sp_loss_batch(at, ar).cpu().numpy().copy()
+    assert_loss_close(good, ref)
+    out = torch.full((len(ds),), -5.0, dtype=torch.float32, device=DEV)
     ctx.egeria_debug_stall_next(kind)
-    ctx.egeria_sp_loss_batch([at], [ar], out)
+    ctx.egeria_sp_loss_batch(at, ar, out)
     assert ctx.egeria_device_status() == eg.ERR_TIMEOUT
-    assert float(out.cpu()[0]) == -5.0             # no loss was written by the launch that gave up
-    assert ctx.egeria_device_status() == eg.OK     # reported once; the counters start afresh
+    got = out.cpu().numpy()
+    assert got[0] == -5.0                          # no loss for the module the stalled block worked on
+    done = got != -5.0
+    assert got[done].tobytes() == good[done].tobytes()
+    assert ctx.egeria_device_status() == eg.OK     # reported once; counters and slots start afresh
     for _ in range(3):                             # both sets of progress counters come round
-        again = ctx.egeria_sp_loss_batch([at], [ar]).cpu().numpy()
+        again = ctx.egeria_sp_loss_batch(at, ar).cpu().numpy()
         assert again.tobytes() == good.tobytes()
+    ctx.check_device_status()
+    ctx.close()
+
+
+def test_the_two_ways_of_finishing_alternate_on_one_context():
+    """One context, evaluations that alternate between batch sizes at which the finish validates
+    partial rows by their contents (two sets of slots in turn, each launch emptying what the one
+    before wrote) and some at which it goes by the unit counters (b > 128: the slots stay as
+    written and are cleared before the next evaluation of the first kind), a CUDA-core module
+    among them: every evaluation against the oracle."""
+    ds = [4096] * 6 + [1001, 8192]
+    M = len(ds)
+    big = [wl.make_pair(160, d, "relu" if m % 2 else "normal", 0.1 + 0.02 * m, seed=600 + m, device=DEV) for m, d in enumerate(ds)]
+    assert not eg.egeria_debug_plan_tasks(ds, 160, 148)[2] and eg.egeria_debug_plan_tasks(ds, 24, 148)[2]
+    ctx = eg.Context(ds, 160, 5, 1e-3, device=DEV)
+    refs = {}
+    for rep, b in enumerate([160, 24, 24, 128, 160, 160, 24, 100, 64, 24, 130, 128]):
+        at = [t[:b].contiguous() for t, _ in big]
+        ar = [r[:b].contiguous() for _, r in big]
+        if b not in refs:
+            refs[b] = oracle.sp_loss_batch([wl.bf16_bits(t) for t in at], [wl.bf16_bits(r) for r in ar])
+        losses = ctx.egeria_sp_loss_batch(at, ar).cpu().numpy()
+        assert_loss_close(losses, refs[b], f"evaluation {rep} b={b}")
     ctx.check_device_status()
     ctx.close()
 

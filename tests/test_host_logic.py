@@ -237,3 +237,74 @@ def test_planned_help_goes_from_well_off_modules_to_needy_ones():
                                             weights=help_[donors, 1], minlength=len(d)))
     assert after.max() < 0.6 * rows_per_warp.max()                             # the worst module is much better off
     assert after.max() / after.min() < 1.6
+
+
+def test_first_tasks_of_the_finish_are_a_partition():
+    """Who starts the end of a launch with which task (Plan::first_task): every task with a warp of
+    its own is named exactly once, by a warp of a CTA that worked on the module (or lends it warps),
+    the tasks are spread over the CTAs, the cursor's share is the rest, and the choice of protocol
+    follows from it."""
+    for name, only in (("tiny", -1), ("bert_base", -1), ("resnet50", -1), ("resnet56", -1), ("gpt2_medium", -1),
+                       ("resnet50", 0), ("bert_base", 3), ("gpt2_medium", 0), ("resnet56", 26), ("resnet56", 0)):
+        w = wl.WORKLOADS[name]
+        d, n = list(w.d), 148
+        first, tasks, validate = eg.egeria_debug_plan_tasks(d, w.b, n, only)
+        help_ = eg.egeria_debug_plan_help(d, w.b, n) if only < 0 else np.full((n, 2), -1)
+        worked = [set() for _ in range(n)]
+        if only < 0:
+            for m, _, _, _, c in eg.egeria_debug_plan(d, w.b, n):
+                worked[c].add(int(m))
+        else:                                        # the module alone over all CTAs
+            for _, _, _, _, c in eg.egeria_debug_plan([d[only]], w.b, n):
+                worked[c].add(only)
+        seen = {}
+        for c in range(n):
+            for wp in range(12):
+                ft = int(first[c, wp])
+                if ft < 0:
+                    continue
+                m, t = ft >> 16, ft & 0xffff
+                assert m in worked[c] or (help_[c, 1] > 0 and m == help_[c, 0]), (name, c, wp, m)
+                assert (m, t) not in seen, (name, m, t)
+                seen[(m, t)] = c
+        active = [m for m in range(len(d)) if only < 0 or m == only]
+        for m in range(len(d)):
+            n_tasks, n_static = int(tasks[m, 0]), int(tasks[m, 1])
+            mine = sorted(t for (mm, t) in seen if mm == m)
+            if m not in active:
+                assert mine == []
+                continue
+            assert mine == list(range(n_static)), (name, m)
+            assert 0 < n_static <= n_tasks
+            assert n_tasks % w.b == 0
+            if n_tasks > w.b:                       # two levels: only a module alone, stacked modes
+                assert len(active) == 1 and w.b <= 64
+            ctas = {seen[(m, t)] for t in mine}
+            assert len(ctas) >= min(n_static, len([c for c in range(n) if m in worked[c]])) * 0.9   # spread
+        # partial rows announce themselves (no counters) at b <= 128 where every task has a warp of its
+        # own and its partial rows fit one pass of the warp's 16 KB stage
+        plan_units = eg.egeria_debug_plan(d, w.b, n) if only < 0 else eg.egeria_debug_plan([d[only]], w.b, n)
+        pitch = 32 if w.b <= 32 else 64 if w.b <= 64 else 128 if w.b <= 128 else 256
+        one_pass = True
+        for m in active:
+            mm = m if only < 0 else 0
+            rows = sum(2 if side == 2 else 1 for (um, side, _, _, _) in plan_units if um == mm)
+            if tasks[m, 0] > w.b:
+                rows = min(rows, 2 * (16384 // (pitch * 4) // 2))
+            one_pass = one_pass and rows * pitch * 4 <= 16384
+        every_task_static = all(tasks[m, 0] == tasks[m, 1] for m in active)
+        assert validate == (w.b <= 128 and one_pass and every_task_static), (name, only)
+        assert validate == (name in ("tiny", "bert_base", "resnet50") or (name, only) == ("resnet56", 26)), (name, only)
+        assert every_task_static == (name in ("tiny", "bert_base", "resnet50") or only >= 0), (name, only)
+
+
+def test_two_level_tasks_only_for_a_module_alone_at_small_b():
+    d = [64 * 148 * 40]
+    for b, two in ((8, True), (32, True), (64, True), (128, False), (256, False)):
+        first, tasks, validate = eg.egeria_debug_plan_tasks(d, b, 148)
+        assert (tasks[0, 0] > b) == two, b
+        if two:
+            chunk = 64 if b <= 32 else 32
+            assert tasks[0, 0] == b * -(-148 // chunk)
+    first, tasks, validate = eg.egeria_debug_plan_tasks(d + d, 32, 148)   # two modules: one level
+    assert tasks[0, 0] == 32 and tasks[1, 0] == 32
