@@ -141,12 +141,12 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
     if (flags & EGERIA_FLAG_KEEP_GRAMS) take((size_t)M * 2 * b_max * b_max * sizeof(float));
     {
         // scratch of the two-level finalisation (one module evaluated alone): rows x chunks x both
-        // sides x columns, float64; the chunk count is bounded by the units one module can have
+        // sides x columns, float64; a chunk has at least one slot per side, and two_level_chunks aims
+        // at kTwoLevelChunk of them
         size_t bytes = 0;
         for (int mode = 0; mode <= mode_of_b(b_max) && mode <= kStacked64; ++mode) {  // used at b <= 64 only
             const int nc = pitch_of_mode(mode) / 32;
-            const int chunk_slots = kFinStageBytes / (32 * nc * 4) / 2;
-            const size_t chunks = (size_t)(max_units(1, mode, kMaxCtas) + chunk_slots - 1) / chunk_slots;
+            const size_t chunks = (size_t)(max_units(1, mode, kMaxCtas) + kTwoLevelChunk - 1) / kTwoLevelChunk + 1;
             const size_t rows = (size_t)(pitch_of_mode(mode) < b_max ? pitch_of_mode(mode) : b_max);
             const size_t v = rows * chunks * 2 * 32 * nc * sizeof(double);
             if (v > bytes) bytes = v;

@@ -295,14 +295,14 @@ __device__ __forceinline__ double finalize_row_staged(const FinCommon &p, const 
 // ---- Two levels, for a module evaluated alone.  Such a module is cut over all CTAs, so a row of G
 // has a hundred or more partial rows per side, while there are far fewer rows than warps: one warp
 // per row would add them one after the other for tens of microseconds with most warps idle.
-// Instead a task is (row, chunk): a warp adds the row's partials of kChunk consecutive slots per
+// Instead a task is (row, chunk): a warp adds the row's partials of a few consecutive slots per
 // side (one pass of its stage) and leaves the two float64 sums in scratch; the warp that delivers
 // a row's last chunk adds the chunk sums in chunk order and finishes the row.  Which warp does
 // what does not change any sum, so the result is as reproducible as the one-level one.
 
-// Slots per side in one chunk: half the stage each for T and R.
+// Most slots per side in one chunk: half the stage each for T and R (chunk_slots_of_mode).
 template <int NC>
-__host__ __device__ constexpr int fin_chunk_slots() { return kFinStageBytes / (32 * NC * 4) / 2; }  // = chunk_slots_of_mode
+__host__ __device__ constexpr int fin_chunk_slots() { return kFinStageBytes / (32 * NC * 4) / 2; }
 // Doubles of scratch one (row, chunk) task leaves: both sides, this row, every column.
 template <int NC>
 __host__ __device__ constexpr int fin_chunk_doubles() { return 2 * 32 * NC; }
@@ -314,12 +314,12 @@ __device__ __forceinline__ bool finalize_row_chunk(const FinCommon &p, const Sid
                                                    int ch, int n_chunks, int lane, float *stage,
                                                    volatile int *abort_flag) {
     constexpr int kPitch = 32 * NC;
-    constexpr int kChunk = fin_chunk_slots<NC>();
+    const int chunk = chunk_slots(sT.n_slots > sR.n_slots ? sT.n_slots : sR.n_slots, n_chunks);  // <= fin_chunk_slots<NC>()
     const float *rowT = p.slots + (int64_t)sT.first_slot * p.slot_floats + sT.side_off + (int64_t)i * kPitch;
     const float *rowR = p.slots + (int64_t)sR.first_slot * p.slot_floats + sR.side_off + (int64_t)i * kPitch;
-    const int t0 = ch * kChunk, r0 = ch * kChunk;
-    const int nT = (sT.n_slots - t0 < kChunk) ? (sT.n_slots - t0 > 0 ? sT.n_slots - t0 : 0) : kChunk;
-    const int nR = (sR.n_slots - r0 < kChunk) ? (sR.n_slots - r0 > 0 ? sR.n_slots - r0 : 0) : kChunk;
+    const int t0 = ch * chunk, r0 = ch * chunk;
+    const int nT = (sT.n_slots - t0 < chunk) ? (sT.n_slots - t0 > 0 ? sT.n_slots - t0 : 0) : chunk;
+    const int nR = (sR.n_slots - r0 < chunk) ? (sR.n_slots - r0 > 0 ? sR.n_slots - r0 : 0) : chunk;
     const int G = nT + nR;
     const int64_t slot_floats = p.slot_floats;
     if (!fetch_partial_rows<NC>(

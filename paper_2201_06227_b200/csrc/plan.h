@@ -128,9 +128,23 @@ struct Plan {
 
 // Bytes of shared memory one epilogue warp stages partial rows in at the end of a launch.
 constexpr int kFinStageBytes = 16384;
-// Two-level finish of a module evaluated alone (stacked modes): partial slots per side whose rows
-// one (row, chunk) task adds (half a stage per side).
+// Two-level finish of a module evaluated alone (stacked modes).  A (row, chunk) task adds the
+// row's partials of `chunk` consecutive slots per side; at most half a stage per side:
 inline int chunk_slots_of_mode(int mode) { return kFinStageBytes / (pitch_of_mode(mode) * 4) / 2; }
+// How many chunks a row is cut into.  A task costs about a microsecond plus 60 ns per slot, the
+// second level 50 ns per chunk: about kTwoLevelChunk slots per chunk, fewer chunks if the tasks
+// would outnumber the warps of the grid, more if a chunk would not fit the stage.  1: one level.
+constexpr int kTwoLevelChunk = 8;
+inline int two_level_chunks(int mode, int most, int b, int total_warps) {
+    if (most <= 2 * kTwoLevelChunk) return 1;
+    int n = (most + kTwoLevelChunk - 1) / kTwoLevelChunk;
+    if (n > total_warps / b) n = total_warps / b;
+    const int cap = chunk_slots_of_mode(mode);
+    if (n < (most + cap - 1) / cap) n = (most + cap - 1) / cap;
+    return n < 1 ? 1 : n;
+}
+// Slots per side in one chunk when a row with `most` slots on its longer side is cut into n chunks.
+__host__ __device__ inline int chunk_slots(int most, int n_chunks) { return (most + n_chunks - 1) / n_chunks; }
 
 inline int64_t kblocks_of(int64_t d) { return (d + kKBlock - 1) / kKBlock; }
 
@@ -279,9 +293,9 @@ inline void plan_help(Plan &plan, int M, int b, int warps_per_cta) {
 }
 
 // The finish of each tensor-core module as tasks, and who starts with which (Plan::first_task).
-// A module evaluated alone in a stacked mode, cut into more partials per side than one chunk
-// holds, is finished in two levels if the caller has scratch for the chunk sums: its tasks are
-// (row, chunk) pairs, task v = chunk v % n_chunks of row v / n_chunks.  Otherwise a task is a row.
+// A module evaluated alone in a stacked mode and cut into many partials is finished in two
+// levels if the caller has scratch for the chunk sums (two_level_chunks): its tasks are (row,
+// chunk) pairs, task v = chunk v % n_chunks of row v / n_chunks.  Otherwise a task is a row.
 // The warps of a CTA serve the modules it worked on in turn (warp w the (w mod j)-th of its j
 // modules), its planned-help warps the module they help; a module's tasks go to its servers one
 // each, warp 0 of every CTA first, so that they spread over the SMs.
@@ -295,9 +309,8 @@ inline void plan_first_tasks(Plan &plan, int M, int b, int warps_per_cta, bool t
         SideInfo &t = plan.sides[2 * (size_t)m], &r = plan.sides[2 * (size_t)m + 1];
         int tasks = b;
         const int most = t.n_slots > r.n_slots ? t.n_slots : r.n_slots;
-        const int chunk = chunk_slots_of_mode(plan.mode);
-        if (two_level_ok && mode_is_stacked(plan.mode) && n_active == 1 && t.tensor_core && most > chunk)
-            tasks = b * ((most + chunk - 1) / chunk);
+        if (two_level_ok && mode_is_stacked(plan.mode) && n_active == 1 && t.tensor_core)
+            tasks = b * two_level_chunks(plan.mode, most, b, n_ctas * warps_per_cta);
         t.n_tasks = r.n_tasks = tasks;
         t.n_static = r.n_static = 0;
     }
@@ -329,7 +342,7 @@ inline void plan_first_tasks(Plan &plan, int M, int b, int warps_per_cta, bool t
         t.n_static = r.n_static = n;
         if (n < t.n_tasks) all_static = false;
         int rows_per_task = t.n_slots + r.n_slots;  // partial rows a task fetches
-        if (t.n_tasks > b && rows_per_task > 2 * chunk_slots_of_mode(plan.mode)) rows_per_task = 2 * chunk_slots_of_mode(plan.mode);
+        if (t.n_tasks > b) rows_per_task = 2 * chunk_slots(t.n_slots > r.n_slots ? t.n_slots : r.n_slots, t.n_tasks / b);
         if ((int64_t)rows_per_task * pitch_of_mode(plan.mode) * 4 > kFinStageBytes) one_pass = false;
     }
     // (measured slower that way: a row that takes several passes of the stage -- one big module
