@@ -77,7 +77,7 @@ struct TcCfg {
     static constexpr int kTmemCols = (MODE == kStacked32) ? 128 : (MODE == kSingle2 ? 512 : 256);
     static constexpr int kNC = (MODE == kStacked32) ? 1 : (MODE == kStacked64 ? 2 : (MODE == kSingle1 ? 4 : 8));
     static constexpr int kSmemBytes =
-        kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
+        kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kEpiWarps * 2 * (int)sizeof(SideInfo);
 };
 
 struct TcParams {
@@ -226,13 +226,15 @@ __device__ __forceinline__ int module_cursor_tasks(const TcParams &p, int m) {
 // memory for this warp alone.
 template <int NC>
 __device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int lane, float *stage,
-                                                   volatile int *abort_flag, int first = -1) {
+                                                   volatile int *abort_flag, int first = -1,
+                                                   const SideInfo *cached = nullptr) {
     const int b = p.fin.b;
     FinCounters *c = p.ctr + m;
     unsigned long long mine = 0;  // this warp's rows and their terms, packed (row_acc_of)
     int r = 0;
     if (first < 0 && lane == 0) r = atomicAdd(&c->row_cursor, 1);
-    const SideInfo sT = p.fin.sides[2 * m], sR = p.fin.sides[2 * m + 1];  // in flight with the claim
+    // (in flight with the claim; a first task's were fetched into shared memory long ago)
+    const SideInfo sT = cached ? cached[0] : p.fin.sides[2 * m], sR = cached ? cached[1] : p.fin.sides[2 * m + 1];
     const int n_tasks = sT.n_tasks, n_static = sT.n_static;
     r = (first < 0) ? n_static + __shfl_sync(0xffffffffu, r, 0) : first;
     if (n_tasks > b) {
@@ -294,6 +296,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
     volatile uint32_t *tmem_holder =
         reinterpret_cast<volatile uint32_t *>(bars + 2 * Cfg::kStages + 2 * Cfg::kAccStages);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+    // where the partials of each epilogue warp's first task are (two SideInfo per warp), fetched early
+    SideInfo *side_cache = reinterpret_cast<SideInfo *>(smem_aligned + Cfg::kStages * Cfg::kStageBytes + 256);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -502,6 +506,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         // asked for now, needed at the end of the launch
         const CtaHelp planned_help = p.cta_help ? p.cta_help[blockIdx.x] : CtaHelp{-1, 0};
         const int my_first = (first_task && !all_frozen) ? first_task[blockIdx.x * kEpiWarps + (warp - 2)] : -1;
+        if (my_first >= 0 && lane < 16)  // 64 bytes: both sides of the module
+            reinterpret_cast<int32_t *>(side_cache + 2 * (warp - 2))[lane] =
+                reinterpret_cast<const int32_t *>(p.fin.sides + 2 * (my_first >> 16))[lane];
         uint32_t acc = 0, acc_phase = 0;
         bool aborted = false;
         bool prior_done = false;  // the launch before has ended: the shared workspace is ours
@@ -614,7 +621,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                     go = (state == 1);
                     __threadfence();
                 }
-                if (go) detail::finish_module_rows<Cfg::kNC>(p, fm, lane, stage, abort_flag, my_first & 0xffff);
+                __syncwarp();
+                if (go)
+                    detail::finish_module_rows<Cfg::kNC>(p, fm, lane, stage, abort_flag, my_first & 0xffff,
+                                                         side_cache + 2 * (warp - 2));
             }
             // Planned help: the last few warps of a CTA whose own module has warps to spare
             // start with the rows of a module that is short of them (see CtaHelp), once that module
