@@ -243,6 +243,31 @@ def n_sets_for(w: wl.Workload) -> int:
     return min(16, max(2, int(np.ceil(8 * 126e6 / w.input_bytes))))
 
 
+def timed_batches(step_fn, stream, device, steps, reps=5, spin_s=0.1):
+    """Median over `reps` batches of `steps` evaluations of the device time per evaluation, after
+    `spin_s` seconds of the same evaluations untimed: a GPU that has idled (the oracle runs on the
+    host for seconds between workloads) takes its clocks up over tens of milliseconds, longer than
+    a batch of 10-microsecond evaluations lasts."""
+    t0 = time.perf_counter()
+    k = 0
+    while time.perf_counter() - t0 < spin_s:
+        for _ in range(steps):
+            step_fn(k)
+            k += 1
+        torch.cuda.synchronize(device)
+    out = []
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(reps):
+        ev0.record(stream)
+        for _ in range(steps):
+            step_fn(k)
+            k += 1
+        ev1.record(stream)
+        torch.cuda.synchronize(device)
+        out.append(ev0.elapsed_time(ev1) / steps)
+    return sorted(out)[len(out) // 2]
+
+
 def measure_other(eg, name, device, stream, steps, warmup, oracle_too=False, front_only=False):
     """Short device-timed run of another named workload (context for the headline line)."""
     w = wl.WORKLOADS[name]
@@ -258,23 +283,12 @@ def measure_other(eg, name, device, stream, steps, warmup, oracle_too=False, fro
     # the step time: the same inputs through a context without those events (they cost about as
     # much as the launch gap of a 20-microsecond kernel)
     ctx, step, outs, sets, l0 = time_workload(eg, w, device, steps, warmup, n_sets, stream, time_gram=False, sets=sets)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    for i in range(steps):
-        step(warmup + i)
-    ev1.record(stream)
-    torch.cuda.synchronize(device)
-    ms = ev0.elapsed_time(ev1) / steps
+    ms = timed_batches(lambda i: step(warmup + i), stream, device, steps)
     # the same with ONE input set evaluated again and again: for a workload that fits the 126 MB L2
     # (or nearly) the reads then come partly from L2 -- labelled as such, never the headline
     warm_ms = None
     if n_sets > 1:
-        ev0.record(stream)
-        for i in range(steps):
-            step(0)
-        ev1.record(stream)
-        torch.cuda.synchronize(device)
-        warm_ms = ev0.elapsed_time(ev1) / steps
+        warm_ms = timed_batches(lambda i: step(0), stream, device, steps, spin_s=0.02)
     ctx.check_device_status()
     ctx.close()
     peak, _ = hbm_peak()
@@ -289,12 +303,7 @@ def measure_other(eg, name, device, stream, steps, warmup, oracle_too=False, fro
     # the previous one finishes its modules; legitimate here, since no kernel writes the inputs)
     ctx, step, outs, sets, l0 = time_workload(eg, w, device, steps, warmup, n_sets, stream, time_gram=False, sets=sets,
                                               extra_flags=eg.FLAG_OVERLAP)
-    ev0.record(stream)
-    for i in range(steps):
-        step(warmup + i)
-    ev1.record(stream)
-    torch.cuda.synchronize(device)
-    ov_ms = ev0.elapsed_time(ev1) / steps
+    ov_ms = timed_batches(lambda i: step(warmup + i), stream, device, steps)
     ctx.check_device_status()
     ctx.close()
     out["overlapped"] = {"ms_per_step": ov_ms, "value": w.M / (ov_ms * 1e-3),
@@ -330,13 +339,8 @@ def measure_front_only(eg, w, device, stream, steps, warmup, full_ms):
     for _ in range(warmup + 12):
         ctx.plasticity_evaluate_raw(pa, pr, w.b, losses.data_ptr(), slopes.data_ptr(), mask.data_ptr(), sp)
     torch.cuda.synchronize(device)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    for _ in range(steps):
-        ctx.plasticity_evaluate_raw(pa, pr, w.b, losses.data_ptr(), slopes.data_ptr(), mask.data_ptr(), sp)
-    ev1.record(stream)
-    torch.cuda.synchronize(device)
-    ms = ev0.elapsed_time(ev1) / steps
+    ms = timed_batches(lambda i: ctx.plasticity_evaluate_raw(pa, pr, w.b, losses.data_ptr(), slopes.data_ptr(),
+                                                             mask.data_ptr(), sp), stream, device, steps)
     ctx.check_device_status()
     ctx.close()
     share = w.d[0] / w.sum_d
