@@ -385,7 +385,7 @@ def time_workload(eg, w, device, steps, warmup, n_sets, stream, time_gram=True, 
     # The first evaluations of a context measure each SM's streaming rate and the work split then
     # follows it; every input set's plan is rebuilt once after that.  Do that outside the timed region.
     done = warmup
-    for _ in range(4):          # three rounds of three measured evaluations, then the final rebuilds
+    for _ in range(5):          # four rounds of three measured evaluations, then the final rebuilds
         for i in range(max(3, n_sets)):
             step(done)
             done += 1

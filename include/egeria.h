@@ -73,7 +73,10 @@ enum {
      * a B200 do not all get the same share of HBM bandwidth, and the placement of
      * thread blocks on SMs repeats from launch to launch): three evaluations are
      * measured, the shares are set, and this is repeated twice under the new
-     * shares; after the ninth such evaluation the shares stay.  The shares decide
+     * shares; three more evaluations under the final shares then decide whether
+     * they stay (only if the slowest thread block streams at least 1 % faster than
+     * under equal shares; else the split goes back to equal ones).  After the
+     * twelfth such evaluation nothing changes any more.  The shares decide
      * how the fp32 partial sums are grouped, so with the adaptive split the
      * low-order bits of a loss can differ between evaluations across a change of
      * shares and from run to run; with this flag every evaluation of the same
@@ -333,9 +336,10 @@ int egeria_plasticity_window(const egeria_ctx *ctx);
 
 /* The per-thread-block shares of the adaptive split (see EGERIA_FLAG_EQUAL_SPLIT).
  * Copies up to max_weights of them to out_weights (host, may be NULL; 1.0 = the
- * equal share) and returns how many thread blocks the split is over once measured
- * rates are in use, 0 while the split is still (or for good) the equal one, -1 for
- * a NULL context.  Never waits for the device. */
+ * equal share) and returns how many thread blocks the split is over once rates have
+ * been measured (the shares are all 1.0 again if the measurement found them no better
+ * than equal ones), 0 while nothing has been measured (or with EGERIA_FLAG_EQUAL_SPLIT),
+ * -1 for a NULL context.  Never waits for the device. */
 int egeria_split_weights(egeria_ctx *ctx, float *out_weights, int max_weights);
 
 /* Test hook: copy the row-normalised similarity matrices of one module, as

@@ -25,7 +25,7 @@ constexpr int kMaxW = 2048;    // replay keeps 2 * W doubles in shared memory
 constexpr int kPlanSlots = 16; // device-side plans kept, keyed by (b, activation pointers)
 constexpr int kCalibLaunches = 3;  // launches whose per-CTA streaming rates set the split weights
 constexpr size_t kMaxTimedCalls = 4096;  // EGERIA_FLAG_TIME_GRAM: calls timed between two queries
-constexpr int kCalibRounds = 3;    // times the weights are re-measured under the split they produced
+constexpr int kCalibRounds = 3;    // times the weights are (re-)measured; one more round then decides whether they stay
 constexpr uint64_t kTestWaitLimitNs = 1000000ull;  // 1 ms: wait limit of a launch under egeria_debug_stall_next
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -264,6 +264,7 @@ struct egeria_ctx {
     // the same share of HBM bandwidth; the CTA -> SM placement repeats from launch to launch).
     std::vector<float> weights;
     std::vector<double> rate_sum;  // blocks per nanosecond of every CTA, summed over the later rounds
+    double makespan_equal = 0.0;   // longest streaming time of a CTA under the equal split (mean of the round's launches)
     int weights_version = 0;
     bool calibrated = false;   // no more measuring
     int calib_round = 0;
@@ -564,8 +565,10 @@ static void poll_calibration(egeria_ctx *ctx) {
     if (ctx->calibrated || !ctx->host_log || ctx->calib_enqueued < kCalibLaunches) return;
     const int n = ctx->n_ctas;
     std::vector<double> rate(n, 0.0);
+    double makespan = 0.0;  // the slowest CTA's streaming time, mean over the round's launches
     for (int k = 0; k < kCalibLaunches; ++k) {
         const volatile CtaLog *log = ctx->host_log + (size_t)k * kMaxCtas;
+        uint32_t longest = 0;
         for (int c = 0; c < n; ++c) {
             if (log[c].serial != ctx->calib_serial[k]) return;  // this copy has not landed yet
             const uint32_t ns = log[c].duration_ns, blocks = log[c].blocks;
@@ -574,7 +577,21 @@ static void poll_calibration(egeria_ctx *ctx) {
                 return;
             }
             rate[c] += (double)blocks / (double)ns;
+            if (ns > longest) longest = ns;
         }
+        makespan += (double)longest / kCalibLaunches;
+    }
+    if (ctx->calib_round == 0) ctx->makespan_equal = makespan;
+    if (ctx->calib_round >= kCalibRounds) {
+        // The verdict: this round ran under the final shares.  They stay only if the slowest CTA
+        // now finishes at least 1 % earlier than under the equal split; on a GPU whose SMs stream
+        // alike the measured rates are noise, and shares that follow noise lose to equal ones.
+        if (!(makespan < 0.99 * ctx->makespan_equal)) {
+            for (int c = 0; c < n; ++c) ctx->weights[c] = 1.0f;
+            ctx->weights_version++;
+        }
+        ctx->calibrated = true;
+        return;
     }
     // From the second round on the rates were measured under shares close to the final ones: keep
     // adding them up, so that the last word is an average over six launches, not three.
@@ -595,8 +612,7 @@ static void poll_calibration(egeria_ctx *ctx) {
     // Under the equal split the fast CTAs finish early and leave the slow ones more bandwidth, which
     // flatters the slow ones: measure again under the new shares, a few times.
     ctx->calib_round++;
-    ctx->calib_enqueued = 0;
-    if (ctx->calib_round >= kCalibRounds) ctx->calibrated = true;
+    ctx->calib_enqueued = 0;  // (after kCalibRounds rounds: one more, for the verdict above)
 }
 
 // The work split for b rows: all evaluated modules in one split, or (front-only) one split per

@@ -415,7 +415,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             constexpr uint32_t idesc64x64 = ptx::make_idesc_bf16_f32(64, 64);
             constexpr uint32_t idesc128 = ptx::make_idesc_bf16_f32(128, 128);
             constexpr uint32_t idesc256 = ptx::make_idesc_bf16_f32(128, 256);
-            const uint64_t t_entry = ptx::globaltimer_ns();
+            // start of the streaming the launch log reports: the arrival of the first stage (not the
+            // kernel's entry: a programmatic dependent enters while the launch before is still running
+            // and then waits for it, each CTA for a different time)
+            uint64_t t_entry = ptx::globaltimer_ns();
             uint32_t blocks_done = 0;
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
@@ -435,6 +438,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                         break;
                     }
                     ptx::tc_fence_after_sync();
+                    if (!any_mma && p.log) t_entry = ptx::globaltimer_ns();
                     if (stall_after_first_stage && any_mma) {  // stop here: no further stage is released
                         ok = false;
                         break;

@@ -67,7 +67,7 @@ struct SideInfo {
 // much.  The host turns the blocks-per-nanosecond of a few launches into the split weights.
 struct CtaLog {
     uint32_t serial;       // launch this entry belongs to
-    uint32_t duration_ns;  // kernel entry to last MMA issued
+    uint32_t duration_ns;  // arrival of the first stage to last MMA issued
     uint32_t blocks;       // 64-element blocks it processed
     uint32_t pad;
 };

@@ -302,9 +302,9 @@ def _sampled_check(name, full_modules, row_modules, rows):
         return losses
 
     first = check("equal split")
-    for _ in range(12):
+    for _ in range(15):
         ctx.egeria_plasticity_evaluate(at, ar)[0].cpu()       # .cpu() waits: the launch logs land
-    assert ctx.egeria_split_weights()[0] > 0                  # the shares now follow the measured rates
+    assert ctx.egeria_split_weights()[0] > 0                  # the shares were measured (and kept, or found no better than equal ones)
     settled = check("adaptive split")
     assert_loss_close(settled, first.astype(np.float64), f"{name} adaptive vs equal split")
     ctx.close()
@@ -724,7 +724,7 @@ def test_adaptive_split_keeps_the_result(b, ds):
     fixed.close()
     ctx = eg.Context(ds, b, 5, 1e-3, device=DEV)
     outs = []
-    for k in range(14):
+    for k in range(17):
         outs.append(ctx.egeria_sp_loss_batch(at, ar).cpu().numpy().copy())   # .cpu() waits: the logs have landed
     n, w = ctx.egeria_split_weights()
     assert n > 0 and len(w) == n
