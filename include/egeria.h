@@ -49,7 +49,8 @@ typedef enum {
     EGERIA_ERR_UNSUPPORTED_DEVICE = 3, /* current device is not compute capability 10.x */
     EGERIA_ERR_WORKSPACE = 4,          /* workspace NULL, misaligned or too small */
     EGERIA_ERR_CUDA = 5,               /* a CUDA runtime/driver call failed */
-    EGERIA_ERR_TIMEOUT = 6             /* a bounded device-side wait ran out (see egeria_device_status) */
+    EGERIA_ERR_TIMEOUT = 6,            /* a bounded device-side wait ran out (see egeria_device_status) */
+    EGERIA_ERR_CHECK = 7               /* checked build only: an index check inside a kernel failed (egeria_debug_check_record) */
 } egeria_status;
 
 enum {
@@ -360,6 +361,23 @@ egeria_status egeria_debug_plan(int M, const int64_t *d, int b, int n_ctas, int3
 egeria_status egeria_debug_plan_weighted(int M, const int64_t *d, int b, int n_ctas,
                                          const float *weights, int32_t *out_units, int max_units,
                                          int *n_units);
+
+/* 1 if this library was compiled with -DEGERIA_CHECKED (the build script makes such a second
+ * library, libegeria_checked.so), else 0.  In a checked build the kernels compare every index
+ * they take from a table in memory (unit table, slot ranges, first tasks, cursors) and every
+ * offset into a partial slot, a warp's staging area, the chunk-sum scratch or tensor memory
+ * with its bound before using it; a failed check records what it saw (the first failure
+ * wins), makes the kernel skip that access -- nothing traps -- and egeria_device_status then
+ * returns EGERIA_ERR_CHECK once.  It stands in for the memory-checking tools where those cannot
+ * be run, and costs a few per cent.  The paper has no counterpart. */
+int egeria_build_is_checked(void);
+
+/* Test hook: the record of the first failed check since the last egeria_device_status that
+ * reported one (host int32 [5]: which check -- 1 unit range, 2 unit, 3 tensor-memory columns,
+ * 4 slot store, 5 first task, 6 task, 7 fetch, 8 chunk sum, 9 stage, 10 emptied range --, the
+ * offending value's low and high words, thread block, thread); all zero if none.  Waits for
+ * the stream of the last call and clears the record. */
+egeria_status egeria_debug_check_record(egeria_ctx *ctx, int32_t *out_record);
 
 /* Test hook: the help planned for the end of a launch, pure host arithmetic.  The rows of a
  * module are finished by the warps of the thread blocks that worked on it, so a module that got

@@ -16,7 +16,9 @@ import torch
 
 _LIB_PATH = Path(__file__).resolve().parent / "libegeria.so"
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+_LIB_PATH_CHECKED = Path(__file__).resolve().parent / "libegeria_checked.so"
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_CHECK = range(8)
 FLAG_SIGNED_SLOPE, FLAG_FORCE_SIMT, FLAG_KEEP_GRAMS, FLAG_HOST_STAGING, FLAG_TIME_GRAM = 1, 2, 4, 8, 16
 FLAG_EQUAL_SPLIT, FLAG_AUTO_T, FLAG_FRONTMOST, FLAG_FRONT_ONLY, FLAG_OVERLAP = 32, 64, 128, 256, 512
 MAX_B = 256
@@ -32,7 +34,7 @@ EXPORTS = [
     "egeria_split_weights", "egeria_status_string", "egeria_bootstrap_step", "egeria_bootstrap_replay",
     "egeria_bootstrap_reset", "egeria_plasticity_state_bytes", "egeria_plasticity_export", "egeria_plasticity_import",
     "egeria_sp_loss_subset", "egeria_plasticity_evaluate_subset",
-    "egeria_sp_loss_static_status", "egeria_debug_stall_next", "egeria_debug_plan_help", "egeria_debug_plan_tasks", "egeria_plasticity_set_lr", "egeria_plasticity_restarts", "egeria_plasticity_replay_lr",
+    "egeria_sp_loss_static_status", "egeria_debug_stall_next", "egeria_debug_plan_help", "egeria_debug_plan_tasks", "egeria_build_is_checked", "egeria_debug_check_record", "egeria_plasticity_set_lr", "egeria_plasticity_restarts", "egeria_plasticity_replay_lr",
 ]
 
 
@@ -43,6 +45,15 @@ class EgeriaError(RuntimeError):
 
 
 _lib = None
+
+
+def use_checked_library(checked: bool = True) -> None:
+    """Switch this process to the checked build of the library (index checks inside the kernels,
+    see egeria_build_is_checked) or back.  Only with no Context open: a handle belongs to the
+    library that made it."""
+    global _lib, _LIB_PATH
+    _LIB_PATH = _LIB_PATH_CHECKED if checked else Path(__file__).resolve().parent / "libegeria.so"
+    _lib = None
 
 
 def lib() -> ctypes.CDLL:
@@ -98,6 +109,8 @@ def lib() -> ctypes.CDLL:
     L.egeria_debug_plan_tasks.argtypes = [ctypes.c_int, i64p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                           ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                                           ctypes.POINTER(ctypes.c_int)]
+    L.egeria_build_is_checked.argtypes = []
+    L.egeria_debug_check_record.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
     L.egeria_launch_count.argtypes = [vp]
     L.egeria_launch_count.restype = ctypes.c_int64
     L.egeria_status_string.argtypes = [ctypes.c_int]
@@ -453,6 +466,13 @@ class Context:
 
     def check_device_status(self) -> None:
         _check(self.egeria_device_status(), "egeria_device_status")
+
+    def egeria_debug_check_record(self) -> np.ndarray:
+        """The checked build's record of the first failed index check (five int32, all zero if none)."""
+        out = np.zeros(5, dtype=np.int32)
+        _check(lib().egeria_debug_check_record(self._h, out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))),
+               "egeria_debug_check_record")
+        return out
 
     def egeria_gram_kernel_time(self):
         """(total milliseconds, calls) of the Gram kernels since the last query."""

@@ -9,6 +9,7 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libegeria.so"
+LIB_CHECKED = HERE / "libegeria_checked.so"   # the same sources with -DEGERIA_CHECKED (csrc/check.cuh)
 SOURCES = [CSRC / "egeria_api.cu"]
 HEADERS = sorted(CSRC.glob("*.cuh")) + sorted(CSRC.glob("*.h")) + [HERE.parent / "include" / "egeria.h"]
 
@@ -18,29 +19,36 @@ NVCC_FLAGS = [
 ]
 
 
-def stale() -> bool:
-    if not LIB.exists():
+def stale(lib: Path = LIB) -> bool:
+    if not lib.exists():
         return True
-    t = LIB.stat().st_mtime
+    t = lib.stat().st_mtime
     return any(p.stat().st_mtime > t for p in SOURCES + HEADERS)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
-    """Build libegeria.so if missing or older than its sources.  Raises on failure."""
-    if not force and not stale():
-        return LIB
+def _compile(lib: Path, extra, verbose: bool) -> None:
     nvcc = os.environ.get("NVCC", "nvcc")
-    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = [nvcc, *NVCC_FLAGS, "-o", str(tmp), *map(str, SOURCES)]
+    tmp = lib.with_suffix(f".so.tmp{os.getpid()}")
+    cmd = [nvcc, *NVCC_FLAGS, *extra, "-o", str(tmp), *map(str, SOURCES)]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)
     if res.returncode != 0:
-        raise RuntimeError("nvcc failed building libegeria.so")
-    os.replace(tmp, LIB)
+        raise RuntimeError(f"nvcc failed building {lib.name}")
+    os.replace(tmp, lib)
+
+
+def build(force: bool = False, verbose: bool = False, checked: bool = True) -> Path:
+    """Build libegeria.so (and, unless checked=False, libegeria_checked.so) if missing or older than
+    the sources.  Raises on failure."""
+    if force or stale(LIB):
+        _compile(LIB, [], verbose)
+    if checked and (force or stale(LIB_CHECKED)):
+        _compile(LIB_CHECKED, ["-DEGERIA_CHECKED"], verbose)
     return LIB
 
 
 if __name__ == "__main__":
     build(force="--force" in sys.argv, verbose=True)
     print(LIB)
+    print(LIB_CHECKED)

@@ -65,6 +65,7 @@ struct Layout {
     size_t rule0, raw, plist, n_evals, counter, freeze_eval, last_slope, Tauto, smax, front, unfreeze, boot_raw,
         boot_plist, boot_ints, rule_end;
     size_t replay_raw, replay_plist;  // windows of egeria_plasticity_replay_lr ([M][W] doubles each)
+    size_t chunk_bytes;     // bytes of the chunk-sum scratch
     size_t slot_bytes_cap;  // bytes reserved for partial slots
     size_t slot_set_bytes;  // launches that validate partial rows by their contents (b <= 128) alternate
                             // between the sets [0, slot_set_bytes) and [slot_set_bytes, 2 slot_set_bytes)
@@ -151,6 +152,7 @@ static bool make_layout(int M, const int64_t *d, int b_max, int W, uint32_t flag
             const size_t v = rows * chunks * 2 * 32 * nc * sizeof(double);
             if (v > bytes) bytes = v;
         }
+        L.chunk_bytes = bytes;
         L.chunk = take(bytes);
     }
     size_t slot_bytes = 0, set_bytes = 0;
@@ -334,6 +336,7 @@ const char *egeria_status_string(egeria_status s) {
         case EGERIA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case EGERIA_ERR_CUDA: return "CUDA call failed";
         case EGERIA_ERR_TIMEOUT: return "bounded device-side wait ran out";
+        case EGERIA_ERR_CHECK: return "index check inside a kernel failed (checked build)";
     }
     return "unknown status";
 }
@@ -970,6 +973,9 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
     }
     fc.slots = slot_base;
     fc.slot_floats = slot_floats;
+    fc.status = ctx->at<int32_t>(L.status);
+    fc.slots_floats = (int64_t)((fc.sentinel ? L.slot_set_bytes : L.slot_bytes_cap) / sizeof(float));
+    fc.chunk_doubles = (int64_t)(L.chunk_bytes / sizeof(double));
     fc.sides = reinterpret_cast<const SideInfo *>(region + L.sides);
     fc.b = b;
     fc.out_losses = out_losses;
@@ -997,6 +1003,8 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         tp.first_stride = kMaxCtas * kEpiWarps;
         tp.empty_ptr = empty_ptr;
         tp.empty_n = empty_n;
+        tp.empty_floats = (int64_t)(L.slot_set_bytes / sizeof(float));
+        tp.n_units = front_only ? (int)P.units.size() : P.n_units_tc;
         tp.slots = slot_base;
         tp.status = ctx->at<int32_t>(L.status);
         FinCounters *sets = ctx->at<FinCounters>(L.fin_ctr);
@@ -1293,6 +1301,16 @@ egeria_status egeria_debug_stall_next(egeria_ctx *ctx, int kind) {
     return EGERIA_OK;
 }
 
+int egeria_build_is_checked(void) { return kCheckedBuild ? 1 : 0; }
+
+egeria_status egeria_debug_check_record(egeria_ctx *ctx, int32_t *out_record) {
+    if (!ctx || !out_record) return EGERIA_ERR_INVALID_ARG;
+    EG_CUDA(cudaStreamSynchronize(ctx->last_stream));
+    EG_CUDA(cudaMemcpy(out_record, ctx->ws + ctx->L.status + sizeof(int32_t), 5 * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    EG_CUDA(cudaMemset(ctx->ws + ctx->L.status + sizeof(int32_t), 0, 5 * sizeof(int32_t)));  // the next failure is recorded afresh
+    return EGERIA_OK;
+}
+
 egeria_status egeria_device_status(egeria_ctx *ctx) {
     if (!ctx) return EGERIA_ERR_INVALID_ARG;
     EG_CUDA(cudaStreamSynchronize(ctx->last_stream));
@@ -1309,6 +1327,7 @@ egeria_status egeria_device_status(egeria_ctx *ctx) {
         EG_CUDA(cudaMemset(ctx->ws + ctx->L.status, 0, sizeof(int32_t)));
     }
     if (word == kStatusTimeout) return EGERIA_ERR_TIMEOUT;
+    if (word == kStatusCheck) return EGERIA_ERR_CHECK;  // (what failed: egeria_debug_check_record)
     return word == 0 ? EGERIA_OK : EGERIA_ERR_CUDA;
 }
 
@@ -1350,7 +1369,7 @@ static StaticLayout static_layout() {
     L.cta_begin_simt = take((kStaticCtas + 1) * sizeof(int32_t));
     L.sides = take(2 * sizeof(SideInfo));
     L.rowloss = take(kMaxB * sizeof(double));
-    L.ticket = take(2 * sizeof(int32_t) + 2 * sizeof(FinCounters));  // [0] finalisation ticket, [1] status word,
+    L.ticket = take(8 * sizeof(int32_t) + 2 * sizeof(FinCounters));  // [0] finalisation ticket, [1] status word (+ the checked build's record),
                                                                      // then two sets of progress counters
     L.slots = take((size_t)max_units(1, kSingle1, kStaticCtas) * slot_floats_of_mode(kSingle1) * sizeof(float));
     L.total = off;
@@ -1451,7 +1470,7 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     memcpy(image + L.cta_begin_tc, P.cta_begin_tc.data(), P.cta_begin_tc.size() * sizeof(int32_t));
     memcpy(image + L.cta_begin_simt, P.cta_begin_simt.data(), P.cta_begin_simt.size() * sizeof(int32_t));
     memcpy(image + L.sides, P.sides.data(), P.sides.size() * sizeof(SideInfo));
-    EG_CUDA(cudaMemsetAsync(ws + L.ticket, 0, 2 * sizeof(int32_t) + 2 * sizeof(FinCounters), stream));
+    EG_CUDA(cudaMemsetAsync(ws + L.ticket, 0, 8 * sizeof(int32_t) + 2 * sizeof(FinCounters), stream));
     EG_CUDA(cudaMemcpyAsync(ws, image, L.rowloss, cudaMemcpyHostToDevice, stream));
     // A kernel that gives up (a bounded wait ran out) writes no loss: leave a NaN there for that case.
     EG_CUDA(cudaMemsetAsync(out_loss, 0xff, sizeof(float), stream));
@@ -1463,6 +1482,9 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
     fc.slot_floats = slot_floats;
     fc.sentinel = 0u;  // counters and fences say when a partial is complete: the scratch needs no preparation
     fc.wait_limit_ns = kWaitLimitNs;
+    fc.status = ticket + 1;
+    fc.slots_floats = (int64_t)max_units(1, kSingle1, kStaticCtas) * slot_floats_of_mode(kSingle1);
+    fc.chunk_doubles = 0;
     fc.sides = reinterpret_cast<const SideInfo *>(ws + L.sides);
     fc.b = b;
     fc.out_losses = out_loss;
@@ -1489,9 +1511,11 @@ extern "C" egeria_status egeria_sp_loss_static(void *cuda_stream, const void *At
         tp.first_stride = 0;
         tp.empty_ptr = nullptr;
         tp.empty_n = 0;
+        tp.empty_floats = 0;
+        tp.n_units = P.n_units_tc;
         tp.slots = reinterpret_cast<float *>(ws + L.slots);
         tp.status = ticket + 1;
-        tp.ctr = reinterpret_cast<FinCounters *>(ticket + 2);
+        tp.ctr = reinterpret_cast<FinCounters *>(ticket + 8);
         tp.ctr_next = tp.ctr + 1;
         tp.log = nullptr;
         tp.serial = 0;

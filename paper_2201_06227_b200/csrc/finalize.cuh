@@ -12,6 +12,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "check.cuh"
 #include "plan.h"
 #include "slope.cuh"
 
@@ -36,6 +37,9 @@ struct FinCommon {
     int64_t slot_floats;
     uint32_t sentinel;      // 1: a partial row has arrived when none of its elements is kSlotEmpty (no counters)
     uint64_t wait_limit_ns; // limit of the wait for partial rows that have not arrived
+    int32_t *status;        // device status word (and the checked build's record after it)
+    int64_t slots_floats;   // floats from `slots` to the end of the slots this launch may use
+    int64_t chunk_doubles;  // doubles in chunk_sums
     const SideInfo *sides;  // [2 * M]
     int32_t b;
     float *out_losses;      // [M]
@@ -166,6 +170,15 @@ __device__ __forceinline__ bool fetch_partial_rows(const FinCommon &p, int G, Sr
     constexpr int kIssuesPerRow = (kPieces + 31) / 32;
     const uint32_t stage_addr = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
     const int sub = lane / kLanesPerRow, piece = lane % kLanesPerRow;
+    if (!eg_check(G >= 0 && G * kPitch * 4 <= kFinStageBytes, p.status, kCheckFetch, G)) return false;
+    if (kCheckedBuild) {
+        bool inside = true;
+        for (int sl = lane; sl < G; sl += 32) {
+            const int64_t off = src_of(sl) - p.slots;
+            inside = inside && off >= 0 && off + kPitch <= p.slots_floats;
+        }
+        if (!eg_check(__all_sync(0xffffffffu, inside), p.status, kCheckFetch, -1)) return false;
+    }
     for (int sl0 = 0; sl0 < G; sl0 += kRowsPerIssue) {
         const int sl = sl0 + sub;
         if (sl < G) {
@@ -344,6 +357,9 @@ __device__ __forceinline__ bool finalize_row_chunk(const FinCommon &p, const Sid
         }
     }
     __syncwarp();  // the stage is free again
+    if (!eg_check(((int64_t)i * n_chunks + ch + 1) * fin_chunk_doubles<NC>() <= p.chunk_doubles && chunk <= fin_chunk_slots<NC>(),
+                  p.status, kCheckChunkSum, (int64_t)i * n_chunks + ch))
+        return false;
     double *out = p.chunk_sums + ((int64_t)i * n_chunks + ch) * fin_chunk_doubles<NC>();
 #pragma unroll
     for (int c = 0; c < NC; ++c) {  // [side][c][lane]: consecutive lanes, consecutive doubles

@@ -108,9 +108,11 @@ struct TcParams {
     uint64_t wait_limit_ns;    // limit of every bounded wait of this launch (kWaitLimitNs, shorter for the hook)
     uint4 *empty_ptr;          // the set of slots this launch does NOT use: what the launch before wrote there
     uint32_t empty_n;          // ... is put back to kSlotEmpty at the start (empty_n 16-byte pieces; 0: nothing)
+    int64_t empty_floats;      // floats in that set (the checked build compares empty_n with it)
     const int32_t *first_task; // [gridDim.x * kEpiWarps] the task each epilogue warp starts the finish with
                                // ((module << 16) | task, -1: none), or nullptr; front-only: one table per front
     int32_t first_stride;      // front-only: entries from one front's table to the next
+    int32_t n_units;           // entries of `units` (the checked build compares unit indices with it)
     int32_t M;
     int32_t n_active;          // tensor-core modules this launch evaluates (front-only: 1)
     FinCommon fin;             // slots, sides, b, outputs, freezing-rule state
@@ -237,6 +239,12 @@ __device__ __forceinline__ void finish_module_rows(const TcParams &p, int m, int
     const SideInfo sT = cached ? cached[0] : p.fin.sides[2 * m], sR = cached ? cached[1] : p.fin.sides[2 * m + 1];
     const int n_tasks = sT.n_tasks, n_static = sT.n_static;
     r = (first < 0) ? n_static + __shfl_sync(0xffffffffu, r, 0) : first;
+    if (!eg_check(n_static >= 0 && n_static <= n_tasks && n_tasks >= b && n_tasks % b == 0 && r >= 0 &&
+                      sT.n_slots >= 0 && sR.n_slots >= 0 && sT.first_slot >= 0 && sR.first_slot >= 0 &&
+                      ((int64_t)sT.first_slot + sT.n_slots) * p.fin.slot_floats <= p.fin.slots_floats &&
+                      ((int64_t)sR.first_slot + sR.n_slots) * p.fin.slot_floats <= p.fin.slots_floats,
+                  p.status, kCheckTask, ((long long)m << 32) | (uint32_t)r))
+        return;
     if (n_tasks > b) {
         // (row, chunk) tasks: task v is chunk v % n_chunks of row v / n_chunks
         const int n_chunks = n_tasks / b;
@@ -317,6 +325,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             u_begin = cta_begin[blockIdx.x];
             u_end = cta_begin[blockIdx.x + 1];
         }
+        if (!eg_check(u_begin >= 0 && u_begin <= u_end && u_end <= p.n_units, p.status, kCheckUnitRange,
+                      ((long long)u_begin << 32) | (uint32_t)u_end))
+            u_begin = u_end = 0;
     }
 
     // The launch after this one may begin (its CTAs get an SM when one of ours ends).  A front-only
@@ -359,6 +370,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             const int u_stop = (p.test_stall == 1 && blockIdx.x == 0) ? u_begin : u_end;  // test hook: no loads
             for (int ui = u_begin; ui < u_stop && ok; ++ui) {
                 const Unit u = p.units[ui];
+                if (!eg_check(u.module >= 0 && u.module < p.M && u.kb0 >= 0 && u.nkb >= 1 && u.side >= 0 && u.side <= 2,
+                              p.status, kCheckUnit, ui)) {
+                    ok = false;
+                    break;
+                }
                 const CUtensorMap *tm_t = p.tmaps + 2 * u.module;
                 const CUtensorMap *tm_r = tm_t + 1;
                 if (u.module != last_module) {
@@ -370,6 +386,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 const int kb_end = u.kb0 + u.nkb;
                 for (int kb = u.kb0; kb < kb_end; kb += Cfg::kKbPerStage) {
                     if (!ptx::mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u, abort_flag, p.wait_limit_ns)) {
+                        ok = false;
+                        break;
+                    }
+                    if (!eg_check(stage < (uint32_t)Cfg::kStages, p.status, kCheckStage, stage)) {
                         ok = false;
                         break;
                     }
@@ -510,7 +530,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
         // asked for now, needed at the end of the launch
         const CtaHelp planned_help = p.cta_help ? p.cta_help[blockIdx.x] : CtaHelp{-1, 0};
         const int my_first = (first_task && !all_frozen) ? first_task[blockIdx.x * kEpiWarps + (warp - 2)] : -1;
-        if (my_first >= 0 && lane < 16)  // 64 bytes: both sides of the module
+        if (my_first >= 0 && (!kCheckedBuild || (my_first >> 16) < p.M) && lane < 16)  // 64 bytes: both sides of the module
             reinterpret_cast<int32_t *>(side_cache + 2 * (warp - 2))[lane] =
                 reinterpret_cast<const int32_t *>(p.fin.sides + 2 * (my_first >> 16))[lane];
         uint32_t acc = 0, acc_phase = 0;
@@ -528,8 +548,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             // ... and the partial slots the launch before wrote and read are empty again for the
             // launch after this one (this launch uses the other set)
             const uint4 empty = make_uint4(kSlotEmpty, kSlotEmpty, kSlotEmpty, kSlotEmpty);
-            for (uint32_t i = blockIdx.x * kEpiThreads + (threadIdx.x - 64); i < p.empty_n; i += gridDim.x * kEpiThreads)
-                p.empty_ptr[i] = empty;
+            if (eg_check((int64_t)p.empty_n * 4 <= p.empty_floats, p.status, kCheckEmpty, p.empty_n))
+                for (uint32_t i = blockIdx.x * kEpiThreads + (threadIdx.x - 64); i < p.empty_n; i += gridDim.x * kEpiThreads)
+                    p.empty_ptr[i] = empty;
         };
         for (int ui = u_begin; ui < u_end; ++ui) {
             const Unit u = p.units[ui];
@@ -540,13 +561,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             }
             claim_workspace();  // the first unit's streaming is over by now; usually so is the launch before
             ptx::tc_fence_after_sync();
-            float *slot = p.slots + (int64_t)u.slot * p.fin.slot_floats;
+            const bool slot_ok = eg_check(u.slot >= 0 && ((int64_t)u.slot + 1) * p.fin.slot_floats <= p.fin.slots_floats &&
+                                              u.module >= 0 && u.module < p.M,
+                                          p.status, kCheckUnit, ui);
+            float *slot = p.slots + (int64_t)(slot_ok ? u.slot : 0) * p.fin.slot_floats;
             const uint32_t t_row = tmem_base + acc * Cfg::kAccCols + ((uint32_t)(q * 32) << 16);
             // This warp's share of the accumulator: 32 x 32 chunks part, part + 3, ...; the load of
             // the next chunk is in flight while the current one is stored.
             detail::Chunk ch, nx;
             int k = part;
-            bool have = detail::next_chunk<MODE>(k, q, lane, b, slot, ch);
+            bool have = slot_ok && detail::next_chunk<MODE>(k, q, lane, b, slot, ch);
             uint32_t v[32], w[32];
             if (have) ptx::tmem_ld_32x32(t_row + ch.col, w);
             while (have) {
@@ -556,6 +580,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
                 k += 3;
                 const bool have_next = detail::next_chunk<MODE>(k, q, lane, b, slot, nx);
                 if (have_next) ptx::tmem_ld_32x32(t_row + nx.col, w);
+                if (kCheckedBuild) {
+                    const int64_t off = ch.dst - slot;
+                    const bool fine = ch.col + 32 <= (uint32_t)Cfg::kAccCols &&
+                                      (!ch.valid || (off >= 0 && off + 32 <= p.fin.slot_floats));
+                    if (!eg_check(__all_sync(0xffffffffu, fine), p.status, ch.col + 32 <= (uint32_t)Cfg::kAccCols ? kCheckSlotStore : kCheckTmem, off))
+                        ch.valid = false;
+                }
                 if (ch.valid) {
 #pragma unroll
                     for (int c = 0; c < 32; c += 8) ptx::st_global_v8(ch.dst + c, v + c);
@@ -583,7 +614,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             // readers validate what they read, the count is a hint and needs no fence before it.)
             if (!p.fin.sentinel) __threadfence();
             detail::epi_bar_sync();
-            if (epi_leader) atomicAdd(&p.ctr[u.module].units_done, 1);
+            if (epi_leader && slot_ok) atomicAdd(&p.ctr[u.module].units_done, 1);
         }
         claim_workspace();  // (CTAs without a unit, and the counters' clearing if the wait above gave up)
         if (all_frozen && blockIdx.x == 0 && warp == 2) {
@@ -603,8 +634,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             // counter to wait for either -- the partial rows say themselves whether they are here.
             if (my_first >= 0) {
                 const int fm = my_first >> 16;
-                bool go = true;
-                if (!p.fin.sentinel) {
+                __syncwarp();  // (side_cache was written by lanes 0..15)
+                bool go = eg_check(fm < p.M && (my_first & 0xffff) < side_cache[2 * (warp - 2)].n_static &&
+                                       side_cache[2 * (warp - 2)].n_static <= side_cache[2 * (warp - 2)].n_tasks,
+                                   p.status, kCheckFirstTask, my_first);
+                if (go && !p.fin.sentinel) {
                     // ... by the counter, then: this task is nobody else's, so the wait is not a
                     // courtesy and runs to the launch's limit
                     const int total = p.fin.sides[2 * fm].module_units;

@@ -9,6 +9,11 @@ if str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
 
+def pytest_addoption(parser):
+    parser.addoption("--checked-library", action="store_true",
+                     help="run against libegeria_checked.so (index checks inside the kernels)")
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (sm_100a)")
 
@@ -32,3 +37,12 @@ def _built_library():
     """The CUDA library is built in-tree (nvcc cross-compiles without a GPU)."""
     from paper_2201_06227_b200 import build
     build.build()
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _which_library(request, _built_library):
+    """With --checked-library every test of the session talks to the checked build."""
+    if request.config.getoption("--checked-library"):
+        from paper_2201_06227_b200 import binding
+        binding.use_checked_library(True)
+        assert binding.lib().egeria_build_is_checked() == 1

@@ -1277,3 +1277,21 @@ def test_tiny_end_to_end_chain():
         assert bool(masks[-1]) == ref["converged"]
     ctx.check_device_status()
     ctx.close()
+
+
+def test_checked_build_finds_nothing_on_the_parity_cases():
+    """The second library the build makes (index checks inside the kernels: unit table, slot
+    ranges, first tasks, cursors, offsets into slots, stages, chunk scratch and tensor memory) runs
+    a cross-section of this file -- every kernel mode, both ways of finishing, two levels, front-only,
+    CUDA-core modules, the bounded waits -- in a process of its own: same results, and no check fires
+    (every test there ends with a status query, which would say EGERIA_ERR_CHECK)."""
+    import subprocess
+    import sys
+    assert eg.lib().egeria_build_is_checked() in (0, 1)
+    sel = ("single_module_tensor_core_path or cut_over_every_cta or many_modules or hundreds or two_ways or "
+           "bounded_wait or front_only or overlapped or resnet56_workload_full or bert_base_workload_full or "
+           "tiny_workload_full or nan_of_any or unfreez")
+    r = subprocess.run([sys.executable, "-m", "pytest", str(Path(__file__)), "-m", "gpu", "-x", "-q", "--checked-library",
+                        "-k", sel, "-p", "no:cacheprovider"], capture_output=True, text=True, cwd=str(Path(__file__).parent.parent))
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout and "failed" not in r.stdout
