@@ -25,10 +25,13 @@
  *     EGERIA_ERR_UNSUPPORTED_DEVICE or EGERIA_ERR_CUDA.
  *   - One context per stream; a context is not thread-safe.
  *   - A call on a context passes the kernel state that belongs to that call (which of two sets of
- *     progress counters to use, the serial number of the rule evaluation), and may
- *     enqueue small copies (a new work plan, the launch log of the adaptive split):
+ *     progress counters and of partial slots to use, the serial number of the rule evaluation),
+ *     and may enqueue small copies (a new work plan, the launch log of the adaptive split):
  *     enqueue every evaluation of a context through the library; replaying one from a
- *     captured CUDA graph would reuse that state and give wrong results.
+ *     captured CUDA graph would reuse that state and give wrong results.  The evaluation calls
+ *     (egeria_sp_loss_batch, egeria_plasticity_evaluate and their _subset and _host forms)
+ *     therefore return EGERIA_ERR_INVALID_ARG on a stream that is being captured, and record
+ *     nothing.
  */
 #ifndef EGERIA_H_
 #define EGERIA_H_

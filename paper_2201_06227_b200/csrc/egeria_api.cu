@@ -915,6 +915,14 @@ static egeria_status sp_loss_impl(egeria_ctx *ctx, void *cuda_stream, const void
         if ((reinterpret_cast<uintptr_t>(At[m]) | reinterpret_cast<uintptr_t>(Ar[m])) & 1) return EGERIA_ERR_INVALID_ARG;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    {
+        // An evaluation carries state that belongs to this one call (which set of counters and of
+        // partial slots, the rule's serial number): a graph would replay it with that state, and
+        // read the partial rows of the replay before as its own.  Turned away, nothing recorded.
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return EGERIA_ERR_CUDA;
+        if (capturing != cudaStreamCaptureStatusNone) return EGERIA_ERR_INVALID_ARG;
+    }
     ctx->last_stream = stream;
     egeria_status s = set_attrs(ctx);
     if (s != EGERIA_OK) return s;
@@ -1100,6 +1108,12 @@ egeria_status egeria_sp_loss_batch_host(egeria_ctx *ctx, void *cuda_stream, cons
     if (b < 2 || b > ctx->b_max) return EGERIA_ERR_INVALID_ARG;
     HostRange range("egeria_sp_loss_batch_host");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    {
+        // (the call synchronises the stream, which a capturing stream cannot do; and see sp_loss_impl)
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return EGERIA_ERR_CUDA;
+        if (capturing != cudaStreamCaptureStatusNone) return EGERIA_ERR_INVALID_ARG;
+    }
     for (int m = 0; m < ctx->M; ++m) {
         if (d[m] != ctx->d[m] || !At_host[m] || !Ar_host[m]) return EGERIA_ERR_INVALID_ARG;
         const size_t bytes = (size_t)b * d[m] * 2;

@@ -1279,6 +1279,38 @@ def test_tiny_end_to_end_chain():
     ctx.close()
 
 
+def test_an_evaluation_is_turned_away_from_a_capturing_stream():
+    """An evaluation carries per-call state (which set of counters and partial slots, the rule's
+    serial number); replayed from a graph it would be wrong without a sign.  On a capturing
+    stream the call returns EGERIA_ERR_INVALID_ARG, records nothing, and the context goes on."""
+    at, ar = wl.make_pair(48, 4096, "relu", 0.2, seed=77, device=DEV)
+    ctx = eg.Context([4096], 48, 5, 1e-3, eg.FLAG_EQUAL_SPLIT, device=DEV)
+    good = ctx.egeria_sp_loss_batch([at], [ar]).cpu().numpy().copy()
+    out = torch.full((1,), -3.0, dtype=torch.float32, device=DEV)
+    x = torch.zeros(4, device=DEV)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        g.capture_begin()
+        try:
+            x.add_(1.0)
+            with pytest.raises(eg.EgeriaError) as e:
+                ctx.egeria_sp_loss_batch([at], [ar], out, stream=side)
+        finally:
+            g.capture_end()
+    assert e.value.status == eg.ERR_INVALID_ARG
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    assert float(out.cpu()[0]) == -3.0 and float(x.cpu()[0]) == 1.0    # the graph holds the add and nothing of ours
+    again = ctx.egeria_sp_loss_batch([at], [ar]).cpu().numpy()
+    assert again.tobytes() == good.tobytes()
+    ctx.check_device_status()
+    ctx.close()
+
+
 def test_checked_build_finds_nothing_on_the_parity_cases():
     """The second library the build makes (index checks inside the kernels: unit table, slot
     ranges, first tasks, cursors, offsets into slots, stages, chunk scratch and tensor memory) runs
