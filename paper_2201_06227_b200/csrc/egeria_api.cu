@@ -586,7 +586,7 @@ static void poll_calibration(egeria_ctx *ctx) {
     }
     if (ctx->calib_round == 0) ctx->makespan_equal = makespan;
     if (ctx->calib_round >= kCalibRounds) {
-        // The verdict: this round ran under the final shares.  They stay only if the slowest CTA
+        // The decision: this round of launches ran under the final shares.  They stay only if the slowest CTA
         // now finishes at least 1 % earlier than under the equal split; on a GPU whose SMs stream
         // alike the measured rates are noise, and shares that follow noise lose to equal ones.
         if (!(makespan < 0.99 * ctx->makespan_equal)) {
@@ -615,7 +615,7 @@ static void poll_calibration(egeria_ctx *ctx) {
     // Under the equal split the fast CTAs finish early and leave the slow ones more bandwidth, which
     // flatters the slow ones: measure again under the new shares, a few times.
     ctx->calib_round++;
-    ctx->calib_enqueued = 0;  // (after kCalibRounds rounds: one more, for the verdict above)
+    ctx->calib_enqueued = 0;  // (after kCalibRounds rounds: one more, for the decision above)
 }
 
 // The work split for b rows: all evaluated modules in one split, or (front-only) one split per
