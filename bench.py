@@ -287,13 +287,14 @@ def measure_other(eg, name, device, stream, steps, warmup, oracle_too=False, fro
     # (a workload that keeps HBM busy for 0.2 ms a launch is timed in one batch, like the headline:
     # a tenth of a second of it brings the power cap in, and that is the sustained figure)
     small = w.input_bytes < 2e8
-    ms = timed_batches(lambda i: step(warmup + i), stream, device, steps, reps=5 if small else 1,
+    batch = max(steps, 200) if small else steps   # (a 20-step batch of 8 us evaluations is mostly its own start)
+    ms = timed_batches(lambda i: step(warmup + i), stream, device, batch, reps=5 if small else 1,
                        spin_s=0.1 if small else 0.0)
     # the same with ONE input set evaluated again and again: for a workload that fits the 126 MB L2
     # (or nearly) the reads then come partly from L2 -- labelled as such, never the headline
     warm_ms = None
     if n_sets > 1:
-        warm_ms = timed_batches(lambda i: step(0), stream, device, steps, spin_s=0.02)
+        warm_ms = timed_batches(lambda i: step(0), stream, device, batch, spin_s=0.02)
     ctx.check_device_status()
     ctx.close()
     peak, _ = hbm_peak()
@@ -308,7 +309,7 @@ def measure_other(eg, name, device, stream, steps, warmup, oracle_too=False, fro
     # the previous one finishes its modules; legitimate here, since no kernel writes the inputs)
     ctx, step, outs, sets, l0 = time_workload(eg, w, device, steps, warmup, n_sets, stream, time_gram=False, sets=sets,
                                               extra_flags=eg.FLAG_OVERLAP)
-    ov_ms = timed_batches(lambda i: step(warmup + i), stream, device, steps, reps=5 if small else 1,
+    ov_ms = timed_batches(lambda i: step(warmup + i), stream, device, batch, reps=5 if small else 1,
                           spin_s=0.1 if small else 0.0)
     ctx.check_device_status()
     ctx.close()
