@@ -177,8 +177,11 @@ __device__ __forceinline__ bool chunk_of(int k, int q, int lane, int b, float *s
         ch.valid = r < b;
         return true;
     } else if (MODE == kSingle1) {
-        const int r = q * 32 + lane, c0 = 32 * k;
-        if (k >= 4 || c0 >= b || q * 32 >= b) return false;
+        // pieces of 16 columns: eight of them split 3 + 3 + 2 over the quarter's three warps (four
+        // pieces of 32 would be 2 + 1 + 1, and the warp with two is what the others wait for);
+        // every piece up to b rounded up to 32 columns is stored, as in the other modes
+        const int r = q * 32 + lane, c0 = 16 * k;
+        if (k >= 8 || c0 >= ((b + 31) & ~31) || q * 32 >= b) return false;
         ch.col = c0;
         ch.dst = slot + r * 128 + c0;
         ch.valid = r < b;
@@ -206,7 +209,7 @@ __device__ __forceinline__ bool chunk_of(int k, int q, int lane, int b, float *s
 // First existing chunk among k, k + 3, k + 6, ... (k is advanced to it).  Warp-uniform.
 template <int MODE>
 __device__ __forceinline__ bool next_chunk(int &k, int q, int lane, int b, float *slot, Chunk &ch) {
-    constexpr int kChunks = (MODE == kStacked32) ? 1 : (MODE == kStacked64 ? 2 : (MODE == kSingle1 ? 4 : 12));
+    constexpr int kChunks = (MODE == kStacked32) ? 1 : (MODE == kStacked64 ? 2 : (MODE == kSingle1 ? 8 : 12));
     for (; k < kChunks; k += 3)
         if (chunk_of<MODE>(k, q, lane, b, slot, ch)) return true;
     return false;
@@ -572,24 +575,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             int k = part;
             bool have = slot_ok && detail::next_chunk<MODE>(k, q, lane, b, slot, ch);
             uint32_t v[32], w[32];
-            if (have) ptx::tmem_ld_32x32(t_row + ch.col, w);
+            constexpr int kCols = (MODE == kSingle1) ? 16 : 32;  // columns of one piece
+            auto load_piece = [&](uint32_t col) {
+                if (MODE == kSingle1)
+                    ptx::tmem_ld_32x16(t_row + col, w);
+                else
+                    ptx::tmem_ld_32x32(t_row + col, w);
+            };
+            if (have) load_piece(ch.col);
             while (have) {
                 ptx::tmem_ld_wait();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) v[c] = (w[c] == kSlotEmpty) ? kCanonicalNan : w[c];  // never stored as a value
+                for (int c = 0; c < kCols; ++c) v[c] = (w[c] == kSlotEmpty) ? kCanonicalNan : w[c];  // never stored as a value
                 k += 3;
                 const bool have_next = detail::next_chunk<MODE>(k, q, lane, b, slot, nx);
-                if (have_next) ptx::tmem_ld_32x32(t_row + nx.col, w);
+                if (have_next) load_piece(nx.col);
                 if (kCheckedBuild) {
                     const int64_t off = ch.dst - slot;
-                    const bool fine = ch.col + 32 <= (uint32_t)Cfg::kAccCols &&
-                                      (!ch.valid || (off >= 0 && off + 32 <= p.fin.slot_floats));
-                    if (!eg_check(__all_sync(0xffffffffu, fine), p.status, ch.col + 32 <= (uint32_t)Cfg::kAccCols ? kCheckSlotStore : kCheckTmem, off))
+                    const bool fine = ch.col + kCols <= (uint32_t)Cfg::kAccCols &&
+                                      (!ch.valid || (off >= 0 && off + kCols <= p.fin.slot_floats));
+                    if (!eg_check(__all_sync(0xffffffffu, fine), p.status, ch.col + kCols <= (uint32_t)Cfg::kAccCols ? kCheckSlotStore : kCheckTmem, off))
                         ch.valid = false;
                 }
                 if (ch.valid) {
 #pragma unroll
-                    for (int c = 0; c < 32; c += 8) ptx::st_global_v8(ch.dst + c, v + c);
+                    for (int c = 0; c < kCols; c += 8) ptx::st_global_v8(ch.dst + c, v + c);
                 }
                 if (MODE == kSingle2 && ch.mirror_c0 >= 0) {
                     // mirror G01 into the lower-left block: lanes write consecutive floats
@@ -743,7 +753,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const TcParams p
             // hand to the one with the most rows left.
             // (With fewer rows in all than half the epilogue warps of the grid there is nothing to
             // lend a hand with, and the look itself would be the last thing the kernel waits for.)
-            const int help_rounds = (2 * (int64_t)b * p.n_active < (int64_t)gridDim.x * kEpiWarps) ? 0 : 3;
+            // (Nor where every task had a warp of its own from the start: p.fin.sentinel.)
+            const int help_rounds =
+                (p.fin.sentinel || 2 * (int64_t)b * p.n_active < (int64_t)gridDim.x * kEpiWarps) ? 0 : 3;
             for (int round = 0; round < help_rounds; ++round) {
                 int best_left = 0, best_m = -1;
                 for (int mm = lane; mm < p.M; mm += 32) {
